@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the Hadamard-quantized layer forward on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic activations shaped like the
+transformer block and ResBlock convolution of a latent UNet at 32x32 latent, batch 32 (M = 32768 tokens /
+pixels per layer):
+    4 fused quantized linears  (QKV 512->1536, out-proj 512->512, FF1 512->2048, FF2 2048->512; Hadamard block = K)
+  + 1 fused quantized 3x3 conv (NHWC [32,32,32,256] x [256,3,3,256], stride 1, pad 1; Hadamard over Cin = 256)
+each as  online Hadamard transform -> INT4 quantize -> int8 tensor-core product with the folded (2-limb) weights of
+the Single-Hadamard scheme -> rescale + bias -> bf16.  W4A4.
+
+Prints ONE JSON line (see the keys below).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2512_05746_b200 import inputs  # noqa: E402
+
+METRIC = "int8 tensor TOPS (2*M*N*K*limbs) of the fused Hadamard-quant W4A4 linear+conv step"
+UNIT = "TOPS"
+M_TOKENS = 32768
+CONV = dict(Nb=32, H=32, W=32, C=256, Cout=256, R=3, S=3, stride=1, pad=1, had_block=256)
+WORKLOAD = ("configs[2] transformer-block linears (M=32768; QKV, out-proj, FF1, FF2) + configs[1] 3x3 conv at "
+            "batch 32 (M=32768, K=2304, N=256); W4A4, folded 2-limb weights, nibble codes, bf16 out")
+A_BITS, W_BITS = 4, 4
+
+
+def layer_list():
+    layers = []
+    for name, K, N, hb in inputs.TRANSFORMER_LINEARS:
+        layers.append(dict(kind="linear", name=name, M=M_TOKENS, K=K, N=N, had_block=hb))
+    c = CONV
+    layers.append(dict(kind="conv", name="conv3x3", M=c["Nb"] * c["H"] * c["W"], K=c["R"] * c["S"] * c["C"],
+                       N=c["Cout"], had_block=c["had_block"]))
+    return layers
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+
+
+# ------------------------------------------------------------------------------------------------ CUDA arm
+
+def build_layers(torch, hq, device, seed):
+    """Synthetic inputs and offline-prepared weights for every layer of the step, resident on `device`."""
+    layers = layer_list()
+    for i, L in enumerate(layers):
+        if L["kind"] == "linear":
+            cfg = inputs.config_transformer_linear(L["name"], M=L["M"], seed=seed)
+            x_host, w, b = cfg["x"], cfg["w"], cfg["bias"]
+        else:
+            c = CONV
+            cfg = inputs.config_conv_small(seed=seed, batch=c["Nb"])
+            x_host, w, b = cfg["x"], cfg["w"], cfg["bias"]
+        pw = hq.hq_weight_prepare(w, W_BITS, L["had_block"], hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE).to_device(device)
+        L["pw"] = pw
+        L["limbs"] = pw.desc.limbs
+        L["x_host"] = torch.from_numpy(x_host).pin_memory()
+        L["x"] = L["x_host"].to(device, non_blocking=True)
+        L["bias"] = torch.from_numpy(b).to(device)
+        rows, cols = (L["M"], L["K"]) if L["kind"] == "linear" else (L["M"], CONV["C"])
+        L["rows"], L["cols"] = rows, cols
+        ws_bytes = hq.hq_workspace_size(rows, cols, hq.HQ_CODES_NIBBLE)
+        L["ws"] = torch.empty((ws_bytes,), dtype=torch.uint8, device=device)
+        oshape = (L["M"], L["N"]) if L["kind"] == "linear" else (CONV["Nb"], CONV["H"], CONV["W"], CONV["Cout"])
+        L["y"] = torch.empty(oshape, dtype=torch.bfloat16, device=device)
+        L["y_host"] = torch.empty(oshape, dtype=torch.bfloat16).pin_memory()
+        L["ops"] = 2.0 * L["M"] * L["N"] * L["K"] * L["limbs"]
+        L["ops_1limb"] = 2.0 * L["M"] * L["N"] * L["K"]
+        # algorithmic HBM bytes of the two kernels (fp32 in, nibble codes out + scales; codes + weights in, bf16 out)
+        L["quant_bytes"] = rows * cols * 4.0 + rows * cols * 0.5 + rows * 4.0
+        L["gemm_bytes"] = (L["M"] * L["K"] * 0.5 if L["kind"] == "linear" else rows * cols * 0.5) + \
+            L["N"] * L["K"] * L["limbs"] + L["M"] * L["N"] * 2.0 + 4.0 * L["M"] + 8.0 * L["N"]
+        L["static_scale"] = None
+    torch.cuda.synchronize()
+    # The conv uses one static activation scale (the paper's learned per-tensor scale): calibrate it once with the
+    # library's own dynamic pass: S = max over pixels of the per-pixel scale.
+    for L in layers:
+        if L["kind"] == "conv":
+            x2d = L["x"].view(L["rows"], L["cols"])
+            pitch = L["cols"] // 2
+            codes = torch.empty((L["rows"], pitch), dtype=torch.uint8, device=device)
+            scales = torch.empty((L["rows"],), dtype=torch.float32, device=device)
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales)
+            L["static_scale"] = scales.max().reshape(1).contiguous()
+    torch.cuda.synchronize()
+    return layers
+
+
+def run_step(hq, layers, status, stream=None):
+    for L in layers:
+        if L["kind"] == "linear":
+            hq.hq_qlinear(L["x"], L["pw"], L["bias"], A_BITS, L["y"], L["ws"], dev_status=status, stream=stream)
+        else:
+            c = CONV
+            hq.hq_qconv(L["x"], L["pw"], c["R"], c["S"], c["stride"], c["pad"], L["bias"], A_BITS, L["y"], L["ws"],
+                        static_scale=L["static_scale"], dev_status=status, stream=stream)
+
+
+def run_step_split(torch, hq, layers, status, evs):
+    """Same kernels as run_step, launched through the unfused entry points with an event between them."""
+    stream = torch.cuda.current_stream()
+    for L in layers:
+        rows, cols = L["rows"], L["cols"]
+        pitch = cols // 2
+        codes = L["ws"][: rows * pitch].view(rows, pitch)
+        off = (rows * pitch + 255) // 256 * 256
+        scales = L["ws"][off: off + rows * 4].view(torch.float32)
+        x2d = L["x"].view(rows, cols)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        if L["kind"] == "linear":
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales)
+            e1.record(stream)
+            hq.hq_qgemm(codes, hq.HQ_CODES_NIBBLE, A_BITS, L["K"], L["pw"], scale_a=scales, bias=L["bias"],
+                        alpha=L["pw"].alpha, y=L["y"], dev_status=status)
+        else:
+            c = CONV
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales[:1],
+                                 static_scale=L["static_scale"])
+            e1.record(stream)
+            hq.hq_qconv2d(codes, hq.HQ_CODES_NIBBLE, A_BITS, c["Nb"], c["H"], c["W"], c["C"], L["pw"], c["R"], c["S"],
+                          c["stride"], c["pad"], scale_a=L["static_scale"], bias=L["bias"], alpha=L["pw"].alpha,
+                          y=L["y"], dev_status=status)
+        e2.record(stream)
+        evs.append((L, e0, e1, e2))
+
+
+def oracle_sample_step(orc, sample_rows, seed):
+    """One bounded sample of the step on the CPU oracle; returns (ops done, seconds)."""
+    ops, t0 = 0.0, time.perf_counter()
+    for name, K, N, hb in inputs.TRANSFORMER_LINEARS:
+        cfg = inputs.config_transformer_linear(name, M=sample_rows, seed=seed)
+        out = orc.qlinear(cfg["x"], cfg["w"], cfg["bias"], a_bits=A_BITS, w_bits=W_BITS, had_block=hb,
+                          weight_mode="folded")
+        ops += 2.0 * sample_rows * N * K * 2
+        del out
+    c = CONV
+    cfg = inputs.config_conv_small(seed=seed, batch=max(1, sample_rows // (c["H"] * c["W"])))
+    nb = cfg["x"].shape[0]
+    orc.qconv(cfg["x"], cfg["w"], cfg["bias"], a_bits=A_BITS, w_bits=W_BITS, had_block=c["had_block"], stride=1, pad=1,
+              weight_mode="folded", static_scale=0.5)
+    ops += 2.0 * nb * c["H"] * c["W"] * c["Cout"] * c["R"] * c["S"] * c["C"] * 2
+    return ops, time.perf_counter() - t0
+
+
+def cpu_baseline(sample_rows=256, seed=0):
+    import oracle as orc
+    orc.lib()
+    ops, sec = oracle_sample_step(orc, sample_rows, seed)
+    return dict(value=ops / sec / 1e12, unit=UNIT, cores=orc.num_threads(), kind="oracle",
+                sample=f"{sample_rows} of {M_TOKENS} rows of each linear and {max(1, sample_rows // 1024)} of 32 images "
+                       f"of the conv, whole oracle layer (dense Hadamard, quantize, weight prep, triple-loop product, "
+                       f"rescale); {sec:.1f} s")
+
+
+def main_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle as orc
+    orc.lib()
+    sample_rows = 256
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(orc, 64, 0)
+    tot_ops, tot_sec = 0.0, 0.0
+    for _ in range(args.steps):
+        ops, sec = oracle_sample_step(orc, sample_rows, 0)
+        tot_ops += ops
+        tot_sec += sec
+    value = tot_ops / tot_sec / 1e12
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=tot_sec / args.steps * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="int64", data="synthetic",
+                config=dict(workload=WORKLOAD, sample=f"{sample_rows} rows per layer per step"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=orc.num_threads(), kind="oracle",
+                                  sample=f"{sample_rows} rows per layer per step"),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return main_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2512_05746_b200 import binding as hq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    warmup = max(args.warmup, 3)
+    layers = build_layers(torch, hq, device, seed=rank)
+    status = torch.zeros((1,), dtype=torch.int32, device=device)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident throughput ---------------------------------------------------------------
+    for _ in range(warmup):
+        run_step(hq, layers, status)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        run_step(hq, layers, status)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    hq.hq_check_status(status)
+
+    # ---- per-kernel attribution (same kernels, events between the two launches of each layer) -----------
+    evs = []
+    for _ in range(args.steps):
+        run_step_split(torch, hq, layers, status, evs)
+    torch.cuda.synchronize()
+    per = {}
+    for L, a, b, c in evs:
+        d = per.setdefault(L["name"], dict(quant_ms=0.0, gemm_ms=0.0, n=0, L=L))
+        d["quant_ms"] += a.elapsed_time(b)
+        d["gemm_ms"] += b.elapsed_time(c)
+        d["n"] += 1
+
+    # ---- end to end: pinned host input -> device -> fused call -> host output -----------------------
+    e2e_steps = max(2, min(args.steps, 5))
+    h2d = sum(L["x_host"].numel() * L["x_host"].element_size() for L in layers)
+    d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in layers)
+
+    def e2e_step():
+        for L in layers:
+            L["x"].copy_(L["x_host"], non_blocking=True)
+        run_step(hq, layers, status)
+        for L in layers:
+            L["y_host"].copy_(L["y"], non_blocking=True)
+
+    e2e_step()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    f1.record(stream)
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+
+    ops_step = sum(L["ops"] for L in layers)
+    ops_step_1 = sum(L["ops_1limb"] for L in layers)
+    value = ops_step * args.steps * world / (ms * 1e-3) / 1e12
+    e2e_value = ops_step * e2e_steps * world / (e2e_ms * 1e-3) / 1e12
+
+    if rank == 0:
+        pk = peaks()
+        int8_peak = 2.0 * pk["bf16_sustained"]          # int8 : bf16 nominal dense ratio is 2 (4.5 : 2.25 PFLOP/s)
+        dom = max(per.values(), key=lambda d: d["gemm_ms"])      # dominant kernel: the longest GEMM launch
+        L = dom["L"]
+        gemm_ms = dom["gemm_ms"] / dom["n"]
+        ach = L["ops"] / (gemm_ms * 1e-3) / 1e12
+        roofline = dict(bound="tensor", kernel=f"qgemm_kernel<nibble> ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
+                                                f"limbs={L['limbs']})",
+                        achieved=ach, peak=int8_peak, unit="TOPS", frac=ach / int8_peak, traffic=None,
+                        peak_source=f"2 x bf16 sustained ({pk['source']})", launch_ms=gemm_ms)
+        qd = max(per.values(), key=lambda d: d["quant_ms"])
+        q_ms = qd["quant_ms"] / qd["n"]
+        q_gbs = qd["L"]["quant_bytes"] / (q_ms * 1e-3) / 1e9
+        roofline_quant = dict(bound="hbm", kernel=f"fwht_quant_fast ({qd['L']['name']}: {qd['L']['rows']}x{qd['L']['cols']})",
+                              achieved=q_gbs, peak=pk["hbm_gbs"], unit="GB/s", frac=q_gbs / pk["hbm_gbs"], traffic=None,
+                              peak_source=f"copy bandwidth ({pk['source']})", launch_ms=q_ms)
+        per_layer = {k: dict(quant_ms=d["quant_ms"] / d["n"], gemm_ms=d["gemm_ms"] / d["n"],
+                             gemm_tops=d["L"]["ops"] / (d["gemm_ms"] / d["n"] * 1e-3) / 1e12,
+                             quant_gbs=d["L"]["quant_bytes"] / (d["quant_ms"] / d["n"] * 1e-3) / 1e9)
+                     for k, d in per.items()}
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=warmup,
+                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype="int8", data="synthetic",
+                    config=dict(workload=WORKLOAD, l2="inputs larger than L2 (0.5 GB read per step)",
+                                tops_1limb_equiv=ops_step_1 * args.steps * world / (ms * 1e-3) / 1e12,
+                                layers_per_s=len(layers) * args.steps * world / (ms * 1e-3)),
+                    clocks=clocks, gpu_launches=2 * len(layers) * args.steps,
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                             steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
+                    roofline=roofline, roofline_fwht_quant=roofline_quant, per_layer=per_layer)
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

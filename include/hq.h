@@ -1,0 +1,163 @@
+/*
+ * hq.h -- C ABI of the B200 (sm_100a) Hadamard-quantized layer forward.
+ *
+ * The operations are the ones HQ-DM states for a quantized linear / convolution layer:
+ *   online Hadamard transform of the activations (Eq. 10, with H_k of Eq. 5-7)
+ *   -> symmetric quantization to N-bit integer codes with a floating-point scale (Eq. 3)
+ *   -> integer matrix product / convolution with offline-prepared integer weights (Eq. 12, Eq. 14)
+ *   -> rescale by S_XH * S_W in front of the integer product (Eq. 12, Eq. 14), plus bias.
+ *
+ * Conventions (all entry points):
+ *   - Return value is an hq_status; nothing throws, prints or allocates device memory.
+ *   - "device" pointers are CUDA device addresses owned by the caller for the duration of
+ *     the asynchronous work; "host" pointers are ordinary process memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is enqueued
+ *     asynchronously on it; a non-OK status means nothing was launched.
+ *   - Activations are row-major [rows][cols] with the channel (reduction) axis contiguous;
+ *     convolution activations are NHWC.  Weights are [N][RS][C] (output channel, filter tap,
+ *     input channel), i.e. the transpose of the paper's W in R^{Ci x Co}.
+ *   - Row pitches ("ld*") are in ELEMENTS for floating-point tensors and in BYTES for code
+ *     tensors.  Base pointers and pitches of code / output tensors must be 16-byte aligned.
+ *   - dev_status (optional, may be NULL) is a device int32 the kernels set to a non-zero
+ *     word if a bounded on-chip wait expired; copy it to the host and pass it to
+ *     hq_check_status.  It is never cleared by the library.
+ */
+#ifndef HQ_H_
+#define HQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HQ_OK = 0,
+    HQ_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, unknown enum value */
+    HQ_ERR_SHAPE = 2,         /* sizes that contradict each other (cols % had_block, K mismatch ...) */
+    HQ_ERR_UNSUPPORTED = 3,   /* legal request this build has no kernel for */
+    HQ_ERR_ALIGNMENT = 4,     /* pointer or pitch not aligned as stated above */
+    HQ_ERR_WORKSPACE = 5,     /* workspace too small (ask hq_workspace_size) */
+    HQ_ERR_OVERFLOW_RISK = 6, /* int32 accumulators could overflow for these bit-widths and K */
+    HQ_ERR_CUDA = 7,          /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
+    HQ_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (reported via dev_status) */
+} hq_status;
+
+typedef enum { HQ_F32 = 0, HQ_BF16 = 1 } hq_dtype;
+
+/* Storage of activation codes.  NIBBLE: two codes per byte, element 2j in the low nibble, 2j+1 in
+ * the high nibble, two's complement (3-bit codes are sign-extended to a nibble).  INT8: one code per byte. */
+typedef enum { HQ_CODES_NIBBLE = 0, HQ_CODES_INT8 = 1 } hq_container;
+
+/* PER_ROW: one dynamic scale per row (token / pixel), S = max|xH| / qmax.  STATIC: one scalar for
+ * the whole tensor, read from device memory (the learned per-timestep scale of the paper). */
+typedef enum { HQ_SCALE_PER_ROW = 0, HQ_SCALE_STATIC = 1 } hq_scale_mode;
+
+/* How the offline weight integers are formed.
+ *  PLAIN : B = Q(W)                       (Eq. 3 per output channel)
+ *  FOLDED: B = H_raw * Q(W)               (the inner product of Eq. 12 / Eq. 14, exact integers; the
+ *                                          paper's Single-Hadamard semantics; needs w_bits + log2(had_block) bits)
+ *  DOUBLE: B = Q(H^T W), H orthonormal    (the Double-Hadamard scheme the paper compares against) */
+typedef enum { HQ_W_PLAIN = 0, HQ_W_FOLDED = 1, HQ_W_DOUBLE = 2 } hq_weight_mode;
+
+/* Host-side description of a prepared weight blob (filled by hq_weight_prepare). */
+typedef struct {
+    int64_t N;          /* output channels */
+    int64_t C;          /* input channels per tap */
+    int32_t RS;         /* filter taps (1 for a linear layer, 9 for 3x3) */
+    int32_t w_bits;     /* 4 or 8 */
+    int32_t had_block;  /* 2^k, or <= 1 for no transform */
+    int32_t mode;       /* hq_weight_mode */
+    int32_t limbs;      /* 1: B fits a signed byte; 2: B = 256*hi + lo, lo in [-128,127] */
+    int32_t container;  /* hq_container of the activation codes this blob pairs with (fixes the byte order along K) */
+    int64_t C_pad;      /* C rounded up to the kernel's K tile (128); padding is zero */
+    int64_t N_pad;      /* N rounded up to 128; padding rows are zero */
+    int64_t bytes;      /* size of the blob */
+    int32_t max_abs_b;  /* largest |B| entry, for the accumulator-range check */
+    int32_t reserved;
+} hq_weight_desc;
+
+int hq_version(void);
+const char* hq_status_string(hq_status s);
+
+/* Decode a dev_status word the caller copied back to the host: HQ_OK if zero, else HQ_ERR_TIMEOUT. */
+hq_status hq_check_status(const int32_t* dev_status_host_copy);
+
+/* ---- Eq. 10 + Eq. 3: codes = Q(x * BlockDiag(H_k)) ------------------------------------------------
+ * x          device, [rows][cols] of xdt, pitch ldx elements (16-byte aligned rows).
+ * had_block  2^k dividing cols (Eq. 10: cols = m * 2^k), or 0/1 for H = I (the bypass after Eq. 10).
+ * bits       3, 4 or 8.  NIBBLE container needs bits <= 4 and cols even.
+ * mode       PER_ROW: scales[rows] is written, S = max_j |(xH)_j| / qmax(bits), H orthonormal (the
+ *            2^(-k/2) of Eq. 7 is inside S); an all-zero row gets S = 1.
+ *            STATIC : static_scale (device, 1 float) is read; scales[0] (if scales != NULL) receives a copy.
+ * codes      device, [rows] x ld_codes bytes; code = clamp(rint(xH / S), -2^(bits-1), 2^(bits-1)-1), ties to even.
+ * Errors: NULL pointers, cols % had_block, had_block not a power of two -> no launch. */
+hq_status hq_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx,
+                            int had_block, int bits, hq_scale_mode mode, const float* static_scale,
+                            void* codes, hq_container cont, int64_t ld_codes, float* scales, void* stream);
+
+/* ---- Offline weight side (host code, not timed): Eq. 3 per output channel, then the chosen mode. ----
+ * w          host fp32 [N][RS][C].
+ * container  the activation container the blob will be multiplied with.
+ * blob       host buffer of hq_weight_blob_bytes(...) bytes; copy it to the device as is.
+ * s_w        host [N] per-output-channel scales (for DOUBLE: scales of H^T W).
+ * desc       filled on success.
+ * Errors: FOLDED/DOUBLE with C % had_block != 0; FOLDED whose integers need more than 2 limbs -> HQ_ERR_OVERFLOW_RISK. */
+int64_t hq_weight_blob_bytes(int64_t N, int32_t RS, int64_t C, int32_t w_bits, int32_t had_block,
+                             hq_weight_mode mode);
+hq_status hq_weight_prepare(const float* w, int64_t N, int32_t RS, int64_t C, int32_t w_bits, int32_t had_block,
+                            hq_weight_mode mode, hq_container container, void* blob, int64_t blob_bytes,
+                            float* s_w, hq_weight_desc* desc);
+
+/* ---- Eq. 12: integer product + rescale ------------------------------------------------------------
+ * acc[m][o] = sum_k a[m][k] * B[o][k]  (int32, exact);  y = alpha * S_a[m] * S_w[o] * acc + bias[o].
+ * a_codes    device, [M] x lda bytes, container and a_bits as produced by hq_hadamard_quant.
+ * desc/w_dev host descriptor and device copy of the blob; desc->RS must be 1 and desc->C == K.
+ * scale_a    device [M], or [1] if scale_a_is_scalar.  scale_w device [N].  bias device [N] or NULL.
+ * alpha      2^(-k/2) for FOLDED weights with had_block = 2^k, else 1 (hq_alpha_for computes it).
+ * acc_out    device int32 [M][N] (pitch N) or NULL.   y: device [M] x ldy elements of ydt, or NULL.
+ * Errors: K mismatch, container mismatch with the blob, accumulator bound K * qmax_a * max|B| >= 2^31
+ * -> HQ_ERR_OVERFLOW_RISK. */
+hq_status hq_qgemm(const void* a_codes, hq_container cont, int a_bits, int64_t M, int64_t K, int64_t lda,
+                   const hq_weight_desc* desc, const void* w_dev, const float* scale_a, int scale_a_is_scalar,
+                   const float* scale_w, const float* bias, float alpha, int32_t* acc_out, void* y,
+                   hq_dtype ydt, int64_t ldy, int32_t* dev_status, void* stream);
+
+/* ---- Eq. 14 (transform on the channel axis): integer convolution + rescale --------------------------
+ * a_codes NHWC [Nb][H][W] x (C codes, densely packed); weights [Cout][R][S][C] inside the blob; R = S in {1,3},
+ * stride in {1,2}, pad in {0,1}; zero padding.  Output NHWC [Nb][Ho][Wo][Cout], Ho = (H + 2 pad - R)/stride + 1.
+ * scale_a_is_scalar != 0: y = alpha * S_a * S_w[o] * acc + bias[o].
+ * scale_a_is_scalar == 0: scale_a is [Nb*H*W], one per INPUT pixel, and each tap is rescaled by the scale of
+ *   the pixel it read: y = alpha * S_w[o] * sum_taps S_a[pix(tap)] * acc_tap + bias[o]. */
+hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
+                     int64_t C, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                     const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias,
+                     float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, void* stream);
+
+/* ---- Fused layer: transform -> quantize -> integer product -> rescale in one call (Eq. 12 / Eq. 14). ----
+ * Codes and scales live in `workspace` (device, hq_workspace_size bytes); the code container is desc->container.
+ * alpha is derived from the descriptor.  y pitch ldy elements. */
+hq_status hq_workspace_size(int64_t rows, int64_t cols, hq_container cont, size_t* bytes);
+hq_status hq_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx, const hq_weight_desc* desc,
+                     const void* w_dev, const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                     const float* static_scale, void* y, hq_dtype ydt, int64_t ldy, void* workspace,
+                     size_t ws_bytes, int32_t* dev_status, void* stream);
+hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                   const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                   const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                   const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                   int32_t* dev_status, void* stream);
+
+/* alpha of the rescale for a descriptor: 2^(-k/2) for FOLDED weights (the second normalisation of Eq. 12), else 1. */
+float hq_alpha_for(const hq_weight_desc* desc);
+
+/* ---- Measurement helper: issue-rate probe of the int8 tensor pipe (no global traffic). ---------------
+ * Runs `iters` back-to-back 128x256x32 int8 MMAs per SM on resident shared-memory tiles on `ctas` CTAs.
+ * The caller times it with events; ops = ctas * iters * 2*128*256*32.  dev_status as above. */
+hq_status hq_mma_i8_probe(int ctas, int iters, int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HQ_H_ */

@@ -1,0 +1,236 @@
+"""ctypes binding of the C-ABI library ``libhq.so`` (declared in ``include/hq.h``).
+
+Argument marshalling only: every function here forwards to the entry point of the same name.
+Device buffers are torch CUDA tensors (torch is used for memory and streams, nothing else);
+their ``data_ptr()`` is what crosses the boundary.  Importing this module loads the CUDA
+library and raises if it has not been built -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_DIR, "libhq.so")
+
+HQ_OK = 0
+HQ_F32, HQ_BF16 = 0, 1
+HQ_CODES_NIBBLE, HQ_CODES_INT8 = 0, 1
+HQ_SCALE_PER_ROW, HQ_SCALE_STATIC = 0, 1
+HQ_W_PLAIN, HQ_W_FOLDED, HQ_W_DOUBLE = 0, 1, 2
+WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBLE}
+
+EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
+           "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
+           "hq_alpha_for", "hq_mma_i8_probe"]
+
+
+class HqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (hq_status {status})")
+
+
+class WeightDesc(C.Structure):
+    _fields_ = [("N", C.c_int64), ("C", C.c_int64), ("RS", C.c_int32), ("w_bits", C.c_int32),
+                ("had_block", C.c_int32), ("mode", C.c_int32), ("limbs", C.c_int32), ("container", C.c_int32),
+                ("C_pad", C.c_int64), ("N_pad", C.c_int64), ("bytes", C.c_int64), ("max_abs_b", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_05746_b200.build` "
+                          "(there is no CPU fallback for the CUDA path)")
+    L = C.CDLL(LIB_PATH)
+    p, i64, i32 = C.c_void_p, C.c_int64, C.c_int
+    L.hq_version.restype = C.c_int
+    L.hq_status_string.restype = C.c_char_p
+    L.hq_status_string.argtypes = [C.c_int]
+    L.hq_check_status.argtypes = [p]
+    L.hq_hadamard_quant.argtypes = [p, i32, i64, i64, i64, i32, i32, i32, p, p, i32, i64, p, p]
+    L.hq_weight_blob_bytes.restype = i64
+    L.hq_weight_blob_bytes.argtypes = [i64, C.c_int32, i64, C.c_int32, C.c_int32, i32]
+    L.hq_weight_prepare.argtypes = [p, i64, C.c_int32, i64, C.c_int32, C.c_int32, i32, i32, p, i64, p,
+                                    C.POINTER(WeightDesc)]
+    L.hq_qgemm.argtypes = [p, i32, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, i32, p, p, C.c_float, p, p, i32,
+                           i64, p, p]
+    L.hq_qconv2d.argtypes = [p, i32, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, i32,
+                             p, p, C.c_float, p, p, i32, p, p]
+    L.hq_workspace_size.argtypes = [i64, i64, i32, C.POINTER(C.c_size_t)]
+    L.hq_qlinear.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i32, i64, p,
+                             C.c_size_t, p, p]
+    L.hq_qconv.argtypes = [p, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32, i32,
+                           p, p, i32, p, C.c_size_t, p, p]
+    L.hq_alpha_for.restype = C.c_float
+    L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
+    L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
+    for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
+                 "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe"):
+        getattr(L, name).restype = C.c_int
+    return L
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.hq_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != HQ_OK:
+        raise HqError(status, what)
+
+
+def _dptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t):
+    import torch
+    if t.dtype == torch.float32:
+        return HQ_F32
+    if t.dtype == torch.bfloat16:
+        return HQ_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def hq_version() -> int:
+    return lib.hq_version()
+
+
+def hq_check_status(dev_status) -> None:
+    """dev_status: a torch int32 tensor of one element (device); raises HqError on a recorded timeout."""
+    host = np.array([int(dev_status.cpu()[0])], dtype=np.int32)
+    _check(lib.hq_check_status(host.ctypes.data_as(C.c_void_p)), "hq_check_status")
+
+
+def hq_hadamard_quant(x, had_block: int, bits: int, codes, container: int, scales=None, static_scale=None,
+                      stream=None) -> None:
+    """x [rows, cols] (fp32/bf16, last dim contiguous) -> codes (uint8 [rows, pitch]) and scales (fp32)."""
+    rows, cols = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_hadamard_quant(_dptr(x), _dtype_code(x), rows, cols, x.stride(0), had_block, bits, mode,
+                                 _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
+                                 _stream(stream)), "hq_hadamard_quant")
+
+
+class PreparedWeight:
+    """Result of hq_weight_prepare: host blob + scales + descriptor, and (after .to_device()) device copies."""
+
+    def __init__(self, desc: WeightDesc, blob: np.ndarray, s_w: np.ndarray):
+        self.desc, self.blob, self.s_w = desc, blob, s_w
+        self.blob_dev = None
+        self.s_w_dev = None
+
+    def to_device(self, device="cuda"):
+        import torch
+        self.blob_dev = torch.from_numpy(self.blob).to(device)
+        self.s_w_dev = torch.from_numpy(self.s_w).to(device)
+        return self
+
+    @property
+    def alpha(self) -> float:
+        return float(lib.hq_alpha_for(C.byref(self.desc)))
+
+
+def hq_weight_blob_bytes(N: int, RS: int, Cin: int, w_bits: int, had_block: int, mode: int) -> int:
+    return int(lib.hq_weight_blob_bytes(N, RS, Cin, w_bits, had_block, mode))
+
+
+def hq_weight_prepare(w: np.ndarray, w_bits: int, had_block: int, mode: int, container: int) -> PreparedWeight:
+    """w: host fp32 [N, C] or [N, R, S, C]."""
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    N, Cin = w.shape[0], w.shape[-1]
+    RS = w.size // (N * Cin)
+    nbytes = hq_weight_blob_bytes(N, RS, Cin, w_bits, had_block, mode)
+    blob = np.zeros((max(nbytes, 1),), np.int8)
+    s_w = np.zeros((N,), np.float32)
+    desc = WeightDesc()
+    _check(lib.hq_weight_prepare(w.ctypes.data_as(C.c_void_p), N, RS, Cin, w_bits, had_block, mode, container,
+                                 blob.ctypes.data_as(C.c_void_p), nbytes, s_w.ctypes.data_as(C.c_void_p),
+                                 C.byref(desc)), "hq_weight_prepare")
+    return PreparedWeight(desc, blob, s_w)
+
+
+def hq_qgemm(a_codes, container: int, a_bits: int, K: int, pw: PreparedWeight, scale_a=None, bias=None,
+             alpha: float = 1.0, acc_out=None, y=None, dev_status=None, stream=None) -> None:
+    M = a_codes.shape[0]
+    scalar = 1 if (scale_a is not None and scale_a.numel() == 1) else 0
+    ydt = _dtype_code(y) if y is not None else HQ_BF16
+    ldy = y.stride(0) if y is not None else 0
+    _check(lib.hq_qgemm(_dptr(a_codes), container, a_bits, M, K, a_codes.stride(0), C.byref(pw.desc),
+                        _dptr(pw.blob_dev), _dptr(scale_a), scalar, _dptr(pw.s_w_dev), _dptr(bias), alpha,
+                        _dptr(acc_out), _dptr(y), ydt, ldy, _dptr(dev_status), _stream(stream)), "hq_qgemm")
+
+
+def hq_qconv2d(a_codes, container: int, a_bits: int, Nb: int, H: int, W: int, Cin: int, pw: PreparedWeight, R: int,
+               S: int, stride: int, pad: int, scale_a=None, bias=None, alpha: float = 1.0, acc_out=None, y=None,
+               dev_status=None, stream=None) -> None:
+    scalar = 1 if (scale_a is None or scale_a.numel() == 1) else 0
+    ydt = _dtype_code(y) if y is not None else HQ_BF16
+    _check(lib.hq_qconv2d(_dptr(a_codes), container, a_bits, Nb, H, W, Cin, C.byref(pw.desc), _dptr(pw.blob_dev), R,
+                          S, stride, pad, _dptr(scale_a), scalar, _dptr(pw.s_w_dev), _dptr(bias), alpha,
+                          _dptr(acc_out), _dptr(y), ydt, _dptr(dev_status), _stream(stream)), "hq_qconv2d")
+
+
+def hq_workspace_size(rows: int, cols: int, container: int) -> int:
+    out = C.c_size_t(0)
+    _check(lib.hq_workspace_size(rows, cols, container, C.byref(out)), "hq_workspace_size")
+    return int(out.value)
+
+
+def hq_qlinear(x, pw: PreparedWeight, bias, a_bits: int, y, workspace, static_scale=None, dev_status=None,
+               stream=None) -> None:
+    M, K = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_qlinear(_dptr(x), _dtype_code(x), M, K, x.stride(0), C.byref(pw.desc), _dptr(pw.blob_dev),
+                          _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y), _dtype_code(y),
+                          y.stride(0), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                          _dptr(dev_status), _stream(stream)), "hq_qlinear")
+
+
+def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias, a_bits: int, y, workspace,
+             static_scale=None, dev_status=None, stream=None) -> None:
+    Nb, H, W, Cin = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride,
+                        pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y),
+                        _dtype_code(y), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                        _dptr(dev_status), _stream(stream)), "hq_qconv")
+
+
+def hq_mma_i8_probe(ctas: int, iters: int, dev_status=None, stream=None) -> None:
+    _check(lib.hq_mma_i8_probe(ctas, iters, _dptr(dev_status), _stream(stream)), "hq_mma_i8_probe")
+
+
+def decode_blob(pw: PreparedWeight) -> np.ndarray:
+    """Host-side inverse of the blob layout: returns the weight integers B as int32 [N, RS, C].
+    (A test and debugging aid: pure byte shuffling, no arithmetic beyond 256*hi + lo.)"""
+    d = pw.desc
+    Kp = d.RS * d.C_pad
+    rows = pw.blob[: d.N_pad * d.limbs * Kp].reshape(-1, Kp).astype(np.int32)
+    o = np.arange(d.N)
+    if d.limbs == 1:
+        full = rows[o]
+    else:
+        hi = rows[(o // 128) * 256 + (o % 128)]
+        lo = rows[(o // 128) * 256 + 128 + (o % 128)]
+        full = 256 * hi + lo
+    full = full.reshape(d.N, d.RS, d.C_pad)[:, :, : d.C]
+    if d.container == HQ_CODES_NIBBLE:
+        c = np.arange(d.C)
+        r = c & 7
+        slot = np.where(r & 1, 4 + (r >> 1), r >> 1)
+        full = full[:, :, (c & ~7) + slot]
+    return np.ascontiguousarray(full)

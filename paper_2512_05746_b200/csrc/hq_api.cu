@@ -1,0 +1,105 @@
+// Entry points that are not a kernel of their own: status helpers and the fused layer calls, which run
+// transform+quantize (Eq. 10, Eq. 3) and then the integer product with its rescale (Eq. 12 / Eq. 14) on one stream.
+#include "hq_common.cuh"
+
+namespace hq {
+hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
+                                int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                hq_container cont, int64_t ld_codes, float* scales, cudaStream_t st);
+hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64_t M, int64_t K, int64_t lda,
+                       const hq_weight_desc* desc, const void* w_dev, const float* scale_a, int scale_a_is_scalar,
+                       const float* scale_w, const float* bias, float alpha, int32_t* acc_out, void* y,
+                       hq_dtype ydt, int64_t ldy, int32_t* dev_status, cudaStream_t st);
+hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
+                         int64_t C, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                         const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias,
+                         float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st);
+
+namespace {
+int64_t code_pitch(int64_t cols, hq_container cont) {
+    const int64_t b = cont == HQ_CODES_NIBBLE ? cols / 2 : cols;
+    return (b + 15) / 16 * 16;
+}
+int64_t scales_offset(int64_t rows, int64_t cols, hq_container cont) {
+    return (rows * code_pitch(cols, cont) + 255) / 256 * 256;
+}
+}  // namespace
+}  // namespace hq
+
+extern "C" int hq_version(void) { return 100; }
+
+extern "C" const char* hq_status_string(hq_status s) {
+    switch (s) {
+        case HQ_OK: return "ok";
+        case HQ_ERR_INVALID_ARG: return "invalid argument";
+        case HQ_ERR_SHAPE: return "inconsistent shape";
+        case HQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HQ_ERR_ALIGNMENT: return "misaligned pointer or pitch";
+        case HQ_ERR_WORKSPACE: return "workspace too small";
+        case HQ_ERR_OVERFLOW_RISK: return "int32 accumulator could overflow";
+        case HQ_ERR_CUDA: return "CUDA call failed";
+        case HQ_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+extern "C" hq_status hq_check_status(const int32_t* dev_status_host_copy) {
+    if (dev_status_host_copy == nullptr) return HQ_ERR_INVALID_ARG;
+    return *dev_status_host_copy == 0 ? HQ_OK : HQ_ERR_TIMEOUT;
+}
+
+extern "C" hq_status hq_workspace_size(int64_t rows, int64_t cols, hq_container cont, size_t* bytes) {
+    if (bytes == nullptr) return HQ_ERR_INVALID_ARG;
+    if (cont != HQ_CODES_NIBBLE && cont != HQ_CODES_INT8) return HQ_ERR_INVALID_ARG;
+    if (rows < 0 || cols <= 0) return HQ_ERR_SHAPE;
+    *bytes = size_t(hq::scales_offset(rows, cols, cont)) + size_t(rows > 0 ? rows : 1) * sizeof(float);
+    return HQ_OK;
+}
+
+extern "C" hq_status hq_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx,
+                                const hq_weight_desc* desc, const void* w_dev, const float* scale_w,
+                                const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale, void* y,
+                                hq_dtype ydt, int64_t ldy, void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                void* stream) {
+    using namespace hq;
+    if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+    const hq_container cont = hq_container(desc->container);
+    size_t need = 0;
+    hq_status s = hq_workspace_size(M, K, cont, &need);
+    if (s != HQ_OK) return s;
+    if (ws_bytes < need) return HQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* codes = static_cast<unsigned char*>(workspace);
+    float* scales = reinterpret_cast<float*>(codes + scales_offset(M, K, cont));
+    const int64_t ldc = code_pitch(K, cont);
+    s = launch_hadamard_quant(x, xdt, M, K, ldx, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
+    if (s != HQ_OK) return s;
+    return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, mode == HQ_SCALE_STATIC, scale_w, bias,
+                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st);
+}
+
+extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                              const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                              const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                              const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                              int32_t* dev_status, void* stream) {
+    using namespace hq;
+    if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+    const hq_container cont = hq_container(desc->container);
+    const int64_t rows = Nb * H * W;
+    size_t need = 0;
+    hq_status s = hq_workspace_size(rows, C, cont, &need);
+    if (s != HQ_OK) return s;
+    if (ws_bytes < need) return HQ_ERR_WORKSPACE;
+    const int64_t ldc = code_pitch(C, cont);
+    if (ldc != (cont == HQ_CODES_NIBBLE ? C / 2 : C)) return HQ_ERR_ALIGNMENT;   // conv needs densely packed pixels
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* codes = static_cast<unsigned char*>(workspace);
+    float* scales = reinterpret_cast<float*>(codes + scales_offset(rows, C, cont));
+    s = launch_hadamard_quant(x, xdt, rows, C, C, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
+    if (s != HQ_OK) return s;
+    return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
+                          mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st);
+}

@@ -1,0 +1,363 @@
+// Fused online Hadamard transform + symmetric quantization (Eq. 10 with Eq. 5-7, then Eq. 3).
+//
+// HBM-bound: every input element is read once (128-bit loads) and 0.5 or 1 byte is written.
+// Fast path (block size n = 2^k, k = 8..12): a block of n channels is owned by n/32 threads, each
+// holding 32 values in registers.
+//   phase A  thread t holds elements {4t + c + (n/8) i : c < 4, i < 8}: fully coalesced 16-byte loads;
+//            a 32-point in-register transform covers index bits {0, 1, k-3, k-2, k-1};
+//   exchange one trip through shared memory (XOR-swizzled, conflict-free both ways);
+//   phase B  thread t holds the 32 contiguous elements 32t .. 32t+31: in-register stages for bits {2,3,4},
+//            warp-shuffle stages for bits 5 .. k-4 (none for k = 8);
+//   then     |max| over the row (shuffles, plus a shared-memory max when a row spans several blocks or
+//            warps), scale, round-half-even by a magic-number add, clamp, pack, one 16-byte store per thread.
+// The butterflies run unnormalised (H_raw); 2^(-k/2) is folded into the scale (Eq. 7).
+// A generic shared-memory kernel covers every other block size, including the identity (no transform).
+#include "hq_common.cuh"
+
+namespace hq {
+namespace {
+
+constexpr float kMagic = 12582912.0f;            // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+constexpr uint32_t kMagicBits = 0x4B400000u;
+
+struct QuantParams {
+    const void* x;
+    int64_t rows, cols, ldx;
+    int m;               // Hadamard blocks per row
+    int rows_per_cta;
+    int threads_per_row;
+    int bits;
+    float norm;          // 2^(-k/2) (1 for the identity)
+    const float* static_scale;
+    uint8_t* codes;
+    int64_t ld_codes;
+    float* scales;
+};
+
+__device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+    uint2 raw = __ldcs(reinterpret_cast<const uint2*>(p));
+    float4 f;
+    f.x = __uint_as_float(raw.x << 16);
+    f.y = __uint_as_float(raw.x & 0xFFFF0000u);
+    f.z = __uint_as_float(raw.y << 16);
+    f.w = __uint_as_float(raw.y & 0xFFFF0000u);
+    return f;
+}
+
+template <int LO, int HI>
+__device__ __forceinline__ void butterflies(float (&v)[32]) {
+#pragma unroll
+    for (int h = LO; h <= HI; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if (!(i & h)) {
+                const float a = v[i], b = v[i | h];
+                v[i] = a + b;
+                v[i | h] = a - b;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ int swz(int slot) { return slot ^ ((slot >> 3) & 7); }
+
+// Round (ties to even), clamp and pack 32 values held by one thread; returns words through `out`.
+template <bool INT8_OUT>
+__device__ __forceinline__ void quantize_pack(const float (&v)[32], float inv, int bits, uint32_t* out) {
+    const float bias = INT8_OUT ? 128.0f : 8.0f;
+    const float mb = kMagic + bias;
+    const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
+    constexpr int PER_WORD = INT8_OUT ? 4 : 8;
+    constexpr int SHIFT = INT8_OUT ? 8 : 4;
+    // Each rounded value is kMagicBits + (code + bias); summing the shifted words and removing the shifted
+    // constants leaves the biased fields, which one XOR turns into two's complement.
+    uint32_t cst = 0;
+#pragma unroll
+    for (int e = 0; e < PER_WORD; ++e) cst += kMagicBits << (SHIFT * e);
+    constexpr uint32_t UNBIAS = INT8_OUT ? 0x80808080u : 0x88888888u;
+#pragma unroll
+    for (int w = 0; w < 32 / PER_WORD; ++w) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int e = 0; e < PER_WORD; ++e) {
+            float f = fmaf(v[w * PER_WORD + e], inv, mb);
+            f = fminf(fmaxf(f, lo), hi);
+            acc += __float_as_uint(f) << (SHIFT * e);
+        }
+        out[w] = (acc - cst) ^ UNBIAS;
+    }
+}
+
+template <int KLOG, typename InT, bool INT8_OUT>
+__global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
+    constexpr int N = 1 << KLOG;
+    constexpr int TB = N / 32;                         // threads per Hadamard block
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float4* xch = reinterpret_cast<float4*>(smem_raw);                              // blockDim.x * 8 float4
+    unsigned int* rowmax = reinterpret_cast<unsigned int*>(smem_raw + size_t(blockDim.x) * 128);
+
+    const int tid = threadIdx.x;
+    const int row_in_cta = tid / p.threads_per_row;
+    const int tr = tid - row_in_cta * p.threads_per_row;
+    const int blk = tr / TB;
+    const int tb = tr & (TB - 1);
+    const int64_t row = int64_t(blockIdx.x) * p.rows_per_cta + row_in_cta;
+    const bool valid = row < p.rows;
+    const bool shared_max = (p.m > 1) || (TB > 32);
+
+    if (tid < p.rows_per_cta) rowmax[tid] = 0u;
+
+    float v[32];
+    {
+        const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float4 f = load4(src + 4 * (tb + TB * i));
+            if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
+            v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+        }
+    }
+    butterflies<1, 16>(v);                             // index bits {0,1} and {k-3,k-2,k-1}
+
+    float4* grp = xch + (tid / TB) * (N / 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        grp[swz(tb + TB * i)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 f = grp[swz(i + 8 * tb)];
+        v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+    }
+    butterflies<4, 16>(v);                             // index bits {2,3,4}
+#pragma unroll
+    for (int s = 0; s < KLOG - 8; ++s) {               // index bits 5 .. k-4 live in lane bits 0 .. k-9
+        const float sgn = ((tb >> s) & 1) ? -1.0f : 1.0f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[e], 1 << s);
+            v[e] = fmaf(sgn, v[e], other);
+        }
+    }
+
+    float inv, scale;
+    if (p.static_scale == nullptr) {
+        float amax = 0.f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) amax = fmaxf(amax, fabsf(v[e]));
+#pragma unroll
+        for (int off = 1; off < (TB < 32 ? TB : 32); off <<= 1)
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+        if (shared_max) {
+            if ((tb & 31) == 0) atomicMax(&rowmax[row_in_cta], __float_as_uint(amax));
+            __syncthreads();
+            amax = __uint_as_float(rowmax[row_in_cta]);
+        }
+        const float qmaxf = float((1 << (p.bits - 1)) - 1);
+        if (amax > 0.f) {
+            scale = amax * (p.norm / qmaxf);
+            inv = qmaxf / amax;
+            if (!(scale > 0.f)) { scale = 1.0f; inv = p.norm; }   // scale underflowed: same rule as an all-zero row
+        } else {
+            scale = 1.0f;
+            inv = 0.f;
+        }
+    } else {
+        scale = __ldg(p.static_scale);
+        inv = p.norm / scale;
+    }
+
+    if (valid) {
+        uint8_t* dst = p.codes + row * p.ld_codes;
+        if (INT8_OUT) {
+            uint32_t w[8];
+            quantize_pack<true>(v, inv, p.bits, w);
+            uint4* d = reinterpret_cast<uint4*>(dst + int64_t(blk) * N + 32 * tb);
+            d[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            d[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else {
+            uint32_t w[4];
+            quantize_pack<false>(v, inv, p.bits, w);
+            *reinterpret_cast<uint4*>(dst + (int64_t(blk) * N + 32 * tb) / 2) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (p.scales != nullptr) {
+            if (p.static_scale == nullptr) { if (tr == 0) p.scales[row] = scale; }
+            else if (row == 0 && tr == 0) p.scales[0] = scale;
+        }
+    }
+}
+
+// Generic path: one CTA per row (grid-stride), the row lives in shared memory, one __syncthreads per stage.
+template <typename InT>
+__global__ void __launch_bounds__(256) fwht_quant_generic(const QuantParams p, int had_block, int int8_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* buf = reinterpret_cast<float*>(smem_raw);
+    __shared__ float red[8];
+    __shared__ float s_amax;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int cols = int(p.cols);
+    for (int64_t row = blockIdx.x; row < p.rows; row += gridDim.x) {
+        const InT* src = reinterpret_cast<const InT*>(p.x) + row * p.ldx;
+        for (int j = tid; j < cols; j += nthr) {
+            float f;
+            if (sizeof(InT) == 4) f = reinterpret_cast<const float*>(src)[j];
+            else f = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[j]);
+            buf[j] = f;
+        }
+        __syncthreads();
+        for (int h = 1; h < had_block; h <<= 1) {
+            for (int pr = tid; pr < cols / 2; pr += nthr) {
+                const int i = (pr / h) * 2 * h + (pr % h);
+                const float a = buf[i], b = buf[i + h];
+                buf[i] = a + b;
+                buf[i + h] = a - b;
+            }
+            __syncthreads();
+        }
+        float inv, scale;
+        if (p.static_scale == nullptr) {
+            float amax = 0.f;
+            for (int j = tid; j < cols; j += nthr) amax = fmaxf(amax, fabsf(buf[j]));
+            for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+            if ((tid & 31) == 0) red[tid >> 5] = amax;
+            __syncthreads();
+            if (tid == 0) {
+                float a = 0.f;
+                for (int w = 0; w < (nthr + 31) / 32; ++w) a = fmaxf(a, red[w]);
+                s_amax = a;
+            }
+            __syncthreads();
+            amax = s_amax;
+            const float qmaxf = float((1 << (p.bits - 1)) - 1);
+            if (amax > 0.f) {
+                scale = amax * (p.norm / qmaxf);
+                inv = qmaxf / amax;
+                if (!(scale > 0.f)) { scale = 1.0f; inv = p.norm; }
+            } else { scale = 1.0f; inv = 0.f; }
+        } else {
+            scale = __ldg(p.static_scale);
+            inv = p.norm / scale;
+        }
+        const float lo = kMagic + float(-(1 << (p.bits - 1))), hi = kMagic + float((1 << (p.bits - 1)) - 1);
+        uint8_t* dst = p.codes + row * p.ld_codes;
+        if (int8_out) {
+            for (int j = tid; j < cols; j += nthr) {
+                const float f = fminf(fmaxf(fmaf(buf[j], inv, kMagic), lo), hi);
+                dst[j] = uint8_t(__float_as_uint(f) & 0xFFu);
+            }
+        } else {
+            for (int j = tid; j < cols / 2; j += nthr) {
+                const float f0 = fminf(fmaxf(fmaf(buf[2 * j], inv, kMagic), lo), hi);
+                const float f1 = fminf(fmaxf(fmaf(buf[2 * j + 1], inv, kMagic), lo), hi);
+                dst[j] = uint8_t((__float_as_uint(f0) & 0xFu) | ((__float_as_uint(f1) & 0xFu) << 4));
+            }
+        }
+        if (tid == 0 && p.scales != nullptr) {
+            if (p.static_scale == nullptr) p.scales[row] = scale;
+            else if (row == 0) p.scales[0] = scale;
+        }
+        __syncthreads();
+    }
+}
+
+template <int KLOG, typename InT>
+cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threads, size_t smem, cudaStream_t st) {
+    if (int8_out) fwht_quant_fast<KLOG, InT, true><<<grid, threads, smem, st>>>(p);
+    else fwht_quant_fast<KLOG, InT, false><<<grid, threads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <typename InT>
+cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int grid, int threads, size_t smem,
+                          cudaStream_t st) {
+    switch (klog) {
+        case 8: return launch_fast<8, InT>(p, int8_out, grid, threads, smem, st);
+        case 9: return launch_fast<9, InT>(p, int8_out, grid, threads, smem, st);
+        case 10: return launch_fast<10, InT>(p, int8_out, grid, threads, smem, st);
+        case 11: return launch_fast<11, InT>(p, int8_out, grid, threads, smem, st);
+        case 12: return launch_fast<12, InT>(p, int8_out, grid, threads, smem, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+// Launches the transform+quantize kernel; shared by the public entry point and the fused layer calls.
+hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
+                                int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                hq_container cont, int64_t ld_codes, float* scales, cudaStream_t st) {
+    if (rows == 0 && cols > 0) return HQ_OK;                       // nothing to do; pointers may be NULL
+    if (x == nullptr || codes == nullptr) return HQ_ERR_INVALID_ARG;
+    if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
+    if (cont != HQ_CODES_NIBBLE && cont != HQ_CODES_INT8) return HQ_ERR_INVALID_ARG;
+    if (mode != HQ_SCALE_PER_ROW && mode != HQ_SCALE_STATIC) return HQ_ERR_INVALID_ARG;
+    if (mode == HQ_SCALE_STATIC && static_scale == nullptr) return HQ_ERR_INVALID_ARG;
+    if (mode == HQ_SCALE_PER_ROW && scales == nullptr) return HQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return HQ_ERR_INVALID_ARG;
+    if (rows < 0 || cols <= 0 || ldx < cols) return HQ_ERR_SHAPE;
+    if (cont == HQ_CODES_NIBBLE && (bits > 4 || (cols & 1))) return HQ_ERR_SHAPE;
+    const int64_t row_bytes = cont == HQ_CODES_NIBBLE ? cols / 2 : cols;
+    if (ld_codes < row_bytes) return HQ_ERR_SHAPE;
+    if (had_block > 1 && (!is_pow2(had_block) || cols % had_block != 0)) return HQ_ERR_SHAPE;
+    const int n = had_block > 1 ? had_block : 1;
+    const int klog = ilog2(n);
+
+    QuantParams p{};
+    p.x = x; p.rows = rows; p.cols = cols; p.ldx = ldx;
+    p.m = int(cols / n);
+    p.bits = bits;
+    p.norm = float(exp2(-0.5 * double(klog)));
+    p.static_scale = mode == HQ_SCALE_STATIC ? static_scale : nullptr;
+    p.codes = static_cast<uint8_t*>(codes);
+    p.ld_codes = ld_codes;
+    p.scales = scales;
+
+    const int elt = xdt == HQ_F32 ? 4 : 2;
+    const bool fast_ok = klog >= 8 && klog <= 12 && cols / 32 <= 256 &&
+                         (reinterpret_cast<uintptr_t>(x) % (4 * elt) == 0) && (ldx % 4 == 0) &&
+                         aligned16(codes) && (ld_codes % 16 == 0);
+    if (fast_ok) {
+        const int tr = int(cols / 32);
+        int rpc = 1;
+        while ((rpc * tr) % 32 != 0) ++rpc;                 // whole warps
+        const int base = rpc;
+        while ((rpc + base) * tr <= 256) rpc += base;
+        p.threads_per_row = tr;
+        p.rows_per_cta = rpc;
+        const int threads = rpc * tr;
+        const size_t smem = size_t(threads) * 128 + size_t(rpc) * 4;
+        const int grid = int((rows + rpc - 1) / rpc);
+        cudaError_t e = xdt == HQ_F32
+                            ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
+                            : dispatch_fast<__nv_bfloat16>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st);
+        return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+    }
+    const size_t smem = size_t(cols) * 4;
+    if (smem > 200 * 1024) return HQ_ERR_UNSUPPORTED;
+    const int grid = int(rows < 148 * 8 ? rows : 148 * 8);
+    cudaError_t e;
+    if (xdt == HQ_F32) {
+        if (smem > 48 * 1024)
+            HQ_CUDA_OK(cudaFuncSetAttribute(fwht_quant_generic<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            int(smem)));
+        fwht_quant_generic<float><<<grid, 256, smem, st>>>(p, n, cont == HQ_CODES_INT8);
+    } else {
+        if (smem > 48 * 1024)
+            HQ_CUDA_OK(cudaFuncSetAttribute(fwht_quant_generic<__nv_bfloat16>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        fwht_quant_generic<__nv_bfloat16><<<grid, 256, smem, st>>>(p, n, cont == HQ_CODES_INT8);
+    }
+    e = cudaGetLastError();
+    return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+}  // namespace hq
+
+extern "C" hq_status hq_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx,
+                                       int had_block, int bits, hq_scale_mode mode, const float* static_scale,
+                                       void* codes, hq_container cont, int64_t ld_codes, float* scales,
+                                       void* stream) {
+    return hq::launch_hadamard_quant(x, xdt, rows, cols, ldx, had_block, bits, mode, static_scale, codes, cont,
+                                     ld_codes, scales, static_cast<cudaStream_t>(stream));
+}

@@ -1,0 +1,170 @@
+"""GPU parity: integer GEMM / convolution with the rescale epilogue (hq_qgemm, hq_qconv2d) against the CPU oracle.
+Integer accumulators must be bit-exact; float outputs within the stated tolerances."""
+import numpy as np
+import pytest
+
+from paper_2512_05746_b200 import inputs
+from hq_testutil import Y_BF16_RTOL, Y_F32_RTOL, pack_nibbles_np, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2512_05746_b200 import binding as hq
+    return torch, hq
+
+
+def to_container(torch, hq, q_np, container):
+    """int8 codes [..., K] -> device uint8 tensor in the requested container (rows densely packed)."""
+    if container == hq.HQ_CODES_NIBBLE:
+        b = pack_nibbles_np(q_np)
+    else:
+        b = q_np.view(np.uint8)
+    return torch.from_numpy(np.ascontiguousarray(b)).cuda()
+
+
+def gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, container, seed=0, with_bias=True):
+    q = inputs.codes((M, K), a_bits, seed=seed)
+    w = inputs.weights((N, K), seed=seed)
+    pw = hq.hq_weight_prepare(w, w_bits, had_block, hq.WEIGHT_MODES[mode], container).to_device()
+    B_ref = hq.decode_blob(pw).reshape(N, K)
+    s_a = inputs.positive_scales(M, seed=seed)
+    b = inputs.bias(N, seed=seed) if with_bias else None
+    a_dev = to_container(torch, hq, q, container)
+    acc = torch.full((M, N), 12345, dtype=torch.int32, device="cuda")
+    y16 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    y32 = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    sa_dev = torch.from_numpy(s_a).cuda()
+    b_dev = None if b is None else torch.from_numpy(b).cuda()
+    hq.hq_qgemm(a_dev, container, a_bits, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, acc_out=acc, y=y16,
+                dev_status=status)
+    hq.hq_qgemm(a_dev, container, a_bits, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y32, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    acc_ref = oracle.gemm_int(q, B_ref)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref), "int32 accumulators differ"
+    y_ref = oracle.dequant(acc_ref, s_a, pw.s_w, b, pw.alpha)
+    assert rel_err(y32.cpu().numpy(), y_ref) <= Y_F32_RTOL
+    assert rel_err(y16.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+    return pw
+
+
+GEMM_CASES = [
+    # M, K, N, a_bits, w_bits, had_block, mode, container
+    (256, 256, 256, 4, 4, 256, "plain", 1),
+    (256, 256, 256, 4, 4, 256, "folded", 1),
+    (256, 256, 256, 4, 4, 256, "folded", 0),
+    (256, 256, 256, 4, 4, 256, "plain", 0),
+    (1000, 512, 384, 4, 4, 512, "folded", 1),     # ragged M, N = 1.5 tiles
+    (1000, 512, 384, 3, 4, 512, "plain", 0),
+    (130, 2048, 512, 4, 4, 2048, "folded", 0),
+    (513, 768, 200, 4, 4, 256, "plain", 1),       # N not a multiple of 8, K = 6 blocks
+    (300, 320, 72, 8, 8, 64, "plain", 1),         # W8A8, K tail (320 = 2.5 blocks)
+    (97, 1024, 640, 4, 4, 16, "folded", 0),       # folded weights that still fit one limb
+    (4096, 1024, 1280, 4, 4, 1024, "folded", 0),  # several tiles per CTA
+    (64, 4096, 256, 4, 4, 4096, "folded", 1),
+    (1, 256, 256, 4, 4, 256, "double", 0),
+]
+
+
+@pytest.mark.parametrize("M,K,N,a_bits,w_bits,had_block,mode,container", GEMM_CASES)
+def test_qgemm_matches_oracle(env, oracle, M, K, N, a_bits, w_bits, had_block, mode, container):
+    torch, hq = env
+    gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, container, seed=M + K + N)
+
+
+def test_qgemm_extreme_magnitudes(env, oracle):
+    """Largest accumulators the path can produce: (a) folded weights with a constant channel (B = -8*n at one index,
+    so the high limb is at its extreme) against sign-matched extreme codes; (b) W8A8 with every product at 127*128."""
+    torch, hq = env
+    M, K, N = 128, 2048, 128
+    w = inputs.weights((N, K), seed=3)
+    w[0, :] = -1.0                                                  # W_int = -7 everywhere -> B[0][0] = -7*1024
+    for container in (0, 1):
+        pw = hq.hq_weight_prepare(w, 4, 1024, hq.HQ_W_FOLDED, container).to_device()
+        B = hq.decode_blob(pw).reshape(N, K)
+        assert np.abs(B).max() >= 7 * 1024
+        q = np.where(B[1] > 0, -8, 7).astype(np.int8)[None, :].repeat(M, axis=0)    # |acc| of channel 1 = sum |q||B|
+        q[1::2] = -8
+        acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+        hq.hq_qgemm(to_container(torch, hq, q, container), container, 4, K, pw, acc_out=acc)
+        torch.cuda.synchronize()
+        ref = oracle.gemm_int(q, B)
+        assert np.abs(ref).max() > 2 ** 19
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), ref)
+    K8 = 8192
+    w8 = -np.ones((N, K8), np.float32)
+    pw = hq.hq_weight_prepare(w8, 8, 1, hq.HQ_W_PLAIN, hq.HQ_CODES_INT8).to_device()
+    q8 = np.full((M, K8), -128, np.int8)
+    acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+    hq.hq_qgemm(to_container(torch, hq, q8, 1), 1, 8, K8, pw, acc_out=acc)
+    torch.cuda.synchronize()
+    assert int(acc.min()) == int(acc.max()) == 127 * 128 * K8
+
+
+def test_qgemm_scalar_scale_and_determinism(env, oracle):
+    torch, hq = env
+    M, K, N = 700, 512, 512
+    q = inputs.codes((M, K), 4, seed=5)
+    w = inputs.weights((N, K), seed=5)
+    pw = hq.hq_weight_prepare(w, 4, 512, hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE).to_device()
+    a = to_container(torch, hq, q, hq.HQ_CODES_NIBBLE)
+    s = torch.tensor([0.037], device="cuda")
+    outs = []
+    for _ in range(3):
+        y = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        hq.hq_qgemm(a, hq.HQ_CODES_NIBBLE, 4, K, pw, scale_a=s, alpha=pw.alpha, y=y)
+        outs.append(y.cpu().numpy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    y_ref = oracle.dequant(oracle.gemm_int(q, hq.decode_blob(pw).reshape(N, K)), np.array([0.037], np.float32), pw.s_w,
+                           None, pw.alpha)
+    assert rel_err(outs[0], y_ref) <= Y_F32_RTOL
+
+
+CONV_CASES = [
+    # Nb, H, W, C, Cout, R, pad, a_bits, mode, container
+    (8, 32, 32, 256, 256, 3, 1, 4, "folded", 0),     # the small conv configuration
+    (8, 32, 32, 256, 256, 3, 1, 3, "folded", 1),
+    (2, 16, 16, 128, 384, 3, 1, 4, "plain", 1),
+    (3, 8, 8, 256, 128, 3, 1, 4, "folded", 0),       # tiles span two images
+    (2, 64, 64, 128, 128, 3, 1, 4, "plain", 0),      # two output rows per tile
+    (1, 20, 12, 128, 64, 3, 1, 4, "plain", 1),       # width that does not divide 128
+    (2, 16, 16, 256, 256, 1, 0, 4, "folded", 0),     # 1x1
+    (1, 10, 10, 160, 96, 3, 0, 4, "plain", 1),       # no padding, channel tail (160 = 1.25 blocks)
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,R,pad,a_bits,mode,container", CONV_CASES)
+def test_qconv2d_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, a_bits, mode, container):
+    torch, hq = env
+    hb = 128 if C % 128 == 0 else 32
+    q = inputs.codes((Nb, H, W, C), a_bits, seed=H + W + C)
+    w = inputs.weights((Cout, R, R, C), seed=C + Cout)
+    pw = hq.hq_weight_prepare(w, 4, hb, hq.WEIGHT_MODES[mode], container).to_device()
+    B_ref = hq.decode_blob(pw).reshape(Cout, R, R, C)
+    b = inputs.bias(Cout, seed=1)
+    Ho, Wo = H + 2 * pad - R + 1, W + 2 * pad - R + 1
+    acc = torch.full((Nb, Ho, Wo, Cout), 777, dtype=torch.int32, device="cuda")
+    y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    s_a = torch.tensor([0.05], device="cuda")
+    hq.hq_qconv2d(to_container(torch, hq, q, container), container, a_bits, Nb, H, W, C, pw, R, R, 1, pad, scale_a=s_a,
+                  bias=torch.from_numpy(b).cuda(), alpha=pw.alpha, acc_out=acc, y=y, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    acc_ref = oracle.conv2d_int(q, B_ref, 1, pad)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    y_ref = oracle.dequant(acc_ref, np.array([0.05], np.float32), pw.s_w, b, pw.alpha)
+    assert rel_err(y.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+
+
+def test_int8_tensor_pipe_probe_runs(env):
+    torch, hq = env
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_mma_i8_probe(4, 64, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
