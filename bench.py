@@ -42,6 +42,7 @@ def layer_list():
     for name, K, N, hb in inputs.TRANSFORMER_LINEARS:
         layers.append(dict(kind="linear", name=name, M=M_TOKENS, K=K, N=N, had_block=hb))
     c = CONV
+    c["Nb"] = max(1, M_TOKENS // (c["H"] * c["W"]))
     layers.append(dict(kind="conv", name="conv3x3", M=c["Nb"] * c["H"] * c["W"], K=c["R"] * c["S"] * c["C"],
                        N=c["Cout"], had_block=c["had_block"]))
     return layers
@@ -249,13 +250,19 @@ def main_reference(args):
 
 
 def main():
+    global M_TOKENS, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rows", type=int, default=M_TOKENS,
+                    help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     args = ap.parse_args()
+    if args.rows != M_TOKENS:
+        M_TOKENS = int(args.rows)
+        WORKLOAD = f"REDUCED to {M_TOKENS} rows per layer (profiling case, not a benchmark number): " + WORKLOAD
     if args.impl == "reference":
         return main_reference(args)
 
