@@ -41,7 +41,8 @@ typedef enum {
     HQ_ERR_WORKSPACE = 5,     /* workspace too small (ask hq_workspace_size) */
     HQ_ERR_OVERFLOW_RISK = 6, /* int32 accumulators could overflow for these bit-widths and K */
     HQ_ERR_CUDA = 7,          /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
-    HQ_ERR_TIMEOUT = 8        /* a bounded device-side wait expired (reported via dev_status) */
+    HQ_ERR_TIMEOUT = 8,       /* a bounded device-side wait expired (reported via dev_status) */
+    HQ_ERR_SCRATCH_LIMIT = 9  /* hq_qlinear_noalloc: the layer needs more than the library's built-in scratch */
 } hq_status;
 
 typedef enum { HQ_F32 = 0, HQ_BF16 = 1 } hq_dtype;
@@ -148,6 +149,33 @@ hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W
                    const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
                    const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
                    int32_t* dev_status, void* stream);
+
+/* ---- Fused linear layer that allocates nothing and takes no workspace (the paper has no counterpart: this is a
+ * packaging of hq_qlinear for a particular kind of caller, not another operation). ---------------------------------
+ * Who it is for: code that must not, or cannot, obtain device memory at the moment it runs a layer -- an inference
+ * loop whose memory was budgeted and handed out at start-up (a cudaMalloc there would synchronise the device and
+ * could fail late), a plug-in inside a host application that owns the allocator and gives the plug-in none, or a
+ * component written in a language binding that exposes kernels but not the CUDA memory API.  Such a caller still
+ * owns x, the weights and y, but has nowhere to put the intermediate codes and scales that hq_qlinear keeps in its
+ * `workspace` argument.  Here they live in a fixed array inside the library's device image instead:
+ * HQ_NOALLOC_SCRATCH_BYTES (8 MiB) per GPU, reserved by every GPU that loads the library until the process exits.
+ *
+ * Same arguments, results and errors as hq_qlinear without `workspace` / `ws_bytes`, plus:
+ *  - the layer must satisfy hq_workspace_size(M, K, desc->container) <= HQ_NOALLOC_SCRATCH_BYTES (for nibble codes
+ *    that is M * (K/2 + 4) bytes, e.g. 8192 rows of K = 2048 is just over the limit, 8192 rows of K = 1024 fits);
+ *    otherwise HQ_ERR_SCRATCH_LIMIT is returned and nothing is launched;
+ *  - the first call on each device looks up the device address of the array (one CUDA runtime query, no allocation)
+ *    and remembers it; make that first call with the device current and before any stream capture begins;
+ *  - every call on a device uses the same array and the array keeps whatever the previous call left in it.  Nothing in
+ *    it needs to start at zero (each call overwrites every byte it later reads), but two calls whose work overlaps
+ *    on the GPU -- different streams, or different host threads -- race on it: keep calls on one stream, or order them
+ *    with events.
+ * It never calls cudaMalloc, cudaFree or any routine that allocates device or pinned memory. */
+#define HQ_NOALLOC_SCRATCH_BYTES (8u * 1024u * 1024u)
+hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx,
+                             const hq_weight_desc* desc, const void* w_dev, const float* scale_w, const float* bias,
+                             int a_bits, hq_scale_mode mode, const float* static_scale, void* y, hq_dtype ydt,
+                             int64_t ldy, int32_t* dev_status, void* stream);
 
 /* alpha of the rescale for a descriptor: 2^(-k/2) for FOLDED weights (the second normalisation of Eq. 12), else 1. */
 float hq_alpha_for(const hq_weight_desc* desc);

@@ -24,7 +24,8 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
-           "hq_alpha_for", "hq_mma_i8_probe"]
+           "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc"]
+HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
 class HqError(RuntimeError):
@@ -64,11 +65,13 @@ def _load():
                              C.c_size_t, p, p]
     L.hq_qconv.argtypes = [p, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32, i32,
                            p, p, i32, p, C.c_size_t, p, p]
+    L.hq_qlinear_noalloc.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i32, i64,
+                                     p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
-                 "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe"):
+                 "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -198,6 +201,18 @@ def hq_qlinear(x, pw: PreparedWeight, bias, a_bits: int, y, workspace, static_sc
                           _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y), _dtype_code(y),
                           y.stride(0), _dptr(workspace), workspace.numel() * workspace.element_size(),
                           _dptr(dev_status), _stream(stream)), "hq_qlinear")
+
+
+def hq_qlinear_noalloc(x, pw: PreparedWeight, bias, a_bits: int, y, static_scale=None, dev_status=None,
+                       stream=None) -> None:
+    """hq_qlinear without a workspace: the intermediate codes and scales use the library's built-in 8 MiB device
+    array, for callers that have no way to allocate one.  Raises HqError(9) when the layer does not fit."""
+    M, K = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_qlinear_noalloc(_dptr(x), _dtype_code(x), M, K, x.stride(0), C.byref(pw.desc), _dptr(pw.blob_dev),
+                                  _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y),
+                                  _dtype_code(y), y.stride(0), _dptr(dev_status), _stream(stream)),
+           "hq_qlinear_noalloc")
 
 
 def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias, a_bits: int, y, workspace,

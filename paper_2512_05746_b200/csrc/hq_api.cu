@@ -1,6 +1,12 @@
 // Entry points that are not a kernel of their own: status helpers and the fused layer calls, which run
 // transform+quantize (Eq. 10, Eq. 3) and then the integer product with its rescale (Eq. 12 / Eq. 14) on one stream.
+#include <mutex>
+
 #include "hq_common.cuh"
+
+// Scratch of hq_qlinear_noalloc: part of the library's device image, one copy per GPU that loads the library.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char hq_noalloc_scratch[HQ_NOALLOC_SCRATCH_BYTES];
 
 namespace hq {
 hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
@@ -39,6 +45,7 @@ extern "C" const char* hq_status_string(hq_status s) {
         case HQ_ERR_OVERFLOW_RISK: return "int32 accumulator could overflow";
         case HQ_ERR_CUDA: return "CUDA call failed";
         case HQ_ERR_TIMEOUT: return "device-side wait timed out";
+        case HQ_ERR_SCRATCH_LIMIT: return "layer exceeds the built-in scratch of the no-allocation entry point";
     }
     return "unknown status";
 }
@@ -102,4 +109,51 @@ extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st);
+}
+
+namespace hq {
+namespace {
+// Device address of hq_noalloc_scratch on the current device, looked up once per device.
+hq_status noalloc_scratch_address(unsigned char** out) {
+    static std::mutex mu;
+    static unsigned char* addr[64] = {};
+    int dev = 0;
+    HQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return HQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, hq_noalloc_scratch) != cudaSuccess || p == nullptr) return HQ_ERR_CUDA;
+        addr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = addr[dev];
+    return HQ_OK;
+}
+}  // namespace
+}  // namespace hq
+
+// hq_qlinear for callers that cannot allocate: the codes and scales between the two kernels go to the library's
+// own fixed device array (shared by all calls on a device, contents left over from the previous call, fully
+// overwritten before they are read).  The first call per device resolves the array's address.
+extern "C" hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx,
+                                        const hq_weight_desc* desc, const void* w_dev, const float* scale_w,
+                                        const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale,
+                                        void* y, hq_dtype ydt, int64_t ldy, int32_t* dev_status, void* stream) {
+    using namespace hq;
+    if (desc == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    const hq_container cont = hq_container(desc->container);
+    size_t need = 0;
+    hq_status s = hq_workspace_size(M, K, cont, &need);
+    if (s != HQ_OK) return s;
+    if (need > size_t(HQ_NOALLOC_SCRATCH_BYTES)) return HQ_ERR_SCRATCH_LIMIT;
+    unsigned char* codes = nullptr;
+    s = noalloc_scratch_address(&codes);
+    if (s != HQ_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* scales = reinterpret_cast<float*>(codes + scales_offset(M, K, cont));
+    const int64_t ldc = code_pitch(K, cont);
+    s = launch_hadamard_quant(x, xdt, M, K, ldx, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
+    if (s != HQ_OK) return s;
+    return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, mode == HQ_SCALE_STATIC, scale_w, bias,
+                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st);
 }
