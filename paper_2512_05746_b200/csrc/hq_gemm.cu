@@ -6,13 +6,16 @@
 // One persistent CTA per SM walks output tiles of 128 rows x 256 operand rows (256 output channels with
 // one weight limb, 128 with two).  Roles:
 //   warp 0      TMA producer: activation tile (2-D box for a GEMM, 4-D NHWC box per filter tap for a
-//               convolution, out-of-bounds = zero padding) and weight tile into a 4-stage shared-memory ring
+//               convolution, out-of-bounds = zero padding) and weight tile
 //   warp 1      issues tcgen05.mma.kind::i8 (128x256x32) into one of two 256-column TMEM accumulators
-//   warps 2-5   epilogue: tcgen05.ld, limb recombination (256*hi + lo), rescale, bf16/fp32/int32 stores;
-//               runs on accumulator t while the MMA warp fills accumulator t+1
+//   warps 2-5   epilogue: tcgen05.ld, limb recombination (256*hi + lo), rescale, and row-contiguous 16-byte stores
+//               through a small swizzled staging buffer; runs on accumulator t while the MMA warp fills t+1
 //   warps 6-9   (NIBBLE container only) unpack 4-bit codes from a raw TMA tile into the swizzled int8 operand
 //               tile.  A code q is written as the byte q<<4 (= 16q, no sign extension needed), so the accumulator
-//               is 16x the true one and is shifted back exactly in the epilogue.
+//               is 16x the true one; the factor is removed exactly in the epilogue.
+// Weights: when the whole reduction fits (K_pad <= 512 bytes per operand row, 128 KB per tile) the weight tile
+// stays resident in shared memory and the CTA walks a contiguous range of row tiles under it (only activations
+// stream); otherwise weights stream through the same ring as the activations.
 // Every wait is bounded; on expiry a status word is written and the CTA drains and exits.
 #include <cuda.h>
 
@@ -26,20 +29,28 @@ namespace {
 constexpr int kBM = 128;             // rows per tile (TMEM lanes)
 constexpr int kBN = 256;             // operand-B rows per tile (TMEM columns)
 constexpr int kBK = 128;             // bytes of K per stage (one 128-byte swizzle row)
-constexpr int kStages = 4;
+constexpr int kMaxStages = 6;
+constexpr int kResidentKb = 4;       // largest number of K blocks a resident weight tile may have
 constexpr int kABytes = kBM * kBK;           // 16 KB
 constexpr int kBBytes = kBN * kBK;           // 32 KB
-constexpr int kRawBytes = kBM * kBK / 2;     // 8 KB packed activation tile
+constexpr int kRawBytes = kBM * kBK / 2;     // 8 KB packed activation tile (lands in the upper half of its A stage)
 constexpr int kTmemCols = 512;
+constexpr int kEpiWarps = 8;            // two per TMEM lane quarter, each taking half of the tile's columns
+constexpr int kStagingBytes = 2048;          // per epilogue warp: 32 rows x 64 bytes
+constexpr int kParamBytes = kEpiWarps * 2 * (kBN / 2) * 4;   // per epilogue warp: [scale_w | bias][its columns]
+constexpr int kSmemLimit = 232448;           // 227 KB
 
 struct GemmParams {
     int64_t M;            // GEMM rows (unused for conv)
     int N;                // output channels
     int limbs;
     int a_shift;          // 4 when activation bytes are q<<4 (nibble container), else 0
+    int combine_fast;     // 256*hi + lo of the raw (shifted) accumulators fits int32
     int kb_per_tap;       // 128-byte K blocks per filter tap
     int taps;
     int tiles_m, tiles_n;
+    int stages;           // ring depth
+    int b_resident;       // weight tile stays in shared memory; tiles are walked n-major in contiguous ranges
     uint32_t a_box_bytes; // bytes one activation TMA box delivers
     // convolution geometry (conv != 0)
     int conv, Nb, H, W, Ho, Wo, R, S, stride, pad;
@@ -48,23 +59,34 @@ struct GemmParams {
     const float* scale_a; int sa_scalar;
     const float* scale_w; const float* bias; float alpha;
     int32_t* acc_out; void* y; int y_bf16; int64_t ldy;
+    int y_vec_ok, acc_vec_ok;
     int32_t* dev_status;
 };
 
 struct SharedCtl {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
-    uint64_t unpacked[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t rawread[kMaxStages];     // all unpack threads hold their share of the packed tile in registers
+    uint64_t unpacked[kMaxStages];
+    uint64_t bfull[kResidentKb];
+    uint64_t bfree;
     uint64_t tfull[2];
     uint64_t tempty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
-    volatile unsigned int issued;    // stages the producer has armed (for the drain on abort)
 };
 
-template <bool NIBBLE>
-constexpr size_t smem_bytes() {
-    return 1024 + size_t(kStages) * (kABytes + kBBytes + (NIBBLE ? kRawBytes : 0)) + sizeof(SharedCtl) + 64;
+// Shared-memory carve-up (all offsets from a 1024-byte aligned base).
+struct SmemLayout { int b_off, a_off, staging_off, param_off, ctl_off, total; };
+__host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int num_kb) {
+    SmemLayout L;
+    L.b_off = 0;
+    L.a_off = (resident ? num_kb : stages) * kBBytes;
+    L.staging_off = L.a_off + stages * kABytes;
+    L.param_off = L.staging_off + kEpiWarps * kStagingBytes;
+    L.ctl_off = L.param_off + kParamBytes;
+    L.total = L.ctl_off + int(sizeof(SharedCtl)) + 1024;      // + slack for the base alignment
+    return L;
 }
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int32_t* dev_status,
@@ -87,10 +109,26 @@ struct TileCoord {
     int n0, h0, w0;      // conv: first image / output row / output column of the tile
 };
 
+// Tiles of one CTA: `count` tiles, the i-th being first + i * step.
+struct TileWalk { int first, step, count; };
+__device__ __forceinline__ TileWalk tile_walk(const GemmParams& p) {
+    const int T = p.tiles_m * p.tiles_n, G = gridDim.x, c = blockIdx.x;
+    TileWalk w;
+    if (p.b_resident) {
+        w.first = int(int64_t(c) * T / G);
+        w.count = int(int64_t(c + 1) * T / G) - w.first;
+        w.step = 1;
+    } else {
+        w.first = c; w.step = G;
+        w.count = c < T ? (T - c + G - 1) / G : 0;
+    }
+    return w;
+}
+
 __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile) {
     TileCoord t;
-    t.m_tile = tile / p.tiles_n;
-    t.n_tile = tile - t.m_tile * p.tiles_n;
+    if (p.b_resident) { t.n_tile = tile / p.tiles_m; t.m_tile = tile - t.n_tile * p.tiles_m; }
+    else { t.m_tile = tile / p.tiles_n; t.n_tile = tile - t.m_tile * p.tiles_n; }
     t.n0 = t.h0 = t.w0 = 0;
     if (p.conv) {
         const int tw = t.m_tile % p.tiles_w;
@@ -101,29 +139,111 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile) {
     return t;
 }
 
+// Output row (index into [M] / flattened NHWC pixels) of row `r` of a tile, or -1 if that row does not exist.
+__device__ __forceinline__ int out_row_of(const GemmParams& p, const TileCoord& tc, int r) {
+    if (p.conv) {
+        const int iw = r % p.bw;
+        const int ih = (r / p.bw) % p.bh;
+        const int in = r / (p.bw * p.bh);
+        const int n = tc.n0 + in, ho = tc.h0 + ih, wo = tc.w0 + iw;
+        if (in >= p.bn || n >= p.Nb || ho >= p.Ho || wo >= p.Wo) return -1;
+        return (n * p.Ho + ho) * p.Wo + wo;
+    }
+    const int64_t row = int64_t(tc.m_tile) * kBM + r;
+    return row < p.M ? int(row) : -1;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Staging buffer of one epilogue warp: 32 rows x 64 bytes, so that global stores are row-contiguous 16-byte
+// pieces.  A lane holds one output row and hands in 16 columns at a time.  ELT = 2: float bit patterns stored as
+// bf16, a staging row is 32 columns filled by two calls (`half` = 0, 1); ELT = 4: 32-bit words as they are, a
+// staging row is the 16 columns of one call.  The piece index is XOR-swizzled so that both the row-per-lane
+// writes and the row-contiguous reads are free of bank conflicts.
+template <int ELT>
+__device__ __forceinline__ void stage_put(unsigned char* stg, const uint32_t (&v)[16], int lane, int half) {
+    const int wsw = (lane >> 1) & 3;
+    if (ELT == 2) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+            w.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+            w.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+            w.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+            *reinterpret_cast<uint4*>(stg + lane * 64 + (((2 * half + j) ^ wsw) << 4)) = w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4*>(stg + lane * 64 + ((j ^ wsw) << 4)) =
+                make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    }
+}
+
+// Reads the staged rows back row-contiguously (4 lanes per row, 8 rows per pass) and stores them.
+// rows[i] is the output row of staging row (8 i + lane / 4), or -1; col0 is the column of piece 0.
+template <int ELT>
+__device__ __forceinline__ void stage_flush(unsigned char* stg, int lane, void* out, int64_t ld, int N, int col0,
+                                            const int (&rows)[4], bool vec_ok) {
+    constexpr int EPP = 16 / ELT;                  // elements per 16-byte piece
+    __syncwarp();
+    const int pc = lane & 3;
+    const int col = col0 + pc * EPP;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int srow = i * 8 + (lane >> 2);
+        const uint4 w = *reinterpret_cast<const uint4*>(stg + srow * 64 + ((pc ^ ((srow >> 1) & 3)) << 4));
+        const int grow = rows[i];
+        if (grow < 0 || col >= N) continue;
+        unsigned char* dst = static_cast<unsigned char*>(out) + (int64_t(grow) * ld + col) * ELT;
+        if (vec_ok && col + EPP <= N) {
+            *reinterpret_cast<uint4*>(dst) = w;
+        } else {
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int e = 0; e < EPP; ++e) {
+                if (col + e < N) {
+                    if (ELT == 2) reinterpret_cast<uint16_t*>(dst)[e] = uint16_t(ww[e >> 1] >> ((e & 1) * 16));
+                    else reinterpret_cast<uint32_t*>(dst)[e] = ww[e];
+                }
+            }
+        }
+    }
+    __syncwarp();
+}
+
 template <bool NIBBLE>
-__global__ void __launch_bounds__(NIBBLE ? 320 : 192, 1)
+__global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* sA = smem;
-    unsigned char* sB = sA + kStages * kABytes;
-    unsigned char* sRaw = sB + kStages * kBBytes;
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(sRaw + (NIBBLE ? kStages * kRawBytes : 0));
+    const int num_kb = p.kb_per_tap * p.taps;
+    const SmemLayout L = smem_layout(p.stages, p.b_resident != 0, num_kb);
+    unsigned char* sB = smem + L.b_off;
+    unsigned char* sA = smem + L.a_off;
+    unsigned char* sStage = smem + L.staging_off;
+    float* sParam = reinterpret_cast<float*>(smem + L.param_off);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + L.ctl_off);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_tiles = p.tiles_m * p.tiles_n;
-    const int num_kb = p.kb_per_tap * p.taps;
+    const TileWalk walk = tile_walk(p);
+    const int nstages = p.stages;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
             mbar_init(&ctl->empty[s], 1);
+            mbar_init(&ctl->rawread[s], 128);
             mbar_init(&ctl->unpacked[s], 128);
         }
-        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 4); }
+        for (int k = 0; k < kResidentKb; ++k) mbar_init(&ctl->bfull[k], 1);
+        mbar_init(&ctl->bfree, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], kEpiWarps); }
         ctl->abort_flag = 0;
-        ctl->issued = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
@@ -138,13 +258,25 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
+            int cur_n = -1, reloads = 0;
+            long long armed = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const TileCoord tc = tile_coord(p, tile);
+            for (int i = 0; i < walk.count && ok; ++i) {
+                const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+                if (p.b_resident && tc.n_tile != cur_n) {
+                    // the previous weight tile must have been read by its last MMA before it is overwritten
+                    if (reloads > 0 &&
+                        !wait_or_abort(&ctl->bfree, uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
+                    for (int kb = 0; kb < num_kb; ++kb) {
+                        mbar_expect_tx(&ctl->bfull[kb], kBBytes);
+                        tma_load_2d(sB + kb * kBBytes, &tmB, &ctl->bfull[kb], kb * kBK, tc.n_tile * kBN);
+                    }
+                    cur_n = tc.n_tile; ++reloads;
+                }
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_or_abort(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
-                    mbar_expect_tx(&ctl->full[stage], p.a_box_bytes + kBBytes);
-                    unsigned char* a_dst = NIBBLE ? sRaw + stage * kRawBytes : sA + stage * kABytes;
+                    mbar_expect_tx(&ctl->full[stage], p.a_box_bytes + (p.b_resident ? 0u : uint32_t(kBBytes)));
+                    unsigned char* a_dst = sA + stage * kABytes + (NIBBLE ? kABytes - kRawBytes : 0);
                     const int a_k = (NIBBLE ? kBK / 2 : kBK);
                     if (p.conv) {
                         const int tap = kb / p.kb_per_tap, kc = kb - tap * p.kb_per_tap;
@@ -154,9 +286,19 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     } else {
                         tma_load_2d(a_dst, &tmA, &ctl->full[stage], kb * a_k, tc.m_tile * kBM);
                     }
-                    tma_load_2d(sB + stage * kBBytes, &tmB, &ctl->full[stage], kb * kBK, tc.n_tile * kBN);
-                    ctl->issued = ctl->issued + 1;
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    if (!p.b_resident) tma_load_2d(sB + stage * kBBytes, &tmB, &ctl->full[stage], kb * kBK, tc.n_tile * kBN);
+                    ++armed;
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) {
+                // Abort path: wait (bounded) for the copies this thread started so none lands after the CTA exits.
+                if (reloads > 0)
+                    for (int kb = 0; kb < num_kb; ++kb) mbar_wait(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, nullptr, 0);
+                const int back = armed < nstages ? int(armed) : nstages;
+                for (int j = 0; j < back; ++j) {
+                    if (--stage < 0) { stage = nstages - 1; phase ^= 1; }
+                    mbar_wait(&ctl->full[stage], phase, nullptr, 0);
                 }
             }
         }
@@ -165,174 +307,200 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         if (lane == 0) {
             const uint32_t idesc = make_idesc_i8(kBM, kBN);
             int stage = 0; uint32_t phase = 0;
-            unsigned int consumed = 0;
+            int cur_n = -1, reloads = 0;
             bool ok = true;
-            int it = 0;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-                const int as = it & 1;
-                const uint32_t aphase = (it >> 1) & 1;
+            for (int i = 0; i < walk.count && ok; ++i) {
+                const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+                const int as = i & 1;
+                const uint32_t aphase = (i >> 1) & 1;
+                const bool new_b = p.b_resident && tc.n_tile != cur_n;
+                if (new_b) { cur_n = tc.n_tile; ++reloads; }
                 if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
                 for (int kb = 0; kb < num_kb; ++kb) {
+                    if (new_b && !wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
                     if (!wait_or_abort(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                    ++consumed;
                     if (NIBBLE) {
                         if (!wait_or_abort(&ctl->unpacked[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
                     }
                     tc_fence_after();
                     const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
-                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + stage * kBBytes));
+                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + (p.b_resident ? kb : stage) * kBBytes));
 #pragma unroll
                     for (int k = 0; k < kBK / 32; ++k)
                         mma_i8(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
                     mma_commit(&ctl->empty[stage]);
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
                 }
-                if (ok) mma_commit(&ctl->tfull[as]);
-            }
-            if (!ok) {
-                // Abort path: wait (bounded) for TMA copies already in flight so none lands after exit.
-                const unsigned int issued = ctl->issued;
-                while (consumed < issued) {
-                    mbar_wait(&ctl->full[stage], phase, nullptr, 0);
-                    ++consumed;
-                    if (++stage == kStages) { stage = 0; phase ^= 1; }
+                if (ok) {
+                    mma_commit(&ctl->tfull[as]);
+                    if (p.b_resident && i + 1 < walk.count &&
+                        tile_coord(p, walk.first + (i + 1) * walk.step).n_tile != cur_n)
+                        mma_commit(&ctl->bfree);
                 }
             }
         }
-    } else if (warp < 6) {
-        // ------------------------------------------------------------------ epilogue
+    } else if (warp < 2 + kEpiWarps) {
+        // ------------------------------------------------------------------ epilogue (warps 2-9)
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int r_in_tile = q * 32 + lane;
-        int it = 0;
+        const int chalf = (warp - 2) >> 2;            // which half of the tile's columns this warp takes
+        unsigned char* stg = sStage + (warp - 2) * kStagingBytes;
+        float* prm_sw = sParam + (warp - 2) * 2 * (kBN / 2);
+        float* prm_b = prm_sw + kBN / 2;
+        const int cols_per_tile = p.limbs == 2 ? kBN / 2 : kBN;
+        const int cols_per_warp = cols_per_tile / 2;
+        const bool want_y = p.y != nullptr, want_acc = p.acc_out != nullptr;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-            const int as = it & 1;
-            const uint32_t aphase = (it >> 1) & 1;
-            const TileCoord tc = tile_coord(p, tile);
+        for (int i = 0; i < walk.count && ok; ++i) {
+            const int as = i & 1;
+            const uint32_t aphase = (i >> 1) & 1;
+            const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+            const int col_base = tc.n_tile * cols_per_tile;
+            // This warp's columns [wc0, wc0 + cols_per_warp) of the tile; their scale_w / bias go to the warp's own
+            // slice of shared memory (read back as broadcasts), so no CTA-wide barrier is needed.
+            const int wc0 = chalf * cols_per_warp;
+            if (want_y) {
+                __syncwarp();
+                for (int c = lane; c < cols_per_warp; c += 32) {
+                    const int col = col_base + wc0 + c;
+                    prm_sw[c] = col < p.N ? __ldg(p.scale_w + col) : 0.f;
+                    prm_b[c] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
+                }
+                __syncwarp();
+            }
+            const int my_row = out_row_of(p, tc, q * 32 + lane);
+            float sa_eff = 0.f;
+            if (want_y && my_row >= 0) {
+                sa_eff = p.alpha * (p.sa_scalar ? __ldg(p.scale_a) : __ldg(p.scale_a + my_row));
+                if (p.combine_fast) sa_eff *= 1.0f / float(1 << p.a_shift);
+            }
+            int rows[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) rows[j] = out_row_of(p, tc, q * 32 + j * 8 + (lane >> 2));
             if (!wait_or_abort(&ctl->tfull[as], aphase, ctl, p.dev_status, kStatusAccumWait)) { ok = false; break; }
             tc_fence_after();
 
-            int64_t out_row; bool row_ok;
-            if (p.conv) {
-                const int iw = r_in_tile % p.bw;
-                const int ih = (r_in_tile / p.bw) % p.bh;
-                const int in = r_in_tile / (p.bw * p.bh);
-                const int n = tc.n0 + in, ho = tc.h0 + ih, wo = tc.w0 + iw;
-                row_ok = in < p.bn && n < p.Nb && ho < p.Ho && wo < p.Wo;
-                out_row = (int64_t(n) * p.Ho + ho) * p.Wo + wo;
-            } else {
-                out_row = int64_t(tc.m_tile) * kBM + r_in_tile;
-                row_ok = out_row < p.M;
+            // walk the warp's columns in steps of 16
+            int nsteps = cols_per_warp / 16;
+            if (col_base + wc0 + nsteps * 16 > p.N) {
+                const int left = p.N - (col_base + wc0);
+                nsteps = left > 0 ? (left + 15) / 16 : 0;
             }
-            float sa = 0.f;
-            if (row_ok && p.y != nullptr) sa = p.alpha * (p.sa_scalar ? __ldg(p.scale_a) : __ldg(p.scale_a + out_row));
-            const int cols_per_tile = p.limbs == 2 ? kBN / 2 : kBN;
-            const int col_base = tc.n_tile * cols_per_tile;
-            const uint32_t t_row = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN);
-
-            for (int ch = 0; ch < cols_per_tile / 32; ++ch) {
-                const int col0 = col_base + ch * 32;
-                if (col0 >= p.N) break;                 // uniform across the warp
-                uint32_t v[32];
-                tmem_ld_32x32(t_row + uint32_t(ch * 32), v);
+            const uint32_t t_row = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
+            uint32_t hi[16], lo[16];
+            if (nsteps > 0) {
+                tmem_ld_32x16(t_row, hi);
+                if (p.limbs == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
+            }
+            for (int st = 0; st < nsteps; ++st) {
+                const int tcol = wc0 + st * 16;        // column inside the tile
+                uint32_t val[16];
+                tmem_ld_wait_16(hi);
                 if (p.limbs == 2) {
-                    uint32_t lo[32];
-                    tmem_ld_32x32(t_row + uint32_t(kBN / 2 + ch * 32), lo);
-                    tmem_ld_wait();
+                    tmem_ld_wait_16(lo);
+                    if (p.combine_fast) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        v[j] = uint32_t(((int32_t(v[j]) >> p.a_shift) << 8) + (int32_t(lo[j]) >> p.a_shift));
-                } else {
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = uint32_t(int32_t(v[j]) >> p.a_shift);
-                }
-                if (!row_ok) continue;
-                const bool full_chunk = col0 + 32 <= p.N;
-                if (p.acc_out != nullptr) {
-                    int32_t* dst = p.acc_out + out_row * int64_t(p.N) + col0;
-                    if (full_chunk && (p.N & 3) == 0) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<uint4*>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        for (int j = 0; j < 16; ++j) val[j] = uint32_t(int32_t(hi[j]) * 256 + int32_t(lo[j]));
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) if (col0 + j < p.N) dst[j] = int32_t(v[j]);
+                        for (int j = 0; j < 16; ++j)
+                            val[j] = uint32_t(((int32_t(hi[j]) >> p.a_shift) << 8) + (int32_t(lo[j]) >> p.a_shift));
+                    }
+                } else if (p.combine_fast) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) val[j] = hi[j];
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) val[j] = uint32_t(int32_t(hi[j]) >> p.a_shift);
+                }
+                if (st + 1 < nsteps) {                 // the next step's loads fly while this one is processed
+                    tmem_ld_32x16(t_row + uint32_t((st + 1) * 16), hi);
+                    if (p.limbs == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2 + (st + 1) * 16), lo);
+                } else {                               // accumulator fully read: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->tempty[as]);
+                }
+                if (want_acc && my_row >= 0) {         // each lane stores 64 contiguous bytes of its own row
+                    int32_t* dst = p.acc_out + int64_t(my_row) * p.N + col_base + tcol;
+#pragma unroll
+                    for (int j = 0; j < 16; j += 4) {
+                        int32_t a4[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            a4[e] = p.combine_fast ? (int32_t(val[j + e]) >> p.a_shift) : int32_t(val[j + e]);
+                        if (p.acc_vec_ok && col_base + tcol + j + 4 <= p.N) {
+                            *reinterpret_cast<int4*>(dst + j) = make_int4(a4[0], a4[1], a4[2], a4[3]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) if (col_base + tcol + j + e < p.N) dst[j + e] = a4[e];
+                        }
                     }
                 }
-                if (p.y != nullptr) {
-                    float f[32];
+                if (want_y) {
+                    const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
+                    const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
+                    uint32_t f[16];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int c = col0 + j < p.N ? col0 + j : p.N - 1;
-                        const float sw = __ldg(p.scale_w + c);
-                        const float b = p.bias != nullptr ? __ldg(p.bias + c) : 0.f;
-                        f[j] = fmaf(float(int32_t(v[j])), sa * sw, b);
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 sw = sw4[j], bb = b4[j];
+                        f[4 * j + 0] = __float_as_uint(fmaf(float(int32_t(val[4 * j + 0])) * sw.x, sa_eff, bb.x));
+                        f[4 * j + 1] = __float_as_uint(fmaf(float(int32_t(val[4 * j + 1])) * sw.y, sa_eff, bb.y));
+                        f[4 * j + 2] = __float_as_uint(fmaf(float(int32_t(val[4 * j + 2])) * sw.z, sa_eff, bb.z));
+                        f[4 * j + 3] = __float_as_uint(fmaf(float(int32_t(val[4 * j + 3])) * sw.w, sa_eff, bb.w));
                     }
                     if (p.y_bf16) {
-                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.y) + out_row * p.ldy + col0;
-                        if (full_chunk && (p.ldy & 7) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                uint4 pk;
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[j], f[j + 1]);
-                                __nv_bfloat162 h1 = __floats2bfloat162_rn(f[j + 2], f[j + 3]);
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[j + 4], f[j + 5]);
-                                __nv_bfloat162 h3 = __floats2bfloat162_rn(f[j + 6], f[j + 7]);
-                                pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                                pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                                *reinterpret_cast<uint4*>(dst + j) = pk;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(f[j]);
-                        }
+                        stage_put<2>(stg, f, lane, st & 1);
+                        if ((st & 1) || st + 1 == nsteps)
+                            stage_flush<2>(stg, lane, p.y, p.ldy, p.N, col_base + wc0 + (st & ~1) * 16, rows,
+                                           p.y_vec_ok != 0);
                     } else {
-                        float* dst = reinterpret_cast<float*>(p.y) + out_row * p.ldy + col0;
-                        if (full_chunk && (p.ldy & 3) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(dst + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) if (col0 + j < p.N) dst[j] = f[j];
-                        }
+                        stage_put<4>(stg, f, lane, 0);
+                        stage_flush<4>(stg, lane, p.y, p.ldy, p.N, col_base + tcol, rows, p.y_vec_ok != 0);
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->tempty[as]);
+            if (nsteps == 0) {                         // this warp's columns lie beyond N: nothing to read
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->tempty[as]);
+            }
         }
     } else if (NIBBLE) {
-        // ------------------------------------------------------------------ nibble -> int8 unpack (warps 6-9)
-        const int t = threadIdx.x - 192;              // 0..127
+        // ------------------------------------------------------------------ nibble -> int8 unpack (warps 10-13)
+        // The packed tile (128 rows x 64 bytes) lands in the upper half of the 16 KB operand stage; every thread
+        // first takes its share into registers, then (after a barrier of the four warps) the stage is rewritten
+        // in place as 128 rows x 128 bytes with the 128-byte swizzle the MMA descriptor expects.
+        const int t = threadIdx.x - (2 + kEpiWarps) * 32;    // 0..127
         int stage = 0; uint32_t phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int i = 0; i < walk.count && ok; ++i) {
             for (int kb = 0; kb < num_kb; ++kb) {
                 if (!wait_or_abort(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                const uint4* raw = reinterpret_cast<const uint4*>(sRaw + stage * kRawBytes);
                 unsigned char* dstA = sA + stage * kABytes;
+                const uint4* raw = reinterpret_cast<const uint4*>(dstA + kABytes - kRawBytes);
+                uint4 w[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int id = i * 128 + t;           // 16-byte chunk of the packed tile: row = id/4, part = id%4
+                for (int j = 0; j < 4; ++j) w[j] = raw[j * 128 + t];
+                mbar_arrive(&ctl->rawread[stage]);     // the stage may be overwritten once all 128 threads got here
+                if (!wait_or_abort(&ctl->rawread[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int id = j * 128 + t;           // 16-byte chunk of the packed tile: row = id/4, part = id%4
                     const int row = id >> 2, part = id & 3;
-                    const uint4 w = raw[id];
                     uint4 o0, o1;
-                    o0.x = (w.x << 4) & 0xF0F0F0F0u; o0.y = w.x & 0xF0F0F0F0u;
-                    o0.z = (w.y << 4) & 0xF0F0F0F0u; o0.w = w.y & 0xF0F0F0F0u;
-                    o1.x = (w.z << 4) & 0xF0F0F0F0u; o1.y = w.z & 0xF0F0F0F0u;
-                    o1.z = (w.w << 4) & 0xF0F0F0F0u; o1.w = w.w & 0xF0F0F0F0u;
+                    o0.x = (w[j].x << 4) & 0xF0F0F0F0u; o0.y = w[j].x & 0xF0F0F0F0u;
+                    o0.z = (w[j].y << 4) & 0xF0F0F0F0u; o0.w = w[j].y & 0xF0F0F0F0u;
+                    o1.x = (w[j].z << 4) & 0xF0F0F0F0u; o1.y = w[j].z & 0xF0F0F0F0u;
+                    o1.z = (w[j].w << 4) & 0xF0F0F0F0u; o1.w = w[j].w & 0xF0F0F0F0u;
                     unsigned char* rowp = dstA + row * 128;
                     *reinterpret_cast<uint4*>(rowp + (((2 * part) ^ (row & 7)) << 4)) = o0;
                     *reinterpret_cast<uint4*>(rowp + (((2 * part + 1) ^ (row & 7)) << 4)) = o1;
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(&ctl->unpacked[stage]);
-                if (++stage == kStages) { stage = 0; phase ^= 1; }
+                if (++stage == nstages) { stage = 0; phase ^= 1; }
             }
         }
     }
@@ -425,20 +593,48 @@ int sm_count() {
     return cached[dev];
 }
 
+// Ring depth and weight residency for a problem; fills p.stages / p.b_resident and returns the shared-memory size.
 template <bool NIBBLE>
-hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, cudaStream_t st) {
+size_t plan_smem(GemmParams& p) {
+    const int num_kb = p.kb_per_tap * p.taps;
+    p.b_resident = num_kb <= kResidentKb ? 1 : 0;
+    for (int stages = kMaxStages; stages >= 2; --stages) {
+        const SmemLayout L = smem_layout(stages, p.b_resident != 0, num_kb);
+        if (L.total <= kSmemLimit) { p.stages = stages; return size_t(L.total); }
+    }
+    return 0;
+}
+
+template <bool NIBBLE>
+hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams& p, cudaStream_t st) {
     static bool attr_set[64] = {};
-    constexpr size_t smem = smem_bytes<NIBBLE>();
+    const size_t smem = plan_smem<NIBBLE>(p);
+    if (smem == 0) return HQ_ERR_UNSUPPORTED;
     int dev = 0;
     HQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        HQ_CUDA_OK(cudaFuncSetAttribute(qgemm_kernel<NIBBLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+        HQ_CUDA_OK(cudaFuncSetAttribute(qgemm_kernel<NIBBLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    qgemm_kernel<NIBBLE><<<grid, NIBBLE ? 320 : 192, smem, st>>>(tmA, tmB, p);
+    qgemm_kernel<NIBBLE><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, p);
     return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+// Epilogue settings shared by the GEMM and the convolution.
+void fill_epilogue(GemmParams& p, hq_container cont, int a_bits, const hq_weight_desc* desc, int64_t K_total,
+                   const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias, float alpha,
+                   int32_t* acc_out, void* y, hq_dtype ydt, int64_t ldy, int32_t* dev_status) {
+    p.a_shift = cont == HQ_CODES_NIBBLE ? 4 : 0;
+    // 256*hi + lo (one limb: the accumulator itself) of the shifted accumulators is (true value) << a_shift
+    const double bound = double(K_total) * double(1 << (a_bits - 1)) * double(desc->max_abs_b > 0 ? desc->max_abs_b : 1);
+    p.combine_fast = bound * double(1 << p.a_shift) < 2147483648.0 ? 1 : 0;
+    p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
+    p.acc_out = acc_out; p.y = y; p.y_bf16 = ydt == HQ_BF16; p.ldy = ldy; p.dev_status = dev_status;
+    const int yelt = ydt == HQ_BF16 ? 2 : 4;
+    p.y_vec_ok = y != nullptr && aligned16(y) && (ldy * yelt) % 16 == 0;
+    p.acc_vec_ok = acc_out != nullptr && aligned16(acc_out) && (int64_t(desc->N) * 4) % 16 == 0;
 }
 
 hq_status check_common(const void* a_codes, hq_container cont, int a_bits, const hq_weight_desc* desc,
@@ -479,14 +675,14 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     if (M > (int64_t(1) << 30)) return HQ_ERR_UNSUPPORTED;
 
     GemmParams p{};
-    p.M = M; p.N = int(desc->N); p.limbs = desc->limbs; p.a_shift = cont == HQ_CODES_NIBBLE ? 4 : 0;
+    p.M = M; p.N = int(desc->N); p.limbs = desc->limbs;
     p.kb_per_tap = int(desc->C_pad / kBK); p.taps = 1;
     p.tiles_m = int((M + kBM - 1) / kBM);
     p.tiles_n = int(desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
     p.a_box_bytes = cont == HQ_CODES_NIBBLE ? kRawBytes : kABytes;
     p.conv = 0;
-    p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
-    p.acc_out = acc_out; p.y = y; p.y_bf16 = ydt == HQ_BF16; p.ldy = ldy; p.dev_status = dev_status;
+    fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
+                  dev_status);
 
     CUtensorMap tmA, tmB;
     const bool nib = cont == HQ_CODES_NIBBLE;
@@ -517,7 +713,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     if (!scale_a_is_scalar && y != nullptr && R * S > 1) return HQ_ERR_UNSUPPORTED;   // per-tap rescale: separate kernel
 
     GemmParams p{};
-    p.N = int(desc->N); p.limbs = desc->limbs; p.a_shift = cont == HQ_CODES_NIBBLE ? 4 : 0;
+    p.N = int(desc->N); p.limbs = desc->limbs;
     p.kb_per_tap = int(desc->C_pad / kBK); p.taps = R * S;
     p.conv = 1; p.Nb = int(Nb); p.H = int(H); p.W = int(W); p.Ho = int(Ho); p.Wo = int(Wo);
     p.R = R; p.S = S; p.stride = stride; p.pad = pad;
@@ -535,8 +731,8 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     const bool nib = cont == HQ_CODES_NIBBLE;
     const int box_rows = p.bw * p.bh * p.bn;
     p.a_box_bytes = uint32_t(box_rows) * (nib ? kBK / 2 : kBK);
-    p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
-    p.acc_out = acc_out; p.y = y; p.y_bf16 = ydt == HQ_BF16; p.ldy = desc->N; p.dev_status = dev_status;
+    fill_epilogue(p, cont, a_bits, desc, int64_t(R) * S * C, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out,
+                  y, ydt, desc->N, dev_status);
 
     CUtensorMap tmA, tmB;
     const uint64_t dims[4] = {uint64_t(row_bytes), uint64_t(W), uint64_t(H), uint64_t(Nb)};
