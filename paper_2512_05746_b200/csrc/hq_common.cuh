@@ -44,26 +44,25 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One poll of a phase.  The suspend-time hint (ns) lets the hardware park the thread until the phase completes or
+// the time passes, instead of returning at once: waiting warps then leave the issue slots to the working ones.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(1000000u)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after about a second of polling, records `code` and returns false.
+// Bounded wait: gives up after about a second, records `code` and returns false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* dev_status, int32_t code) {
-    for (int it = 0; it < 2048; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (clock64() - t0 < 2000000000LL) {
+    while (clock64() - t0 < 2000000000LL)
         if (mbar_try_wait(bar, parity)) return true;
-        __nanosleep(32);
-    }
     if (dev_status) atomicExch(dev_status, code);
     return false;
 }

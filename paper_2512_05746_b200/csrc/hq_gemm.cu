@@ -91,13 +91,11 @@ __host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, SharedCtl* ctl, int32_t* dev_status,
                                               int32_t code) {
-    for (int it = 0; it < 4096; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (clock64() - t0 < 2000000000LL) {
+    while (clock64() - t0 < 2000000000LL) {           // each poll parks the thread for up to a millisecond
         if (mbar_try_wait(bar, parity)) return true;
         if (ctl->abort_flag) return false;
-        __nanosleep(32);
     }
     ctl->abort_flag = 1;
     if (dev_status) atomicExch(dev_status, code);
@@ -109,26 +107,36 @@ struct TileCoord {
     int n0, h0, w0;      // conv: first image / output row / output column of the tile
 };
 
-// Tiles of one CTA: `count` tiles, the i-th being first + i * step.
-struct TileWalk { int first, step, count; };
-__device__ __forceinline__ TileWalk tile_walk(const GemmParams& p) {
+// Tiles of one CTA, walked without divisions: `count` tiles starting at (m_tile, n_tile).  With resident weights a
+// CTA owns a contiguous range of the n-major tile order; otherwise tile c, c + G, c + 2G, ... of the m-major order.
+struct TileCursor { int m_tile, n_tile, count, dm, dn; };
+__device__ __forceinline__ TileCursor tile_begin(const GemmParams& p) {
     const int T = p.tiles_m * p.tiles_n, G = gridDim.x, c = blockIdx.x;
-    TileWalk w;
+    TileCursor t;
     if (p.b_resident) {
-        w.first = int(int64_t(c) * T / G);
-        w.count = int(int64_t(c + 1) * T / G) - w.first;
-        w.step = 1;
+        const int first = int(int64_t(c) * T / G);
+        t.count = int(int64_t(c + 1) * T / G) - first;
+        t.n_tile = first / p.tiles_m; t.m_tile = first - t.n_tile * p.tiles_m;
+        t.dm = t.dn = 0;
     } else {
-        w.first = c; w.step = G;
-        w.count = c < T ? (T - c + G - 1) / G : 0;
+        t.count = c < T ? (T - c + G - 1) / G : 0;
+        t.m_tile = c / p.tiles_n; t.n_tile = c - t.m_tile * p.tiles_n;
+        t.dm = G / p.tiles_n; t.dn = G - t.dm * p.tiles_n;
     }
-    return w;
+    return t;
+}
+__device__ __forceinline__ void tile_next(const GemmParams& p, TileCursor& t) {
+    if (p.b_resident) {
+        if (++t.m_tile == p.tiles_m) { t.m_tile = 0; ++t.n_tile; }
+    } else {
+        t.n_tile += t.dn; t.m_tile += t.dm;
+        if (t.n_tile >= p.tiles_n) { t.n_tile -= p.tiles_n; ++t.m_tile; }
+    }
 }
 
-__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, int tile) {
+__device__ __forceinline__ TileCoord tile_coord(const GemmParams& p, const TileCursor& cur) {
     TileCoord t;
-    if (p.b_resident) { t.n_tile = tile / p.tiles_m; t.m_tile = tile - t.n_tile * p.tiles_m; }
-    else { t.m_tile = tile / p.tiles_n; t.n_tile = tile - t.m_tile * p.tiles_n; }
+    t.m_tile = cur.m_tile; t.n_tile = cur.n_tile;
     t.n0 = t.h0 = t.w0 = 0;
     if (p.conv) {
         const int tw = t.m_tile % p.tiles_w;
@@ -216,6 +224,65 @@ __device__ __forceinline__ void stage_flush(unsigned char* stg, int lane, void* 
     __syncwarp();
 }
 
+// Epilogue of one warp for the common case: bf16 output with 16-byte aligned rows, all of the warp's columns inside
+// N, limbs recombined as 256*hi + lo without overflow.  Per 16 columns: two TMEM loads, one integer multiply-add,
+// int->float, two float operations per value, bf16 packing and two 16-byte staging stores; every 32 columns the
+// staged block is read back row-contiguously and stored (4 lanes per row, rows without an output are skipped).
+template <int LIMBS>
+__device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
+                                              const float* prm_b, float sa_eff, __nv_bfloat16* const (&dst)[4],
+                                              uint64_t* tempty_bar) {
+    constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
+    const uint32_t wsw = (lane >> 1) & 3;
+    unsigned char* wr = stg + lane * 64;
+    const unsigned char* rd = stg + (lane >> 2) * 64 + (((lane & 3) ^ ((lane >> 3) & 3)) << 4);
+    uint32_t hi[16], lo[16];
+    tmem_ld_32x16(t_row, hi);
+    if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
+#pragma unroll
+    for (int st = 0; st < NSTEPS; ++st) {
+        int32_t w[16];
+        tmem_ld_wait_16(hi);
+        if (LIMBS == 2) {
+            tmem_ld_wait_16(lo);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) w[j] = int32_t(hi[j]) * 256 + int32_t(lo[j]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) w[j] = int32_t(hi[j]);
+        }
+        if (st + 1 < NSTEPS) {
+            tmem_ld_32x16(t_row + uint32_t((st + 1) * 16), hi);
+            if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2 + (st + 1) * 16), lo);
+        } else {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar);
+        }
+        const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
+        const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float4 s0 = sw4[2 * j], s1 = sw4[2 * j + 1], c0 = b4[2 * j], c1 = b4[2 * j + 1];
+            uint4 o;
+            o.x = pack_bf16x2(fmaf(float(w[8 * j + 0]) * s0.x, sa_eff, c0.x), fmaf(float(w[8 * j + 1]) * s0.y, sa_eff, c0.y));
+            o.y = pack_bf16x2(fmaf(float(w[8 * j + 2]) * s0.z, sa_eff, c0.z), fmaf(float(w[8 * j + 3]) * s0.w, sa_eff, c0.w));
+            o.z = pack_bf16x2(fmaf(float(w[8 * j + 4]) * s1.x, sa_eff, c1.x), fmaf(float(w[8 * j + 5]) * s1.y, sa_eff, c1.y));
+            o.w = pack_bf16x2(fmaf(float(w[8 * j + 6]) * s1.z, sa_eff, c1.z), fmaf(float(w[8 * j + 7]) * s1.w, sa_eff, c1.w));
+            *reinterpret_cast<uint4*>(wr + (((2 * (st & 1) + j) ^ wsw) << 4)) = o;
+        }
+        if (st & 1) {
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rd + i * 512);
+                if (dst[i] != nullptr) *reinterpret_cast<uint4*>(dst[i] + (st >> 1) * 32) = v;
+            }
+            __syncwarp();
+        }
+    }
+}
+
 template <bool NIBBLE>
 __global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
@@ -230,7 +297,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + L.ctl_off);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const TileWalk walk = tile_walk(p);
+    const TileCursor walk = tile_begin(p);
     const int nstages = p.stages;
 
     if (threadIdx.x == 0) {
@@ -261,8 +328,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             int cur_n = -1, reloads = 0;
             long long armed = 0;
             bool ok = true;
-            for (int i = 0; i < walk.count && ok; ++i) {
-                const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+            TileCursor cur = walk;
+            for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur)) {
+                const TileCoord tc = tile_coord(p, cur);
                 if (p.b_resident && tc.n_tile != cur_n) {
                     // the previous weight tile must have been read by its last MMA before it is overwritten
                     if (reloads > 0 &&
@@ -309,12 +377,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             int stage = 0; uint32_t phase = 0;
             int cur_n = -1, reloads = 0;
             bool ok = true;
-            for (int i = 0; i < walk.count && ok; ++i) {
-                const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+            TileCursor cur = walk;
+            for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur)) {
                 const int as = i & 1;
                 const uint32_t aphase = (i >> 1) & 1;
-                const bool new_b = p.b_resident && tc.n_tile != cur_n;
-                if (new_b) { cur_n = tc.n_tile; ++reloads; }
+                const bool new_b = p.b_resident && cur.n_tile != cur_n;
+                if (new_b) { cur_n = cur.n_tile; ++reloads; }
                 if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
@@ -335,9 +403,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 }
                 if (ok) {
                     mma_commit(&ctl->tfull[as]);
-                    if (p.b_resident && i + 1 < walk.count &&
-                        tile_coord(p, walk.first + (i + 1) * walk.step).n_tile != cur_n)
-                        mma_commit(&ctl->bfree);
+                    // the next tile of the range starts a new weight tile: tell the producer when this one is done with
+                    if (p.b_resident && i + 1 < walk.count && cur.m_tile + 1 == p.tiles_m) mma_commit(&ctl->bfree);
                 }
             }
         }
@@ -352,15 +419,19 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int cols_per_warp = cols_per_tile / 2;
         const bool want_y = p.y != nullptr, want_acc = p.acc_out != nullptr;
         bool ok = true;
-        for (int i = 0; i < walk.count && ok; ++i) {
+        TileCursor cur = walk;
+        int last_n = -1;
+        float sa_next = 0.f;
+        for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur)) {
             const int as = i & 1;
             const uint32_t aphase = (i >> 1) & 1;
-            const TileCoord tc = tile_coord(p, walk.first + i * walk.step);
+            const TileCoord tc = tile_coord(p, cur);
             const int col_base = tc.n_tile * cols_per_tile;
             // This warp's columns [wc0, wc0 + cols_per_warp) of the tile; their scale_w / bias go to the warp's own
             // slice of shared memory (read back as broadcasts), so no CTA-wide barrier is needed.
             const int wc0 = chalf * cols_per_warp;
-            if (want_y) {
+            if (want_y && tc.n_tile != last_n) {       // consecutive tiles under resident weights share their columns
+                last_n = tc.n_tile;
                 __syncwarp();
                 for (int c = lane; c < cols_per_warp; c += 32) {
                     const int col = col_base + wc0 + c;
@@ -370,16 +441,43 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 __syncwarp();
             }
             const int my_row = out_row_of(p, tc, q * 32 + lane);
-            float sa_eff = 0.f;
-            if (want_y && my_row >= 0) {
-                sa_eff = p.alpha * (p.sa_scalar ? __ldg(p.scale_a) : __ldg(p.scale_a + my_row));
-                if (p.combine_fast) sa_eff *= 1.0f / float(1 << p.a_shift);
+            // the row scale of this tile was requested while the previous tile was processed
+            float sa_raw = sa_next;
+            if (i == 0 && want_y) {
+                if (p.sa_scalar) sa_raw = __ldg(p.scale_a);
+                else if (my_row >= 0) sa_raw = __ldg(p.scale_a + my_row);
+            }
+            int next_row = -1;
+            if (i + 1 < walk.count && want_y && !p.sa_scalar) {
+                TileCursor nx = cur;
+                tile_next(p, nx);
+                next_row = out_row_of(p, tile_coord(p, nx), q * 32 + lane);
             }
             int rows[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) rows[j] = out_row_of(p, tc, q * 32 + j * 8 + (lane >> 2));
             if (!wait_or_abort(&ctl->tfull[as], aphase, ctl, p.dev_status, kStatusAccumWait)) { ok = false; break; }
             tc_fence_after();
+            if (next_row >= 0) sa_next = __ldg(p.scale_a + next_row);
+            else if (p.sa_scalar) sa_next = sa_raw;
+            float sa_eff = 0.f;
+            if (want_y && my_row >= 0) {
+                sa_eff = p.alpha * sa_raw;
+                if (p.combine_fast) sa_eff *= 1.0f / float(1 << p.a_shift);
+            }
+            if (want_y && !want_acc && p.y_bf16 && p.y_vec_ok && p.combine_fast &&
+                col_base + wc0 + cols_per_warp <= p.N) {
+                __nv_bfloat16* dst[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    dst[j] = rows[j] >= 0 ? reinterpret_cast<__nv_bfloat16*>(p.y) + int64_t(rows[j]) * p.ldy +
+                                                (col_base + wc0 + (lane & 3) * 8)
+                                          : nullptr;
+                const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
+                if (p.limbs == 2) epilogue_fast<2>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, dst, &ctl->tempty[as]);
+                else epilogue_fast<1>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, dst, &ctl->tempty[as]);
+                continue;
+            }
 
             // walk the warp's columns in steps of 16
             int nsteps = cols_per_warp / 16;
