@@ -60,6 +60,7 @@ struct GemmParams {
     const float* scale_w; const float* bias; float alpha;
     int32_t* acc_out; void* y; int y_bf16; int64_t ldy;
     int y_vec_ok, acc_vec_ok;
+    int tma_store;        // bf16 output goes out through bulk tensor stores (rows of a tile are consecutive output rows)
     int32_t* dev_status;
 };
 
@@ -224,18 +225,19 @@ __device__ __forceinline__ void stage_flush(unsigned char* stg, int lane, void* 
     __syncwarp();
 }
 
-// Epilogue of one warp for the common case: bf16 output with 16-byte aligned rows, all of the warp's columns inside
-// N, limbs recombined as 256*hi + lo without overflow.  Per 16 columns: two TMEM loads, one integer multiply-add,
-// int->float, two float operations per value, bf16 packing and two 16-byte staging stores; every 32 columns the
-// staged block is read back row-contiguously and stored (4 lanes per row, rows without an output are skipped).
+// Epilogue of one warp for the common case: bf16 output written by bulk tensor stores, limbs recombined as
+// 256*hi + lo without overflow.  Per 16 columns: two TMEM loads, one integer multiply-add, int->float, two float
+// operations per value, bf16 packing and two 16-byte stores into the warp's staging buffer (32 rows x 64 bytes, laid
+// out in the 64-byte swizzle of the output tensor map); every 32 columns one lane hands the buffer to the copy
+// engine, which clips rows and columns beyond the output, and the warp carries on with the next columns.  Before
+// the buffer is written again the lane waits until the engine has read it.
 template <int LIMBS>
 __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
-                                              const float* prm_b, float sa_eff, __nv_bfloat16* const (&dst)[4],
-                                              uint64_t* tempty_bar) {
+                                              const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0,
+                                              int row0, uint64_t* tempty_bar) {
     constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
     const uint32_t wsw = (lane >> 1) & 3;
     unsigned char* wr = stg + lane * 64;
-    const unsigned char* rd = stg + (lane >> 2) * 64 + (((lane & 3) ^ ((lane >> 3) & 3)) << 4);
     uint32_t hi[16], lo[16];
     tmem_ld_32x16(t_row, hi);
     if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
@@ -259,6 +261,10 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar);
         }
+        if ((st & 1) == 0) {                           // the copy engine must be done reading the staging buffer
+            if (lane == 0) bulk_wait_read_all();
+            __syncwarp();
+        }
         const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
         const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
 #pragma unroll
@@ -272,20 +278,20 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
             *reinterpret_cast<uint4*>(wr + (((2 * (st & 1) + j) ^ wsw) << 4)) = o;
         }
         if (st & 1) {
+            fence_proxy_async_smem();                  // the lanes' writes become visible to the copy engine
             __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 v = *reinterpret_cast<const uint4*>(rd + i * 512);
-                if (dst[i] != nullptr) *reinterpret_cast<uint4*>(dst[i] + (st >> 1) * 32) = v;
+            if (lane == 0) {
+                tma_store_2d(tmY, stg, col0 + (st >> 1) * 32, row0);
+                bulk_commit_group();
             }
-            __syncwarp();
         }
     }
 }
 
 template <bool NIBBLE>
 __global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
-qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+             const __grid_constant__ CUtensorMap tmY, const GemmParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int num_kb = p.kb_per_tap * p.taps;
@@ -314,6 +320,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
+        if (p.tma_store) tma_prefetch_desc(&tmY);
     }
     if (warp == 1) { tmem_alloc(&ctl->tmem_base, kTmemCols); tmem_relinquish(); }
     tc_fence_before();
@@ -465,17 +472,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 sa_eff = p.alpha * sa_raw;
                 if (p.combine_fast) sa_eff *= 1.0f / float(1 << p.a_shift);
             }
-            if (want_y && !want_acc && p.y_bf16 && p.y_vec_ok && p.combine_fast &&
-                col_base + wc0 + cols_per_warp <= p.N) {
-                __nv_bfloat16* dst[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    dst[j] = rows[j] >= 0 ? reinterpret_cast<__nv_bfloat16*>(p.y) + int64_t(rows[j]) * p.ldy +
-                                                (col_base + wc0 + (lane & 3) * 8)
-                                          : nullptr;
+            if (p.tma_store && want_y && !want_acc && p.combine_fast) {
+                // rows of the tile are consecutive output rows (checked on the host); this warp owns 32 of them
+                const int row0 = out_row_of(p, tc, 0) + q * 32;
                 const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
-                if (p.limbs == 2) epilogue_fast<2>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, dst, &ctl->tempty[as]);
-                else epilogue_fast<1>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, dst, &ctl->tempty[as]);
+                if (p.limbs == 2)
+                    epilogue_fast<2>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
+                else
+                    epilogue_fast<1>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
                 continue;
             }
 
@@ -565,6 +569,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (lane == 0) mbar_arrive(&ctl->tempty[as]);
             }
         }
+        if (lane == 0) bulk_wait_read_all();           // shared memory must outlive the copy engine's reads
     } else if (NIBBLE) {
         // ------------------------------------------------------------------ nibble -> int8 unpack (warps 10-13)
         // The packed tile (128 rows x 64 bytes) lands in the upper half of the 16 KB operand stage; every thread
@@ -679,6 +684,20 @@ bool encode_4d(CUtensorMap* tm, const void* base, const uint64_t dims_in[4], con
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output tensor map for the epilogue's bulk stores: bf16 [rows][N] with pitch ldy, boxes of 32 rows x 32 columns
+// in the 64-byte swizzle the staging buffers are written in.
+bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[2] = {N, rows};
+    cuuint64_t strides[1] = {ldy * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(y), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count() {
     static int cached[64] = {};
     int dev = 0;
@@ -704,7 +723,8 @@ size_t plan_smem(GemmParams& p) {
 }
 
 template <bool NIBBLE>
-hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams& p, cudaStream_t st) {
+hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmParams& p,
+                 cudaStream_t st) {
     static bool attr_set[64] = {};
     const size_t smem = plan_smem<NIBBLE>(p);
     if (smem == 0) return HQ_ERR_UNSUPPORTED;
@@ -716,7 +736,7 @@ hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams& p, 
     }
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    qgemm_kernel<NIBBLE><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, p);
+    qgemm_kernel<NIBBLE><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
     return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
@@ -782,13 +802,16 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
                   dev_status);
 
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmY{};
     const bool nib = cont == HQ_CODES_NIBBLE;
     if (!encode_2d(&tmA, a_codes, uint64_t(row_bytes), uint64_t(M), uint64_t(lda), nib ? kBK / 2 : kBK, kBM, !nib))
         return HQ_ERR_CUDA;
+    // bf16 output: the epilogue hands 32 x 32 blocks to the copy engine (rows of a GEMM tile are consecutive)
+    p.tma_store = (y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast) ? 1 : 0;
+    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad);
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, kBN, true)) return HQ_ERR_CUDA;
-    return nib ? launch<true>(tmA, tmB, p, st) : launch<false>(tmA, tmB, p, st);
+    return nib ? launch<true>(tmA, tmB, tmY, p, st) : launch<false>(tmA, tmB, tmY, p, st);
 }
 
 hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
@@ -832,7 +855,12 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     fill_epilogue(p, cont, a_bits, desc, int64_t(R) * S * C, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out,
                   y, ydt, desc->N, dev_status);
 
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmY{};
+    // Bulk stores need the 128 rows of a tile to be 128 consecutive output pixels: full-width tiles that are either
+    // whole images or a whole number of row groups per image.
+    const bool rows_consecutive = p.bw == Wo && p.bw * p.bh * p.bn == kBM && (p.bh == Ho || (p.bn == 1 && Ho % p.bh == 0));
+    p.tma_store = (y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast && rows_consecutive) ? 1 : 0;
+    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(Nb * Ho * Wo), uint64_t(desc->N))) return HQ_ERR_CUDA;
     const uint64_t dims[4] = {uint64_t(row_bytes), uint64_t(W), uint64_t(H), uint64_t(Nb)};
     // With a traversal stride the box extent is given in input elements: stride * (pixels wanted).
     const uint32_t box[4] = {uint32_t(nib ? kBK / 2 : kBK), uint32_t(p.bw * stride), uint32_t(p.bh * stride), uint32_t(p.bn)};
@@ -841,7 +869,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     if (!encode_4d(&tmA, a_codes, dims, box, estr, !nib)) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad) * desc->RS;
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, kBN, true)) return HQ_ERR_CUDA;
-    return nib ? launch<true>(tmA, tmB, p, st) : launch<false>(tmA, tmB, p, st);
+    return nib ? launch<true>(tmA, tmB, tmY, p, st) : launch<false>(tmA, tmB, tmY, p, st);
 }
 
 }  // namespace hq
