@@ -89,13 +89,74 @@ __device__ __forceinline__ void quantize_pack(const float (&v)[32], float inv, i
     }
 }
 
-template <int KLOG, typename InT, bool INT8_OUT>
+template <int E, int LO, int HI>
+__device__ __forceinline__ void butterflies_e(float (&v)[E]) {
+#pragma unroll
+    for (int h = LO; h <= HI; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            if (!(i & h)) {
+                const float a = v[i], b = v[i | h];
+                v[i] = a + b;
+                v[i | h] = a - b;
+            }
+        }
+    }
+}
+
+__host__ __device__ constexpr int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
+
+// Rounds E values (ties to even, optional clamp) and packs them in register order into words: 8 four-bit codes or
+// 4 bytes per word.  Each rounded value is kMagicBits + (code + bias); summing the shifted bit patterns and removing
+// the shifted constants leaves the biased fields, which one XOR turns into two's complement.
+template <int E, bool INT8_OUT, bool CLAMP>
+__device__ __forceinline__ void round_pack(const float (&v)[E], float inv, int bits, uint32_t (&out)[INT8_OUT ? E / 4 : E / 8]) {
+    const float bias = INT8_OUT ? 128.0f : 8.0f;
+    const float mb = kMagic + bias;
+    const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
+    constexpr int PER_WORD = INT8_OUT ? 4 : 8;
+    constexpr int SHIFT = INT8_OUT ? 8 : 4;
+    uint32_t cst = 0;
+#pragma unroll
+    for (int e = 0; e < PER_WORD; ++e) cst += kMagicBits << (SHIFT * e);
+    constexpr uint32_t UNBIAS = INT8_OUT ? 0x80808080u : 0x88888888u;
+#pragma unroll
+    for (int w = 0; w < E / PER_WORD; ++w) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int e = 0; e < PER_WORD; ++e) {
+            float f = fmaf(v[w * PER_WORD + e], inv, mb);
+            if (CLAMP) f = fminf(fmaxf(f, lo), hi);
+            acc += __float_as_uint(f) << (SHIFT * e);
+        }
+        out[w] = (acc - cst) ^ UNBIAS;
+    }
+}
+
+// Fast path.  A Hadamard block of n = 2^KLOG channels is owned by TB = n / E threads that hold E values each.
+//   phase A  thread t holds the float4s {t + TB i}: coalesced 16-byte loads; the E-point in-register transform
+//            covers index bits {0, 1} and the top log2(E) - 2 bits;
+//   exchange one trip through shared memory (XOR-swizzled float4 slots, conflict-free both ways);
+//   phase B  the remaining R = KLOG - log2(E) index bits {2 .. R+1} are done in registers again.  If R leaves room
+//            for both low bits, thread u holds the E contiguous channels E u ..; otherwise (PAIR) it holds the
+//            channel pairs {4 j, 4 j + 1} + 2 (u & 1) of a 2E-channel group, read as float2, and after packing the
+//            two threads of a group interleave their bytes with one shuffle so that each stores contiguous bytes.
+//            KLOG = 12 needs one more stage than fits and takes it with a lane exchange.
+// Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
+template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC>
 __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     constexpr int N = 1 << KLOG;
-    constexpr int TB = N / 32;                         // threads per Hadamard block
+    constexpr int LE = ilog2_c(E);
+    constexpr int TB = N / E;                          // threads per Hadamard block
+    constexpr int R = KLOG - LE;                       // index bits left for phase B
+    constexpr bool PAIR = R >= LE - 1;
+    constexpr bool SHUF = R == LE;
+    static_assert(R <= LE, "block too large for this thread shape");
+    constexpr int J = PAIR ? E / 2 : E / 4;            // float4 slots a phase-B thread (pair) walks
+    constexpr int S = ilog2_c(J);
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float4* xch = reinterpret_cast<float4*>(smem_raw);                              // blockDim.x * 8 float4
-    unsigned int* rowmax = reinterpret_cast<unsigned int*>(smem_raw + size_t(blockDim.x) * 128);
+    float4* xch = reinterpret_cast<float4*>(smem_raw);                              // blockDim.x * E / 4 float4
+    unsigned int* rowmax = reinterpret_cast<unsigned int*>(smem_raw + size_t(blockDim.x) * E * 4);
 
     const int tid = threadIdx.x;
     const int row_in_cta = tid / p.threads_per_row;
@@ -106,46 +167,59 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     const bool valid = row < p.rows;
     const bool shared_max = (p.m > 1) || (TB > 32);
 
-    if (tid < p.rows_per_cta) rowmax[tid] = 0u;
+    if (!STATIC && tid < p.rows_per_cta) rowmax[tid] = 0u;
 
-    float v[32];
+    float v[E];
     {
         const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < E / 4; ++i) {
             float4 f = load4(src + 4 * (tb + TB * i));
             if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
             v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
         }
     }
-    butterflies<1, 16>(v);                             // index bits {0,1} and {k-3,k-2,k-1}
+    butterflies_e<E, 1, E / 2>(v);                     // index bits {0,1} and the top LE-2 bits
 
     float4* grp = xch + (tid / TB) * (N / 4);
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-        grp[swz(tb + TB * i)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float4 f = grp[swz(i + 8 * tb)];
-        v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+    for (int i = 0; i < E / 4; ++i) {
+        const int f = tb + TB * i;
+        grp[f ^ ((f >> S) & 7)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
     }
-    butterflies<4, 16>(v);                             // index bits {2,3,4}
+    if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
+    if (!PAIR) {
 #pragma unroll
-    for (int s = 0; s < KLOG - 8; ++s) {               // index bits 5 .. k-4 live in lane bits 0 .. k-9
-        const float sgn = ((tb >> s) & 1) ? -1.0f : 1.0f;
+        for (int j = 0; j < E / 4; ++j) {
+            const int f = J * tb + j;
+            const float4 q = grp[f ^ ((f >> S) & 7)];
+            v[4 * j + 0] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+        }
+        butterflies_e<E, 4, (4 << R) / 2>(v);          // index bits 2 .. R+1 are register bits 2 .. R+1
+    } else {
+        const float2* grp2 = reinterpret_cast<const float2*>(grp);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const float other = __shfl_xor_sync(0xffffffffu, v[e], 1 << s);
-            v[e] = fmaf(sgn, v[e], other);
+        for (int j = 0; j < E / 2; ++j) {
+            const int f = J * (tb >> 1) + j;
+            const float2 q = grp2[2 * (f ^ ((f >> S) & 7)) + (tb & 1)];
+            v[2 * j + 0] = q.x; v[2 * j + 1] = q.y;
+        }
+        butterflies_e<E, 2, E / 2>(v);                 // index bits 2 .. LE are register bits 1 .. LE-1
+        if (SHUF) {                                    // index bit LE+1 lives in lane bit 1
+            const float sgn = (tb & 2) ? -1.0f : 1.0f;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float other = __shfl_xor_sync(0xffffffffu, v[e], 2);
+                v[e] = fmaf(sgn, v[e], other);
+            }
         }
     }
 
     float inv, scale;
-    if (p.static_scale == nullptr) {
+    if (!STATIC) {
         float amax = 0.f;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) amax = fmaxf(amax, fabsf(v[e]));
+        for (int e = 0; e < E; ++e) amax = fmaxf(amax, fabsf(v[e]));
 #pragma unroll
         for (int off = 1; off < (TB < 32 ? TB : 32); off <<= 1)
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
@@ -168,21 +242,35 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
         inv = p.norm / scale;
     }
 
-    if (valid) {
-        uint8_t* dst = p.codes + row * p.ld_codes;
-        if (INT8_OUT) {
-            uint32_t w[8];
-            quantize_pack<true>(v, inv, p.bits, w);
-            uint4* d = reinterpret_cast<uint4*>(dst + int64_t(blk) * N + 32 * tb);
-            d[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            d[1] = make_uint4(w[4], w[5], w[6], w[7]);
-        } else {
-            uint32_t w[4];
-            quantize_pack<false>(v, inv, p.bits, w);
-            *reinterpret_cast<uint4*>(dst + (int64_t(blk) * N + 32 * tb) / 2) = make_uint4(w[0], w[1], w[2], w[3]);
+    constexpr int NW = INT8_OUT ? E / 4 : E / 8;       // packed words per thread
+    uint32_t w[NW];
+    round_pack<E, INT8_OUT, STATIC>(v, inv, p.bits, w);
+    if (PAIR) {
+        // w holds the codes of channel pairs {4j, 4j+1} (+2 for the odd thread).  The even thread of a pair emits
+        // the first half of the group's bytes, the odd thread the second half; each needs the other's words of
+        // that half, fetched with one exchange, and interleaves at pair granularity (1 byte or 2 bytes).
+        constexpr int H = NW / 2;
+        const bool odd = tb & 1;
+        uint32_t o[NW];
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+            const uint32_t send = odd ? w[i] : w[i + H];
+            const uint32_t keep = odd ? w[i + H] : w[i];
+            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+            const uint32_t ev = odd ? recv : keep, od = odd ? keep : recv;
+            o[2 * i + 0] = __byte_perm(ev, od, INT8_OUT ? 0x5410 : 0x5140);
+            o[2 * i + 1] = __byte_perm(ev, od, INT8_OUT ? 0x7632 : 0x7362);
         }
+#pragma unroll
+        for (int i = 0; i < NW; ++i) w[i] = o[i];
+    }
+    if (valid) {
+        uint8_t* dst = p.codes + row * p.ld_codes + (int64_t(blk) * N + E * tb) / (INT8_OUT ? 1 : 2);
+#pragma unroll
+        for (int i = 0; i < NW / 4; ++i)
+            reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
         if (p.scales != nullptr) {
-            if (p.static_scale == nullptr) { if (tr == 0) p.scales[row] = scale; }
+            if (!STATIC) { if (tr == 0) p.scales[row] = scale; }
             else if (row == 0 && tr == 0) p.scales[0] = scale;
         }
     }
@@ -261,22 +349,33 @@ __global__ void __launch_bounds__(256) fwht_quant_generic(const QuantParams p, i
     }
 }
 
-template <int KLOG, typename InT>
+template <int KLOG, int E, typename InT>
 cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threads, size_t smem, cudaStream_t st) {
-    if (int8_out) fwht_quant_fast<KLOG, InT, true><<<grid, threads, smem, st>>>(p);
-    else fwht_quant_fast<KLOG, InT, false><<<grid, threads, smem, st>>>(p);
-    return cudaGetLastError();
+    const bool stat = p.static_scale != nullptr;
+    auto go = [&](auto kern) -> cudaError_t {
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            if (e != cudaSuccess) return e;
+        }
+        kern<<<grid, threads, smem, st>>>(p);
+        return cudaGetLastError();
+    };
+    if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true>) : go(fwht_quant_fast<KLOG, E, InT, true, false>);
+    return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true>) : go(fwht_quant_fast<KLOG, E, InT, false, false>);
 }
+
+// Values per thread for a block of 2^klog channels.
+constexpr int fast_e(int klog) { return klog <= 9 ? 32 : 64; }
 
 template <typename InT>
 cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int grid, int threads, size_t smem,
                           cudaStream_t st) {
     switch (klog) {
-        case 8: return launch_fast<8, InT>(p, int8_out, grid, threads, smem, st);
-        case 9: return launch_fast<9, InT>(p, int8_out, grid, threads, smem, st);
-        case 10: return launch_fast<10, InT>(p, int8_out, grid, threads, smem, st);
-        case 11: return launch_fast<11, InT>(p, int8_out, grid, threads, smem, st);
-        case 12: return launch_fast<12, InT>(p, int8_out, grid, threads, smem, st);
+        case 8: return launch_fast<8, fast_e(8), InT>(p, int8_out, grid, threads, smem, st);
+        case 9: return launch_fast<9, fast_e(9), InT>(p, int8_out, grid, threads, smem, st);
+        case 10: return launch_fast<10, fast_e(10), InT>(p, int8_out, grid, threads, smem, st);
+        case 11: return launch_fast<11, fast_e(11), InT>(p, int8_out, grid, threads, smem, st);
+        case 12: return launch_fast<12, fast_e(12), InT>(p, int8_out, grid, threads, smem, st);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -314,19 +413,22 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
     p.scales = scales;
 
     const int elt = xdt == HQ_F32 ? 4 : 2;
-    const bool fast_ok = klog >= 8 && klog <= 12 && cols / 32 <= 256 &&
+    const int E = fast_e(klog);
+    const bool fast_ok = klog >= 8 && klog <= 12 && cols / E <= 256 &&
                          (reinterpret_cast<uintptr_t>(x) % (4 * elt) == 0) && (ldx % 4 == 0) &&
                          aligned16(codes) && (ld_codes % 16 == 0);
     if (fast_ok) {
-        const int tr = int(cols / 32);
+        // CTAs of about 128 threads (whole warps, whole rows): small enough that many are resident per SM and the
+        // load phases of some overlap the arithmetic of others.
+        const int tr = int(cols / E);
         int rpc = 1;
         while ((rpc * tr) % 32 != 0) ++rpc;                 // whole warps
         const int base = rpc;
-        while ((rpc + base) * tr <= 256) rpc += base;
+        while ((rpc + base) * tr <= 128) rpc += base;
         p.threads_per_row = tr;
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
-        const size_t smem = size_t(threads) * 128 + size_t(rpc) * 4;
+        const size_t smem = size_t(threads) * E * 4 + size_t(rpc) * 4;
         const int grid = int((rows + rpc - 1) / rpc);
         cudaError_t e = xdt == HQ_F32
                             ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
