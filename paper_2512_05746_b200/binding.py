@@ -193,6 +193,17 @@ def hq_workspace_size(rows: int, cols: int, container: int) -> int:
     return int(out.value)
 
 
+def workspace_views(workspace, rows: int, cols: int, container: int):
+    """The codes [rows, pitch] (uint8) and scales [rows] (fp32) a fused call left in its workspace (pure slicing)."""
+    import torch
+    row_bytes = cols // 2 if container == HQ_CODES_NIBBLE else cols
+    pitch = (row_bytes + 15) // 16 * 16
+    off = (rows * pitch + 255) // 256 * 256
+    codes = workspace[: rows * pitch].view(rows, pitch)
+    scales = workspace[off: off + rows * 4].view(torch.float32)
+    return codes, scales
+
+
 def hq_qlinear(x, pw: PreparedWeight, bias, a_bits: int, y, workspace, static_scale=None, dev_status=None,
                stream=None) -> None:
     M, K = x.shape

@@ -60,6 +60,8 @@ struct GemmParams {
     const float* scale_w; const float* bias; float alpha;
     int32_t* acc_out; void* y; int y_bf16; int64_t ldy;
     int y_vec_ok, acc_vec_ok;
+    int per_tap;          // convolution with one activation scale per input pixel: the accumulator is drained per filter tap
+    int col_pass;         // per_tap with one weight limb: which 64 of a warp's 128 columns this launch produces
     int tma_store;        // bf16 output goes out through bulk tensor stores (rows of a tile are consecutive output rows)
     int32_t* dev_status;
 };
@@ -225,6 +227,37 @@ __device__ __forceinline__ void stage_flush(unsigned char* stg, int lane, void* 
     __syncwarp();
 }
 
+// A lane's 16 consecutive output values (one row) stored straight to global memory, with bounds checks.
+// ELT = 2: float bit patterns stored as bf16; ELT = 4: 32-bit words as they are.
+template <int ELT>
+__device__ __forceinline__ void store_row16(void* out_row, const uint32_t (&v)[16], int col, int N, bool vec_ok) {
+    if (ELT == 2) {
+        __nv_bfloat16* d = static_cast<__nv_bfloat16*>(out_row) + col;
+        if (vec_ok && col + 16 <= N) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                reinterpret_cast<uint4*>(d)[j] = make_uint4(
+                    pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1])),
+                    pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
+                    pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
+                    pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) if (col + j < N) d[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+        }
+    } else {
+        uint32_t* d = static_cast<uint32_t*>(out_row) + col;
+        if (vec_ok && col + 16 <= N) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                reinterpret_cast<uint4*>(d)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) if (col + j < N) d[j] = v[j];
+        }
+    }
+}
+
 // Epilogue of one warp for the common case: bf16 output written by bulk tensor stores, limbs recombined as
 // 256*hi + lo without overflow.  Per 16 columns: two TMEM loads, one integer multiply-add, int->float, two float
 // operations per value, bf16 packing and two 16-byte stores into the warp's staging buffer (32 rows x 64 bytes, laid
@@ -288,7 +321,9 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
     }
 }
 
-template <bool NIBBLE>
+// PERTAP selects the per-filter-tap drain of the accumulator (one activation scale per input pixel); it is a separate
+// instantiation so that its register needs do not weigh on the common path.
+template <bool NIBBLE, bool PERTAP>
 __global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const GemmParams p) {
@@ -385,34 +420,40 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             int cur_n = -1, reloads = 0;
             bool ok = true;
             TileCursor cur = walk;
+            // One accumulator per tile, or (per-tap mode) one per filter tap of a tile; they alternate between the
+            // two TMEM buffers in the order they are produced.
+            const int groups = PERTAP ? p.taps : 1;
+            const int kb_per_group = num_kb / groups;
+            int seq = 0;
             for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur)) {
-                const int as = i & 1;
-                const uint32_t aphase = (i >> 1) & 1;
                 const bool new_b = p.b_resident && cur.n_tile != cur_n;
                 if (new_b) { cur_n = cur.n_tile; ++reloads; }
-                if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (new_b && !wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                    if (!wait_or_abort(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                    if (NIBBLE) {
-                        if (!wait_or_abort(&ctl->unpacked[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
-                    }
+                for (int g = 0; g < groups && ok; ++g, ++seq) {
+                    const int as = seq & 1;
+                    const uint32_t aphase = (seq >> 1) & 1;
+                    if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
-                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + (p.b_resident ? kb : stage) * kBBytes));
+                    const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                    for (int kk = 0; kk < kb_per_group; ++kk) {
+                        const int kb = g * kb_per_group + kk;
+                        if (new_b && !wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                        if (!wait_or_abort(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                        if (NIBBLE) {
+                            if (!wait_or_abort(&ctl->unpacked[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
+                        }
+                        tc_fence_after();
+                        const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
+                        const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + (p.b_resident ? kb : stage) * kBBytes));
 #pragma unroll
-                    for (int k = 0; k < kBK / 32; ++k)
-                        mma_i8(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
-                    mma_commit(&ctl->empty[stage]);
-                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                        for (int k = 0; k < kBK / 32; ++k)
+                            mma_i8(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kk | k) != 0 ? 1u : 0u);
+                        mma_commit(&ctl->empty[stage]);
+                        if (++stage == nstages) { stage = 0; phase ^= 1; }
+                    }
+                    if (ok) mma_commit(&ctl->tfull[as]);
                 }
-                if (ok) {
-                    mma_commit(&ctl->tfull[as]);
-                    // the next tile of the range starts a new weight tile: tell the producer when this one is done with
-                    if (p.b_resident && i + 1 < walk.count && cur.m_tile + 1 == p.tiles_m) mma_commit(&ctl->bfree);
-                }
+                // the next tile of the range starts a new weight tile: tell the producer when this one is done with
+                if (ok && p.b_resident && i + 1 < walk.count && cur.m_tile + 1 == p.tiles_m) mma_commit(&ctl->bfree);
             }
         }
     } else if (warp < 2 + kEpiWarps) {
@@ -446,6 +487,87 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     prm_b[c] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
                 }
                 __syncwarp();
+            }
+            if (PERTAP) {
+                // One scale per INPUT pixel: every filter tap's integer sum is drained on its own, multiplied by the
+                // scale of the pixel that tap read for this output pixel, and added up in fp32 registers (64 columns
+                // per warp and launch).  y = alpha * S_w[o] * sum_taps S_a[pix(tap)] * acc_tap + bias[o].
+                const int pc0 = p.limbs == 2 ? wc0 : wc0 + p.col_pass * 64;   // first column (in the tile) handled here
+                const int r_tile = q * 32 + lane;
+                const int iw = r_tile % p.bw, ih = (r_tile / p.bw) % p.bh, in_ = r_tile / (p.bw * p.bh);
+                const int n = tc.n0 + in_, ho = tc.h0 + ih, wo = tc.w0 + iw;
+                const bool row_ok = in_ < p.bn && n < p.Nb && ho < p.Ho && wo < p.Wo;
+                const int my_out = row_ok ? (n * p.Ho + ho) * p.Wo + wo : -1;
+                auto tap_scale = [&](int g) -> float {
+                    const int r = g / p.S, sx = g - r * p.S;
+                    const int hi_ = ho * p.stride + r - p.pad, wi_ = wo * p.stride + sx - p.pad;
+                    if (!row_ok || hi_ < 0 || hi_ >= p.H || wi_ < 0 || wi_ >= p.W) return 0.f;
+                    return __ldg(p.scale_a + (int64_t(n) * p.H + hi_) * p.W + wi_);
+                };
+                float run[64];
+#pragma unroll
+                for (int j = 0; j < 64; ++j) run[j] = 0.f;
+                float s_next = tap_scale(0);
+                for (int g = 0; g < p.taps && ok; ++g) {
+                    const int seq = i * p.taps + g;
+                    const int as2 = seq & 1;
+                    const float s_g = s_next;
+                    if (g + 1 < p.taps) s_next = tap_scale(g + 1);
+                    if (!wait_or_abort(&ctl->tfull[as2], uint32_t(seq >> 1) & 1u, ctl, p.dev_status, kStatusAccumWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t t_tap = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as2 * kBN + pc0);
+                    uint32_t hi[16], lo[16];
+                    tmem_ld_32x16(t_tap, hi);
+                    if (p.limbs == 2) tmem_ld_32x16(t_tap + uint32_t(kBN / 2), lo);
+#pragma unroll
+                    for (int st = 0; st < 4; ++st) {
+                        int32_t w[16];
+                        tmem_ld_wait_16(hi);
+                        if (p.limbs == 2) {
+                            tmem_ld_wait_16(lo);
+                            if (p.combine_fast) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) w[j] = int32_t(hi[j]) * 256 + int32_t(lo[j]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j)
+                                    w[j] = ((int32_t(hi[j]) >> p.a_shift) << 8) + (int32_t(lo[j]) >> p.a_shift);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) w[j] = p.combine_fast ? int32_t(hi[j]) : (int32_t(hi[j]) >> p.a_shift);
+                        }
+                        if (st < 3) {
+                            tmem_ld_32x16(t_tap + uint32_t((st + 1) * 16), hi);
+                            if (p.limbs == 2) tmem_ld_32x16(t_tap + uint32_t(kBN / 2 + (st + 1) * 16), lo);
+                        } else {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&ctl->tempty[as2]);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) run[st * 16 + j] = fmaf(float(w[j]), s_g, run[st * 16 + j]);
+                    }
+                }
+                if (!ok) break;
+                if (my_out >= 0) {
+                    const float a_eff = p.combine_fast ? p.alpha / float(1 << p.a_shift) : p.alpha;
+                    const int prm0 = pc0 - wc0;                    // offset into the warp's staged column parameters
+                    unsigned char* y_row = static_cast<unsigned char*>(p.y) + int64_t(my_out) * p.ldy * (p.y_bf16 ? 2 : 4);
+#pragma unroll
+                    for (int st = 0; st < 4; ++st) {
+                        uint32_t f[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            f[j] = __float_as_uint(fmaf(run[st * 16 + j] * prm_sw[prm0 + st * 16 + j], a_eff, prm_b[prm0 + st * 16 + j]));
+                        const int col = col_base + pc0 + st * 16;
+                        if (col < p.N) {
+                            if (p.y_bf16) store_row16<2>(y_row, f, col, p.N, p.y_vec_ok != 0);
+                            else store_row16<4>(y_row, f, col, p.N, p.y_vec_ok != 0);
+                        }
+                    }
+                }
+                continue;
             }
             const int my_row = out_row_of(p, tc, q * 32 + lane);
             // the row scale of this tile was requested while the previous tile was processed
@@ -731,12 +853,14 @@ hq_status launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorM
     int dev = 0;
     HQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        HQ_CUDA_OK(cudaFuncSetAttribute(qgemm_kernel<NIBBLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+        HQ_CUDA_OK(cudaFuncSetAttribute(qgemm_kernel<NIBBLE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+        HQ_CUDA_OK(cudaFuncSetAttribute(qgemm_kernel<NIBBLE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    qgemm_kernel<NIBBLE><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
+    if (p.per_tap) qgemm_kernel<NIBBLE, true><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
+    else qgemm_kernel<NIBBLE, false><<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
     return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
@@ -831,7 +955,15 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     const int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
     if (Ho <= 0 || Wo <= 0) return HQ_ERR_SHAPE;
     if (Nb * Ho * Wo > (int64_t(1) << 30)) return HQ_ERR_UNSUPPORTED;
-    if (!scale_a_is_scalar && y != nullptr && R * S > 1) return HQ_ERR_UNSUPPORTED;   // per-tap rescale: separate kernel
+    // One scale per input pixel under a window of several taps: the accumulator is drained per tap (see the kernel).
+    const bool per_tap = !scale_a_is_scalar && y != nullptr && R * S > 1;
+    if (per_tap && acc_out != nullptr) {
+        // the whole-window integer sums never exist in that mode: produce them with a launch of their own
+        s = launch_qconv2d(a_codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, nullptr, 1, nullptr,
+                           nullptr, 1.0f, acc_out, nullptr, ydt, dev_status, st);
+        if (s != HQ_OK) return s;
+        acc_out = nullptr;
+    }
 
     GemmParams p{};
     p.N = int(desc->N); p.limbs = desc->limbs;
@@ -859,17 +991,22 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     // Bulk stores need the 128 rows of a tile to be 128 consecutive output pixels: full-width tiles that are either
     // whole images or a whole number of row groups per image.
     const bool rows_consecutive = p.bw == Wo && p.bw * p.bh * p.bn == kBM && (p.bh == Ho || (p.bn == 1 && Ho % p.bh == 0));
-    p.tma_store = (y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast && rows_consecutive) ? 1 : 0;
+    p.per_tap = per_tap ? 1 : 0;
+    p.tma_store = (!per_tap && y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast && rows_consecutive) ? 1 : 0;
     if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(Nb * Ho * Wo), uint64_t(desc->N))) return HQ_ERR_CUDA;
     const uint64_t dims[4] = {uint64_t(row_bytes), uint64_t(W), uint64_t(H), uint64_t(Nb)};
     // With a traversal stride the box extent is given in input elements: stride * (pixels wanted).
     const uint32_t box[4] = {uint32_t(nib ? kBK / 2 : kBK), uint32_t(p.bw * stride), uint32_t(p.bh * stride), uint32_t(p.bn)};
     const uint32_t estr[4] = {1, uint32_t(stride), uint32_t(stride), 1};
-    if (stride != 1) return HQ_ERR_UNSUPPORTED;          // strided boxes: not enabled yet
     if (!encode_4d(&tmA, a_codes, dims, box, estr, !nib)) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad) * desc->RS;
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, kBN, true)) return HQ_ERR_CUDA;
-    return nib ? launch<true>(tmA, tmB, tmY, p, st) : launch<false>(tmA, tmB, tmY, p, st);
+    s = nib ? launch<true>(tmA, tmB, tmY, p, st) : launch<false>(tmA, tmB, tmY, p, st);
+    if (s == HQ_OK && per_tap && desc->limbs == 1) {      // the other 64 of every warp's 128 columns
+        p.col_pass = 1;
+        s = nib ? launch<true>(tmA, tmB, tmY, p, st) : launch<false>(tmA, tmB, tmY, p, st);
+    }
+    return s;
 }
 
 }  // namespace hq

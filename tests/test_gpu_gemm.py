@@ -162,6 +162,73 @@ def test_qconv2d_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, a_bits, 
     assert rel_err(y.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
 
 
+STRIDE2_CASES = [
+    # Nb, H, W, C, Cout, R, pad, mode, container
+    (2, 32, 32, 256, 256, 3, 1, "folded", 0),        # the down-sampling convolution of a UNet level
+    (3, 16, 16, 128, 192, 3, 1, "plain", 1),
+    (1, 17, 13, 128, 64, 3, 1, "plain", 0),          # odd sizes: the last window hangs over the padding
+    (2, 16, 16, 256, 128, 1, 0, "folded", 1),        # 1x1 stride 2 (a strided skip projection)
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,R,pad,mode,container", STRIDE2_CASES)
+def test_qconv2d_stride2_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, mode, container):
+    torch, hq = env
+    q = inputs.codes((Nb, H, W, C), 4, seed=H + C)
+    w = inputs.weights((Cout, R, R, C), seed=Cout)
+    pw = hq.hq_weight_prepare(w, 4, 128, hq.WEIGHT_MODES[mode], container).to_device()
+    B_ref = hq.decode_blob(pw).reshape(Cout, R, R, C)
+    Ho, Wo = (H + 2 * pad - R) // 2 + 1, (W + 2 * pad - R) // 2 + 1
+    acc = torch.full((Nb, Ho, Wo, Cout), 777, dtype=torch.int32, device="cuda")
+    y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    s_a = torch.tensor([0.03], device="cuda")
+    hq.hq_qconv2d(to_container(torch, hq, q, container), container, 4, Nb, H, W, C, pw, R, R, 2, pad, scale_a=s_a,
+                  alpha=pw.alpha, acc_out=acc, y=y, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    acc_ref = oracle.conv2d_int(q, B_ref, 2, pad)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    y_ref = oracle.dequant(acc_ref, np.array([0.03], np.float32), pw.s_w, None, pw.alpha)
+    assert rel_err(y.cpu().numpy(), y_ref) <= Y_F32_RTOL
+
+
+PERPIXEL_CASES = [
+    # Nb, H, W, C, Cout, stride, a_bits, mode, container, out dtype
+    (8, 32, 32, 256, 256, 1, 4, "folded", 0, "bf16"),    # the small conv configuration with its per-pixel scales
+    (8, 32, 32, 256, 256, 1, 3, "folded", 0, "bf16"),    # W4A3
+    (2, 16, 16, 128, 200, 1, 4, "folded", 1, "f32"),     # ragged Cout
+    (2, 16, 16, 128, 320, 1, 4, "plain", 1, "f32"),      # one weight limb: two column passes
+    (1, 20, 12, 128, 64, 1, 4, "plain", 0, "bf16"),      # ragged tiles
+    (2, 32, 32, 128, 128, 2, 4, "folded", 0, "f32"),     # stride 2
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,stride,a_bits,mode,container,odt", PERPIXEL_CASES)
+def test_qconv2d_per_pixel_scales(env, oracle, Nb, H, W, C, Cout, stride, a_bits, mode, container, odt):
+    """One activation scale per input pixel under a 3x3 window: every tap is rescaled by the scale of the pixel it
+    read.  The integer sums over the whole window are requested in the same call and must still be bit-exact."""
+    torch, hq = env
+    q = inputs.codes((Nb, H, W, C), a_bits, seed=H + W + C + a_bits)
+    w = inputs.weights((Cout, 3, 3, C), seed=Cout)
+    pw = hq.hq_weight_prepare(w, 4, 128, hq.WEIGHT_MODES[mode], container).to_device()
+    B_ref = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    b = inputs.bias(Cout, seed=3)
+    s_a = inputs.positive_scales(Nb * H * W, seed=7)
+    Ho, Wo = (H + 2 - 3) // stride + 1, (W + 2 - 3) // stride + 1
+    acc = torch.full((Nb, Ho, Wo, Cout), 777, dtype=torch.int32, device="cuda")
+    y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16 if odt == "bf16" else torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qconv2d(to_container(torch, hq, q, container), container, a_bits, Nb, H, W, C, pw, 3, 3, stride, 1,
+                  scale_a=torch.from_numpy(s_a).cuda(), bias=torch.from_numpy(b).cuda(), alpha=pw.alpha, acc_out=acc,
+                  y=y, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), oracle.conv2d_int(q, B_ref, stride, 1))
+    y_ref = oracle.conv2d_dequant_perpixel(q, s_a, B_ref, stride, 1, pw.s_w, b, pw.alpha)
+    assert rel_err(y.float().cpu().numpy(), y_ref) <= (Y_BF16_RTOL if odt == "bf16" else Y_F32_RTOL)
+
+
 def test_int8_tensor_pipe_probe_runs(env):
     torch, hq = env
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")

@@ -1,0 +1,118 @@
+"""GPU parity of the fused layer calls (hq_qlinear, hq_qconv): transform -> quantize -> integer product -> rescale.
+
+Two checks per case.  (1) The codes and scales the call left in its workspace follow the code acceptance rule
+against the oracle's.  (2) The output equals the oracle's rescale of the oracle's integer product of THOSE codes
+(the device's own), within the float tolerance -- so a code that legitimately differs at a rounding tie does not
+blur the output check.  For the small configurations the end-to-end distance to the all-oracle layer is bounded too.
+"""
+import numpy as np
+import pytest
+
+from paper_2512_05746_b200 import inputs
+from hq_testutil import SCALE_RTOL, Y_BF16_RTOL, check_codes, rel_err, unpack_nibbles_np
+
+pytestmark = pytest.mark.gpu
+
+
+def rms_rel(y, y_ref):
+    """||y - y_ref|| / ||y_ref||: the end-to-end distance to the all-oracle layer.  A code that differs at a rounding
+    tie moves a few outputs by one weight step, which the element-wise maximum would blow up; the norm does not."""
+    return float(np.sqrt(np.mean((y.astype(np.float64) - y_ref) ** 2)) / np.sqrt(np.mean(y_ref ** 2)))
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2512_05746_b200 import binding as hq
+    return torch, hq
+
+
+def _codes_from_ws(hq, ws, rows, cols, container):
+    codes, scales = hq.workspace_views(ws, rows, cols, container)
+    c = codes.cpu().numpy()
+    q = unpack_nibbles_np(c[:, : cols // 2]) if container == hq.HQ_CODES_NIBBLE else c[:, :cols].view(np.int8)
+    return q, scales.cpu().numpy()
+
+
+def run_linear(torch, hq, oracle, x, w, b, a_bits, had_block, mode, container, rows_checked=None):
+    M, K = x.shape
+    N = w.shape[0]
+    pw = hq.hq_weight_prepare(w, 4, had_block, hq.WEIGHT_MODES[mode], container).to_device()
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(M, K, container),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qlinear(torch.from_numpy(x).cuda(), pw, None if b is None else torch.from_numpy(b).cuda(), a_bits, y, ws,
+                  dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, M, K, container)
+    idx = np.arange(M) if rows_checked is None else rows_checked
+    ref = oracle.qlinear(x[idx], w, b, a_bits=a_bits, w_bits=4, had_block=had_block, weight_mode=mode)
+    assert np.allclose(s_gpu[idx], ref["s_a"], rtol=SCALE_RTOL, atol=0)
+    check_codes(q_gpu[idx], ref["q"], ref["v"], "fused linear")
+    B = hq.decode_blob(pw).reshape(N, K)
+    assert np.array_equal(B, ref["B"].reshape(N, K))
+    y_own = oracle.dequant(oracle.gemm_int(q_gpu[idx], B), s_gpu[idx], pw.s_w, b, pw.alpha)
+    y_gpu = y.float().cpu().numpy()[idx]
+    assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
+    return y_gpu, ref["y"]
+
+
+@pytest.mark.parametrize("mode,container,a_bits", [("folded", 0, 4), ("folded", 1, 4), ("plain", 0, 3), ("double", 1, 4)])
+def test_qlinear_small_configuration(env, oracle, mode, container, a_bits):
+    """X [256,256] with 4 outlier channels, W [256,256], Hadamard block 256, per-token INT4 / INT3, bf16 output."""
+    torch, hq = env
+    cfg = inputs.config_linear_small(0)
+    y_gpu, y_ref = run_linear(torch, hq, oracle, cfg["x"], cfg["w"], None, a_bits, 256, mode, container)
+    if mode != "plain":        # without the weight-side transform the layer is not meant to reproduce X W
+        assert rms_rel(y_gpu, y_ref) <= Y_BF16_RTOL
+
+
+@pytest.mark.parametrize("which", ["qkv", "ff2"])
+def test_qlinear_full_size_sampled_rows(env, oracle, which):
+    """A transformer-block linear at the benchmark's size (32768 tokens), checked on sampled rows."""
+    torch, hq = env
+    cfg = inputs.config_transformer_linear(which)
+    rows = np.sort(np.random.default_rng(1).choice(cfg["M"], size=64, replace=False))
+    rows[0], rows[-1] = 0, cfg["M"] - 1
+    run_linear(torch, hq, oracle, cfg["x"], cfg["w"], cfg["bias"], 4, cfg["had_block"], "folded", 0, rows_checked=rows)
+
+
+@pytest.mark.parametrize("a_bits,static", [(4, False), (3, False), (4, True)])
+def test_qconv_small_configuration(env, oracle, a_bits, static):
+    """NHWC [8,32,32,256] x [256,3,3,256], stride 1, pad 1, Hadamard over the input channels, per-pixel INT4 / INT3
+    (each tap rescaled by the scale of the pixel it read) or one static scale; bf16 output."""
+    torch, hq = env
+    cfg = inputs.config_conv_small(0)
+    x, w, b = cfg["x"], cfg["w"], cfg["bias"]
+    Nb, H, W, C = x.shape
+    Cout = w.shape[0]
+    pw = hq.hq_weight_prepare(w, 4, 256, hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE).to_device()
+    y = torch.zeros((Nb, H, W, Cout), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(Nb * H * W, C, hq.HQ_CODES_NIBBLE),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    s0 = 0.8 if static else None
+    ss = torch.tensor([s0], dtype=torch.float32, device="cuda") if static else None
+    hq.hq_qconv(torch.from_numpy(x).cuda(), pw, 3, 3, 1, 1, torch.from_numpy(b).cuda(), a_bits, y, ws, static_scale=ss,
+                dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    ref = oracle.qconv(x, w, b, a_bits=a_bits, w_bits=4, had_block=256, stride=1, pad=1, weight_mode="folded",
+                       static_scale=s0)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, Nb * H * W, C, hq.HQ_CODES_NIBBLE)
+    v = ref["v"].reshape(-1, C)
+    if static:
+        v = np.clip(v, oracle.qmin(a_bits) - 0.25, oracle.qmax(a_bits) + 0.25)
+        assert s_gpu[0] == np.float32(s0)
+    else:
+        assert np.allclose(s_gpu, ref["s_a"], rtol=SCALE_RTOL, atol=0)
+    check_codes(q_gpu, ref["q"].reshape(-1, C), v, "fused conv")
+    B = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    qg = q_gpu.reshape(Nb, H, W, C)
+    if static:
+        y_own = oracle.dequant(oracle.conv2d_int(qg, B, 1, 1), np.array([s0], np.float32), pw.s_w, b, pw.alpha)
+    else:
+        y_own = oracle.conv2d_dequant_perpixel(qg, s_gpu, B, 1, 1, pw.s_w, b, pw.alpha)
+    assert rel_err(y.float().cpu().numpy(), y_own) <= Y_BF16_RTOL
+    assert rms_rel(y.float().cpu().numpy(), ref["y"]) <= Y_BF16_RTOL
