@@ -89,31 +89,51 @@ __device__ __forceinline__ void quantize_pack(const float (&v)[32], float inv, i
     }
 }
 
-template <int E, int LO, int HI>
-__device__ __forceinline__ void butterflies_e(float (&v)[E]) {
+// ---- two-wide fp32 arithmetic (one instruction for a pair of values held in a 64-bit register) -----------------
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk2(float lo, float hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+
+// Butterflies over pair-index bits: element distance 2*h for h = LO .. HI (pairs stay pairs).
+template <int P, int LO, int HI>
+__device__ __forceinline__ void butterflies_pairs(f32x2 (&v)[P]) {
 #pragma unroll
     for (int h = LO; h <= HI; h <<= 1) {
 #pragma unroll
-        for (int i = 0; i < E; ++i) {
+        for (int i = 0; i < P; ++i) {
             if (!(i & h)) {
-                const float a = v[i], b = v[i | h];
-                v[i] = a + b;
-                v[i | h] = a - b;
+                const f32x2 a = v[i], b = v[i | h];
+                v[i] = add2(a, b);
+                v[i | h] = sub2(a, b);
             }
         }
+    }
+}
+// The stage between the two values of each pair.
+template <int P>
+__device__ __forceinline__ void butterfly_within_pairs(f32x2 (&v)[P]) {
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        float a, b;
+        upk2(v[i], a, b);
+        v[i] = pk2(a + b, a - b);
     }
 }
 
 __host__ __device__ constexpr int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
 
-// Rounds E values (ties to even, optional clamp) and packs them in register order into words: 8 four-bit codes or
-// 4 bytes per word.  Each rounded value is kMagicBits + (code + bias); summing the shifted bit patterns and removing
-// the shifted constants leaves the biased fields, which one XOR turns into two's complement.
+// Rounds E values held as pairs (ties to even, optional clamp) and packs them in register order into words: 8
+// four-bit codes or 4 bytes per word.  Each rounded value is kMagicBits + (code + bias); summing the shifted bit
+// patterns and removing the shifted constants leaves the biased fields, which one XOR turns into two's complement.
 template <int E, bool INT8_OUT, bool CLAMP>
-__device__ __forceinline__ void round_pack(const float (&v)[E], float inv, int bits, uint32_t (&out)[INT8_OUT ? E / 4 : E / 8]) {
+__device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, int bits, uint32_t (&out)[INT8_OUT ? E / 4 : E / 8]) {
     const float bias = INT8_OUT ? 128.0f : 8.0f;
     const float mb = kMagic + bias;
     const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
+    const f32x2 inv2 = pk2(inv, inv), mb2 = pk2(mb, mb);
     constexpr int PER_WORD = INT8_OUT ? 4 : 8;
     constexpr int SHIFT = INT8_OUT ? 8 : 4;
     uint32_t cst = 0;
@@ -124,19 +144,23 @@ __device__ __forceinline__ void round_pack(const float (&v)[E], float inv, int b
     for (int w = 0; w < E / PER_WORD; ++w) {
         uint32_t acc = 0;
 #pragma unroll
-        for (int e = 0; e < PER_WORD; ++e) {
-            float f = fmaf(v[w * PER_WORD + e], inv, mb);
-            if (CLAMP) f = fminf(fmaxf(f, lo), hi);
-            acc += __float_as_uint(f) << (SHIFT * e);
+        for (int e = 0; e < PER_WORD; e += 2) {
+            float f0, f1;
+            upk2(fma2(v[(w * PER_WORD + e) / 2], inv2, mb2), f0, f1);
+            if (CLAMP) { f0 = fminf(fmaxf(f0, lo), hi); f1 = fminf(fmaxf(f1, lo), hi); }
+            acc += __float_as_uint(f0) << (SHIFT * e);
+            acc += __float_as_uint(f1) << (SHIFT * (e + 1));
         }
         out[w] = (acc - cst) ^ UNBIAS;
     }
 }
 
-// Fast path.  A Hadamard block of n = 2^KLOG channels is owned by TB = n / E threads that hold E values each.
+// Fast path.  A Hadamard block of n = 2^KLOG channels is owned by TB = n / E threads that hold E values each, as
+// E/2 two-wide registers (butterflies between pairs are one instruction per two values).
 //   phase A  thread t holds the float4s {t + TB i}: coalesced 16-byte loads; the E-point in-register transform
 //            covers index bits {0, 1} and the top log2(E) - 2 bits;
-//   exchange one trip through shared memory (XOR-swizzled float4 slots, conflict-free both ways);
+//   exchange one trip through shared memory; float4 slot f sits at f + f / J (one slot of padding per J), which
+//            makes both access patterns conflict-free with addresses that are a base plus compile-time offsets;
 //   phase B  the remaining R = KLOG - log2(E) index bits {2 .. R+1} are done in registers again.  If R leaves room
 //            for both low bits, thread u holds the E contiguous channels E u ..; otherwise (PAIR) it holds the
 //            channel pairs {4 j, 4 j + 1} + 2 (u & 1) of a 2E-channel group, read as float2, and after packing the
@@ -147,6 +171,7 @@ template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC>
 __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     constexpr int N = 1 << KLOG;
     constexpr int LE = ilog2_c(E);
+    constexpr int P = E / 2;                           // two-wide registers per thread
     constexpr int TB = N / E;                          // threads per Hadamard block
     constexpr int R = KLOG - LE;                       // index bits left for phase B
     constexpr bool PAIR = R >= LE - 1;
@@ -154,9 +179,11 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     static_assert(R <= LE, "block too large for this thread shape");
     constexpr int J = PAIR ? E / 2 : E / 4;            // float4 slots a phase-B thread (pair) walks
     constexpr int S = ilog2_c(J);
+    static_assert(TB % J == 0 || TB == J, "exchange layout needs TB to be a multiple of J");
+    constexpr int GS = N / 4 + (N / 4) / J;            // padded float4 slots per Hadamard block
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float4* xch = reinterpret_cast<float4*>(smem_raw);                              // blockDim.x * E / 4 float4
-    unsigned int* rowmax = reinterpret_cast<unsigned int*>(smem_raw + size_t(blockDim.x) * E * 4);
+    float4* xch = reinterpret_cast<float4*>(smem_raw);
+    unsigned int* rowmax = reinterpret_cast<unsigned int*>(smem_raw + size_t(blockDim.x / TB) * GS * 16);
 
     const int tid = threadIdx.x;
     const int row_in_cta = tid / p.threads_per_row;
@@ -169,48 +196,47 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
 
     if (!STATIC && tid < p.rows_per_cta) rowmax[tid] = 0u;
 
-    float v[E];
+    f32x2 v[P];
     {
         const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
 #pragma unroll
         for (int i = 0; i < E / 4; ++i) {
             float4 f = load4(src + 4 * (tb + TB * i));
             if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
-            v[4 * i + 0] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+            v[2 * i] = pk2(f.x, f.y);
+            v[2 * i + 1] = pk2(f.z, f.w);
         }
     }
-    butterflies_e<E, 1, E / 2>(v);                     // index bits {0,1} and the top LE-2 bits
+    butterfly_within_pairs<P>(v);                      // index bit 0
+    butterflies_pairs<P, 1, P / 2>(v);                 // index bit 1 and the top LE-2 bits
 
-    float4* grp = xch + (tid / TB) * (N / 4);
+    float4* grp = xch + (tid / TB) * GS;
+    {
+        ulonglong2* wr = reinterpret_cast<ulonglong2*>(grp + tb + (tb >> S));
 #pragma unroll
-    for (int i = 0; i < E / 4; ++i) {
-        const int f = tb + TB * i;
-        grp[f ^ ((f >> S) & 7)] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        for (int i = 0; i < E / 4; ++i) wr[i * (TB + (TB >> S))] = make_ulonglong2(v[2 * i], v[2 * i + 1]);
     }
     if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
     if (!PAIR) {
+        const ulonglong2* rd = reinterpret_cast<const ulonglong2*>(grp + (J + 1) * tb);
 #pragma unroll
         for (int j = 0; j < E / 4; ++j) {
-            const int f = J * tb + j;
-            const float4 q = grp[f ^ ((f >> S) & 7)];
-            v[4 * j + 0] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+            const ulonglong2 q = rd[j];
+            v[2 * j] = q.x; v[2 * j + 1] = q.y;
         }
-        butterflies_e<E, 4, (4 << R) / 2>(v);          // index bits 2 .. R+1 are register bits 2 .. R+1
+        butterflies_pairs<P, 2, (2 << R) / 2>(v);      // index bits 2 .. R+1 are pair-index bits 1 .. R
     } else {
-        const float2* grp2 = reinterpret_cast<const float2*>(grp);
+        const f32x2* rd = reinterpret_cast<const f32x2*>(grp + (J + 1) * (tb >> 1)) + (tb & 1);
 #pragma unroll
-        for (int j = 0; j < E / 2; ++j) {
-            const int f = J * (tb >> 1) + j;
-            const float2 q = grp2[2 * (f ^ ((f >> S) & 7)) + (tb & 1)];
-            v[2 * j + 0] = q.x; v[2 * j + 1] = q.y;
-        }
-        butterflies_e<E, 2, E / 2>(v);                 // index bits 2 .. LE are register bits 1 .. LE-1
+        for (int j = 0; j < P; ++j) v[j] = rd[2 * j];
+        butterflies_pairs<P, 1, P / 2>(v);             // index bits 2 .. LE are pair-index bits 0 .. LE-2
         if (SHUF) {                                    // index bit LE+1 lives in lane bit 1
             const float sgn = (tb & 2) ? -1.0f : 1.0f;
+            const f32x2 sgn2 = pk2(sgn, sgn);
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float other = __shfl_xor_sync(0xffffffffu, v[e], 2);
-                v[e] = fmaf(sgn, v[e], other);
+            for (int e = 0; e < P; ++e) {
+                const f32x2 other = __shfl_xor_sync(0xffffffffu, v[e], 2);
+                v[e] = fma2(sgn2, v[e], other);
             }
         }
     }
@@ -219,7 +245,11 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     if (!STATIC) {
         float amax = 0.f;
 #pragma unroll
-        for (int e = 0; e < E; ++e) amax = fmaxf(amax, fabsf(v[e]));
+        for (int e = 0; e < P; ++e) {
+            float a, b;
+            upk2(v[e], a, b);
+            amax = fmaxf(fmaxf(amax, fabsf(a)), fabsf(b));
+        }
 #pragma unroll
         for (int off = 1; off < (TB < 32 ? TB : 32); off <<= 1)
             amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
@@ -428,7 +458,9 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
         p.threads_per_row = tr;
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
-        const size_t smem = size_t(threads) * E * 4 + size_t(rpc) * 4;
+        // exchange buffer: per Hadamard block n/4 float4 slots plus one slot of padding per J (J = E/2 or E/4)
+        const int jslots = (klog - ilog2(E) >= ilog2(E) - 1) ? E / 2 : E / 4;
+        const size_t smem = size_t(threads / (n / E)) * size_t(n / 4 + n / 4 / jslots) * 16 + size_t(rpc) * 4;
         const int grid = int((rows + rpc - 1) / rpc);
         cudaError_t e = xdt == HQ_F32
                             ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
