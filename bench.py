@@ -214,7 +214,7 @@ def oracle_sample_step(orc, sample_rows, seed):
     return ops, time.perf_counter() - t0
 
 
-def cpu_baseline(sample_rows=256, seed=0):
+def cpu_baseline(sample_rows=8192, seed=0):
     import oracle as orc
     orc.lib()
     ops, sec = oracle_sample_step(orc, sample_rows, seed)
@@ -230,7 +230,7 @@ def main_reference(args):
         return
     import oracle as orc
     orc.lib()
-    sample_rows = 256
+    sample_rows = 2048
     for _ in range(min(args.warmup, 1)):
         oracle_sample_step(orc, 64, 0)
     tot_ops, tot_sec = 0.0, 0.0
@@ -341,10 +341,8 @@ def main():
     barrier()
     e2e_ms = f0.elapsed_time(f1)
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(t[0]), float(t[1])
+    from paper_2512_05746_b200.sharding import max_over_ranks
+    ms, e2e_ms = max_over_ranks(ms, device), max_over_ranks(e2e_ms, device)
 
     ops_step = sum(L["ops"] for L in layers)
     ops_step_1 = sum(L["ops_1limb"] for L in layers)
