@@ -249,6 +249,97 @@ def main_reference(args):
     print(json.dumps(line))
 
 
+def main_unet(args):
+    """All 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent), one after the other on one
+    stream, bf16 activations, W4A4 with folded two-limb weights.  3x3 convolutions use one static activation scale,
+    1x1 convolutions and linears per-row scales.  The bf16 glue between the layers is not part of this path."""
+    import torch
+    from paper_2512_05746_b200 import binding as hq
+    from paper_2512_05746_b200 import unet
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    layers = unet.quantized_layers()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    cache = {}
+
+    def key(L):
+        return ("conv", L["Nb"], L["H"], L["C"], L["Cout"], L["R"], L["stride"]) if L["kind"] == "conv" else \
+               ("linear", L["M"], L["K"], L["N"])
+
+    status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    for L in layers:
+        k = key(L)
+        if k in cache:
+            L["res"] = cache[k]
+            continue
+        if L["kind"] == "conv":
+            rows, cin, cout = L["Nb"] * L["H"] * L["W"], L["C"], L["Cout"]
+            wshape = (cout, L["R"], L["R"], cin)
+            ho = L["H"] // L["stride"]
+            oshape = (L["Nb"], ho, ho, cout)
+        else:
+            rows, cin, cout = L["M"], L["K"], L["N"]
+            wshape = (cout, cin)
+            oshape = (rows, cout)
+        x = torch.randn((rows, cin), generator=gen, device=dev, dtype=torch.float32)
+        nout = max(1, round(0.01 * cin))
+        x[:, torch.randperm(cin, generator=gen, device=dev)[:nout]] *= 20.0          # outlier channels
+        x = x.to(torch.bfloat16)
+        pw = hq.hq_weight_prepare(inputs.weights(wshape, seed=len(cache)), W_BITS, L["had_block"], hq.HQ_W_FOLDED,
+                                  hq.HQ_CODES_NIBBLE).to_device(dev)
+        res = dict(x=x.view((L["Nb"], L["H"], L["W"], cin)) if L["kind"] == "conv" else x, pw=pw,
+                   bias=torch.from_numpy(inputs.bias(cout, seed=len(cache))).to(dev),
+                   y=torch.empty(oshape, dtype=torch.bfloat16, device=dev),
+                   ws=torch.empty((hq.hq_workspace_size(rows, cin, hq.HQ_CODES_NIBBLE),), dtype=torch.uint8, device=dev),
+                   static=None)
+        if L["kind"] == "conv" and L["R"] == 3:           # calibrate the static scale with one dynamic pass
+            codes = torch.empty((rows, cin // 2), dtype=torch.uint8, device=dev)
+            sc = torch.empty((rows,), dtype=torch.float32, device=dev)
+            hq.hq_hadamard_quant(x, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=sc)
+            res["static"] = sc.max().reshape(1).contiguous()
+            del codes, sc
+        cache[k] = res
+        L["res"] = res
+    torch.cuda.synchronize()
+
+    def forward():
+        for L in layers:
+            r = L["res"]
+            if L["kind"] == "conv":
+                hq.hq_qconv(r["x"], r["pw"], L["R"], L["R"], L["stride"], L["pad"], r["bias"], A_BITS, r["y"], r["ws"],
+                            static_scale=r["static"], dev_status=status)
+            else:
+                hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
+
+    steps, warmup = max(1, min(args.steps, 10)), max(3, min(args.warmup, 5))
+    for _ in range(warmup):
+        forward()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        forward()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.stop()
+    hq.hq_check_status(status)
+    macs = sum(L["macs"] for L in layers)
+    ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
+    print(json.dumps(dict(metric="forwards/s of the 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent)",
+                          value=1e3 / ms, unit="forwards/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=ms,
+                          higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int8", data="synthetic",
+                          config=dict(workload="configs[3] quantized layers only: 121 layers, 47 distinct shapes, bf16 in/out, "
+                                               "W4A4 folded two-limb weights, nibble codes", layers=len(layers),
+                                      layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
+                                      tops_1limb_equiv=2.0 * macs / ms / 1e9,
+                                      l2="activations of the large layers exceed L2"),
+                          clocks=clocks, gpu_launches=2 * len(layers) * steps)))
+
+
 def main():
     global M_TOKENS, WORKLOAD
     ap = argparse.ArgumentParser()
@@ -257,6 +348,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="step", choices=["step", "unet"],
+                    help="step: the benchmark step (default); unet: the 121 quantized layers of the UNet-shaped workload")
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     args = ap.parse_args()
@@ -265,6 +358,8 @@ def main():
         WORKLOAD = f"REDUCED to {M_TOKENS} rows per layer (profiling case, not a benchmark number): " + WORKLOAD
     if args.impl == "reference":
         return main_reference(args)
+    if args.workload == "unet":
+        return main_unet(args)
 
     import torch
     import torch.distributed as dist

@@ -60,8 +60,6 @@ __device__ __forceinline__ void butterflies(float (&v)[32]) {
     }
 }
 
-__device__ __forceinline__ int swz(int slot) { return slot ^ ((slot >> 3) & 7); }
-
 // Round (ties to even), clamp and pack 32 values held by one thread; returns words through `out`.
 template <bool INT8_OUT>
 __device__ __forceinline__ void quantize_pack(const float (&v)[32], float inv, int bits, uint32_t* out) {

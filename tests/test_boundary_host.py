@@ -123,3 +123,18 @@ def test_weight_prepare_errors(hq):
     with pytest.raises(hq.HqError) as e:
         hq.hq_weight_prepare(w, 5, 16, hq.HQ_W_PLAIN, hq.HQ_CODES_INT8)
     assert e.value.status == 1
+
+
+def test_unet_layer_list_matches_the_workload_description():
+    """Base 256, multipliers (1,2,3,4), 2 residual blocks per level, attention at 32/16/8, batch 64 on a 64x64 latent:
+    121 quantized layers of 47 distinct shapes, 16.0 TOP per forward counted with one weight limb."""
+    from paper_2512_05746_b200 import unet
+    layers = unet.quantized_layers()
+    assert len(layers) == 121 and len(unet.distinct_shapes(layers)) == 47
+    assert abs(2 * sum(L["macs"] for L in layers) / 1e12 - 16.04) < 0.01
+    for L in layers:
+        cin = L["C"] if L["kind"] == "conv" else L["K"]
+        assert cin % L["had_block"] == 0 and L["had_block"] == 256
+    assert sum(1 for L in layers if L["kind"] == "conv" and L["stride"] == 2) == 3
+    assert sum(1 for L in layers if L["kind"] == "conv" and L["R"] == 1) == 15
+    assert max(L["C"] for L in layers if L["kind"] == "conv") == 2048       # skip concatenation at the deepest level
