@@ -340,6 +340,79 @@ def main_unet(args):
                           clocks=clocks, gpu_launches=2 * len(layers) * steps)))
 
 
+def main_sweep(args):
+    """Shape sweep of transform+quantize followed by the integer GEMM: M x K x N grid, Hadamard block = K, for
+    W4A4 with the folded two-limb weights (nibble codes), W4A4 with plain one-limb weights (nibble codes) and W8A8
+    (int8 codes, plain weights).  W4A3 runs the same kernels as W4A4 (only the quantizer range differs).  One JSON
+    line with one record per point: int TOPS of the GEMM, GB/s of the quantize stage, and the roofline fraction of
+    the GEMM (slower of tensor peak and algorithmic bytes over the measured copy bandwidth)."""
+    import torch
+    from paper_2512_05746_b200 import binding as hq
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    pk = peaks()
+    int8_peak = 2.0 * pk["bf16_sustained"]
+    Ms, Ks, Ns = (4096, 16384, 65536), (256, 512, 1024, 2048, 4096), (512, 1280, 4096)
+    if args.rows != M_TOKENS:
+        Ms = (int(args.rows),)
+    variants = (("W4A4 folded", 4, 4, hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE),
+                ("W4A4 plain", 4, 4, hq.HQ_W_PLAIN, hq.HQ_CODES_NIBBLE),
+                ("W8A8 plain", 8, 8, hq.HQ_W_PLAIN, hq.HQ_CODES_INT8))
+    status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    reps = max(3, min(args.steps, 10))
+    points = []
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    for K in Ks:
+        for N in Ns:
+            w = inputs.weights((N, K), seed=K + N)
+            pws = {v[0]: hq.hq_weight_prepare(w, v[2], K, v[3], v[4]).to_device(dev) for v in variants}
+            b = torch.from_numpy(inputs.bias(N, seed=N)).to(dev)
+            for M in Ms:
+                x = torch.randn((M, K), generator=gen, device=dev, dtype=torch.float32)
+                x[:, torch.randperm(K, generator=gen, device=dev)[: max(1, round(0.01 * K))]] *= 20.0
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                for name, a_bits, w_bits, mode, cont in variants:
+                    pw = pws[name]
+                    pitch = K // 2 if cont == hq.HQ_CODES_NIBBLE else K
+                    codes = torch.empty((M, pitch), dtype=torch.uint8, device=dev)
+                    sc = torch.empty((M,), dtype=torch.float32, device=dev)
+                    q_ms = timed(lambda: hq.hq_hadamard_quant(x, K, a_bits, codes, cont, scales=sc))
+                    g_ms = timed(lambda: hq.hq_qgemm(codes, cont, a_bits, K, pw, scale_a=sc, bias=b, alpha=pw.alpha, y=y,
+                                                     dev_status=status))
+                    limbs = pw.desc.limbs
+                    ops = 2.0 * M * N * K * limbs
+                    gbytes = M * pitch + N * K * limbs + M * N * 2.0 + 4.0 * M + 8.0 * N
+                    t_tensor, t_hbm = ops / (int8_peak * 1e12), gbytes / (pk["hbm_gbs"] * 1e9)
+                    qbytes = M * K * 4.0 + M * pitch + 4.0 * M
+                    points.append(dict(M=M, K=K, N=N, variant=name, limbs=limbs, quant_us=q_ms * 1e3, gemm_us=g_ms * 1e3,
+                                       gemm_tops=ops / g_ms / 1e9, quant_gbs=qbytes / q_ms / 1e6,
+                                       bound="tensor" if t_tensor >= t_hbm else "hbm",
+                                       roofline_frac=max(t_tensor, t_hbm) / (g_ms * 1e-3),
+                                       quant_frac=qbytes / q_ms / 1e6 / pk["hbm_gbs"]))
+                del x, y
+    hq.hq_check_status(status)
+    best = max(points, key=lambda d: d["gemm_tops"])
+    print(json.dumps(dict(metric="shape sweep: int TOPS of the GEMM and GB/s of transform+quantize per point", value=best["gemm_tops"],
+                          unit="TOPS (best point)", n_gpus=1, steps=reps, warmup=3, higher_is_better=True, dtype="int8",
+                          data="synthetic", vs_baseline=None,
+                          config=dict(workload="configs[4] shape sweep", int8_peak_tops=int8_peak, hbm_gbs=pk["hbm_gbs"],
+                                      peak_source=pk["source"]), points=points)))
+
+
 def main():
     global M_TOKENS, WORKLOAD
     ap = argparse.ArgumentParser()
@@ -348,8 +421,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "unet"],
-                    help="step: the benchmark step (default); unet: the 121 quantized layers of the UNet-shaped workload")
+    ap.add_argument("--workload", default="step", choices=["step", "unet", "sweep"],
+                    help="step: the benchmark step (default); unet: the 121 quantized layers of the UNet-shaped workload; "
+                         "sweep: the M x K x N shape sweep")
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     args = ap.parse_args()
@@ -360,6 +434,8 @@ def main():
         return main_reference(args)
     if args.workload == "unet":
         return main_unet(args)
+    if args.workload == "sweep":
+        return main_sweep(args)
 
     import torch
     import torch.distributed as dist
