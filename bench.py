@@ -35,6 +35,12 @@ CONV = dict(Nb=32, H=32, W=32, C=256, Cout=256, R=3, S=3, stride=1, pad=1, had_b
 WORKLOAD = ("configs[2] transformer-block linears (M=32768; QKV, out-proj, FF1, FF2) + configs[1] 3x3 conv at "
             "batch 32 (M=32768, K=2304, N=256); W4A4, folded 2-limb weights, nibble codes, bf16 out")
 A_BITS, W_BITS = 4, 4
+# dram__bytes_read.sum + dram__bytes_write.sum per launch at the full size of the default step, from the one-pass ncu
+# capture of this command (a summary is kept under profiles/; taken with these kernel versions: set an entry to
+# None when its kernel changes).  Outputs partly stay in L2 past the end of a launch, so these are below the
+# algorithmic bytes.
+NCU_DRAM_BYTES = {"gemm": {"qkv": 54.2e6, "ff1": 88.8e6, "ff2": 36.0e6, "conv3x3": 5.4e6, "out_proj": None},
+                  "quant": {"qkv": 67.5e6, "out_proj": 67.5e6, "ff1": 67.5e6, "ff2": 275.1e6, "conv3x3": None}}
 
 
 def layer_list():
@@ -529,13 +535,17 @@ def main():
         ach = L["ops"] / (gemm_ms * 1e-3) / 1e12
         roofline = dict(bound="tensor", kernel=f"qgemm_kernel<nibble> ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
                                                 f"limbs={L['limbs']})",
-                        achieved=ach, peak=int8_peak, unit="TOPS", frac=ach / int8_peak, traffic=None,
+                        achieved=ach, peak=int8_peak, unit="TOPS", frac=ach / int8_peak,
+                        traffic=NCU_DRAM_BYTES["gemm"].get(L["name"]) if M_TOKENS == 32768 else None,
+                        algorithmic_bytes=L["gemm_bytes"],
                         peak_source=f"2 x bf16 sustained ({pk['source']})", launch_ms=gemm_ms)
         qd = max(per.values(), key=lambda d: d["quant_ms"])
         q_ms = qd["quant_ms"] / qd["n"]
         q_gbs = qd["L"]["quant_bytes"] / (q_ms * 1e-3) / 1e9
         roofline_quant = dict(bound="hbm", kernel=f"fwht_quant_fast ({qd['L']['name']}: {qd['L']['rows']}x{qd['L']['cols']})",
-                              achieved=q_gbs, peak=pk["hbm_gbs"], unit="GB/s", frac=q_gbs / pk["hbm_gbs"], traffic=None,
+                              achieved=q_gbs, peak=pk["hbm_gbs"], unit="GB/s", frac=q_gbs / pk["hbm_gbs"],
+                              traffic=NCU_DRAM_BYTES["quant"].get(qd["L"]["name"]) if M_TOKENS == 32768 else None,
+                              algorithmic_bytes=qd["L"]["quant_bytes"],
                               peak_source=f"copy bandwidth ({pk['source']})", launch_ms=q_ms)
         per_layer = {k: dict(quant_ms=d["quant_ms"] / d["n"], gemm_ms=d["gemm_ms"] / d["n"],
                              gemm_tops=d["L"]["ops"] / (d["gemm_ms"] / d["n"] * 1e-3) / 1e12,
