@@ -333,6 +333,26 @@ def main_unet(args):
     ms = e0.elapsed_time(e1) / steps
     clocks = sampler.stop()
     hq.hq_check_status(status)
+    # one more pass with an event after every layer: time and TOPS per distinct shape
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(layers) + 1)]
+    evs[0].record()
+    for i, L in enumerate(layers):
+        r = L["res"]
+        if L["kind"] == "conv":
+            hq.hq_qconv(r["x"], r["pw"], L["R"], L["R"], L["stride"], L["pad"], r["bias"], A_BITS, r["y"], r["ws"],
+                        static_scale=r["static"], dev_status=status)
+        else:
+            hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    per_shape = {}
+    for i, L in enumerate(layers):
+        d = per_shape.setdefault(str(key(L)), dict(count=0, ms=0.0, macs=L["macs"], limbs=L["res"]["pw"].desc.limbs))
+        d["count"] += 1
+        d["ms"] += evs[i].elapsed_time(evs[i + 1])
+    for d in per_shape.values():
+        d["ms_each"] = d["ms"] / d["count"]
+        d["tops"] = 2.0 * d["macs"] * d["limbs"] / (d["ms_each"] * 1e-3) / 1e12
     macs = sum(L["macs"] for L in layers)
     ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
     print(json.dumps(dict(metric="forwards/s of the 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent)",
@@ -343,7 +363,7 @@ def main_unet(args):
                                       layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
                                       l2="activations of the large layers exceed L2"),
-                          clocks=clocks, gpu_launches=2 * len(layers) * steps)))
+                          clocks=clocks, gpu_launches=2 * len(layers) * steps, per_shape=per_shape)))
 
 
 def main_sweep(args):
