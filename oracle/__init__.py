@@ -55,6 +55,10 @@ def lib():
             L.hqo_dequant.argtypes = [p, i64, i64, p, C.c_int, p, p, C.c_double, p]
             L.hqo_conv2d_dequant_perpixel.argtypes = [p, p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int,
                                                       C.c_int, C.c_int, p, p, C.c_double, p]
+            L.hqo_transform_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
+            L.hqo_codes_inverse_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
+            L.hqo_conv2d_int_z.argtypes = [p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int, C.c_int, C.c_int, p]
+            L.hqo_conv2d_int_z.restype = i64
             _lib = L
     return _lib
 
@@ -235,6 +239,38 @@ def conv2d_dequant_perpixel(q, s_a, B, stride: int, pad: int, s_w, bias, alpha: 
     return y
 
 
+def transform_width(x, had_block: int) -> np.ndarray:
+    """u = X~ * BlockDiag(H_k) along the WIDTH axis of an NHWC tensor (orthonormal H_k) -- the product before Eq. 13."""
+    x = _c(x, np.float64)
+    Nb, H, W, Cc = x.shape
+    u = np.empty_like(x)
+    _chk(lib().hqo_transform_width(_ptr(x), Nb, H, W, Cc, had_block, _ptr(u)), "transform_width")
+    return u
+
+
+def codes_inverse_width(q, had_block: int) -> np.ndarray:
+    """z = q * H_raw along the width axis (exact int32) -- the factor "(X H_c)_int * H_c" of Eq. 14 without 2^(-k/2)."""
+    q = _c(q, np.int8)
+    Nb, H, W, Cc = q.shape
+    z = np.empty(q.shape, np.int32)
+    _chk(lib().hqo_codes_inverse_width(_ptr(q), Nb, H, W, Cc, had_block, _ptr(z)), "codes_inverse_width")
+    return z
+
+
+def conv2d_int_z(z, B, stride: int, pad: int) -> np.ndarray:
+    """Direct integer convolution of int32 NHWC activations with B [Cout][R][S][C] -> int64 NHWC (Eq. 14)."""
+    z = _c(z, np.int32)
+    B = _c(B, np.int32)
+    Nb, H, W, Cc = z.shape
+    Cout, R, S, _ = B.shape
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    acc = np.empty((Nb, Ho, Wo, Cout), np.int64)
+    bad = lib().hqo_conv2d_int_z(_ptr(z), _ptr(B), Nb, H, W, Cc, Cout, R, S, stride, pad, _ptr(acc))
+    if bad:
+        raise OverflowError(f"{bad} accumulators exceed int32")
+    return acc
+
+
 # ----------------------------------------------------------------------------- chained layers
 
 def alpha_for(weight_mode: str, had_block: int) -> float:
@@ -283,3 +319,18 @@ def qconv(x, w, bias, *, a_bits: int, w_bits: int, had_block: int, stride: int, 
     else:
         y = dequant(acc, s_a, s_w, bias, alpha)
     return dict(u=u, q=q, s_a=s_a, v=v, B=B, s_w=s_w, acc=acc, alpha=alpha, y=y)
+
+
+def qconv_width(x, w, bias, *, a_bits: int, w_bits: int, had_block_w: int, stride: int, pad: int,
+                static_scale: float) -> dict:
+    """Quantized convolution exactly as Eq. 13-14 state it: the transform runs along the WIDTH axis, the weights are
+    quantized untransformed, and the integer core is Conv((X~ H_c)_int * H_c, W_int) with one activation scale:
+    y = 2^(-k/2) * S * S_w[o] * Conv(q * H_raw, W_int) + bias.   x NHWC, w [Cout][R][S][C]."""
+    u = transform_width(x, had_block_w)
+    q, s_a, v = quantize(u, a_bits, static_scale, want_v=True)      # elementwise with a static scale
+    z = codes_inverse_width(q, had_block_w)
+    w_int, s_w = weight_quantize(w, w_bits)
+    acc = conv2d_int_z(z, w_int, stride, pad)
+    alpha = float(2.0 ** (-0.5 * np.log2(had_block_w))) if had_block_w > 1 else 1.0
+    y = dequant(acc, s_a, s_w, bias, alpha)
+    return dict(u=u, q=q, s_a=s_a, v=v, z=z, B=w_int, s_w=s_w, acc=acc, alpha=alpha, y=y)

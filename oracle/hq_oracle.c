@@ -303,3 +303,85 @@ int hqo_conv2d_dequant_perpixel(const int8_t* q, const float* s_a, const int32_t
     }
     return 0;
 }
+
+/* ---- Convolution with the transform on the WIDTH axis, as Eq. 13-14 state it ------------------------------
+ * The paper reshapes X_c [B][Cin][h][w] to (B*Cin*h) x w and multiplies by the block-diagonal H_c (w x w) from
+ * the right, i.e. every image row of every channel is transformed along w.  Here tensors are NHWC, so the w
+ * axis has stride C; the arithmetic is the same.
+ *
+ * u[n][h][b*nb + j][c] = 2^(-k/2) * sum_i x[n][h][b*nb + i][c] * H_raw[i][j]      (nb = 2^k = had_block) */
+int hqo_transform_width(const double* x, i64 Nb, i64 H, i64 W, i64 C, int had_block, double* u) {
+    if (had_block <= 1) { memcpy(u, x, sizeof(double) * (size_t)(Nb * H * W * C)); return 0; }
+    const int n = had_block;
+    if (!is_pow2(n) || W % n != 0) return -1;
+    int8_t* Hm = (int8_t*)malloc((size_t)n * n);
+    if (!Hm) return -2;
+    hqo_hadamard_raw(n, Hm);
+    const double norm = pow(2.0, -0.5 * (double)ilog2(n));
+#pragma omp parallel for schedule(static)
+    for (i64 nh = 0; nh < Nb * H; ++nh) {
+        for (i64 b = 0; b < W / n; ++b) {
+            for (i64 c = 0; c < C; ++c) {
+                for (int j = 0; j < n; ++j) {
+                    double t = 0.0;
+                    for (int i = 0; i < n; ++i) t += x[(nh * W + b * n + i) * C + c] * (double)Hm[(i64)i * n + j];
+                    u[(nh * W + b * n + j) * C + c] = t * norm;
+                }
+            }
+        }
+    }
+    free(Hm);
+    return 0;
+}
+
+/* The integer factor "(X H_c)_int * H_c" of Eq. 14 with the raw +-1 matrix (its 2^(-k/2) goes to the scale):
+ * z[n][h][b*nb + j][c] = sum_i q[n][h][b*nb + i][c] * H_raw[i][j], exact integers, |z| <= nb * max|q|. */
+int hqo_codes_inverse_width(const int8_t* q, i64 Nb, i64 H, i64 W, i64 C, int had_block, int32_t* z) {
+    const int n = had_block > 1 ? had_block : 1;
+    if (!is_pow2(n) || W % n != 0) return -1;
+    int8_t* Hm = (int8_t*)malloc((size_t)n * n);
+    if (!Hm) return -2;
+    hqo_hadamard_raw(n, Hm);
+#pragma omp parallel for schedule(static)
+    for (i64 nh = 0; nh < Nb * H; ++nh) {
+        for (i64 b = 0; b < W / n; ++b) {
+            for (i64 c = 0; c < C; ++c) {
+                for (int j = 0; j < n; ++j) {
+                    i64 t = 0;
+                    for (int i = 0; i < n; ++i) t += (i64)q[(nh * W + b * n + i) * C + c] * (i64)Hm[(i64)i * n + j];
+                    z[(nh * W + b * n + j) * C + c] = (int32_t)t;
+                }
+            }
+        }
+    }
+    free(Hm);
+    return 0;
+}
+
+/* The integer convolution of Eq. 14 on 32-bit integer activations z (NHWC) and integer weights B [Cout][R][S][C]:
+ * same sum as hqo_conv2d_int.  Returns the number of accumulators that do not fit int32. */
+i64 hqo_conv2d_int_z(const int32_t* z, const int32_t* B, i64 Nb, i64 H, i64 W, i64 C, i64 Cout,
+                     int R, int S, int stride, int pad, i64* acc) {
+    const i64 Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
+    i64 bad = 0;
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+    for (i64 nho = 0; nho < Nb * Ho; ++nho) {
+        const i64 n = nho / Ho, ho = nho % Ho;
+        for (i64 wo = 0; wo < Wo; ++wo) {
+            for (i64 co = 0; co < Cout; ++co) {
+                i64 t = 0;
+                for (int r = 0; r < R; ++r) {
+                    for (int s = 0; s < S; ++s) {
+                        const i64 hi = ho * stride + r - pad, wi = wo * stride + s - pad;
+                        if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;
+                        for (i64 ci = 0; ci < C; ++ci)
+                            t += (i64)z[((n * H + hi) * W + wi) * C + ci] * (i64)B[((co * R + r) * S + s) * C + ci];
+                    }
+                }
+                acc[((n * Ho + ho) * Wo + wo) * Cout + co] = t;
+                if (t > 2147483647LL || t < -2147483648LL) ++bad;
+            }
+        }
+    }
+    return bad;
+}

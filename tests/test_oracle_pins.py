@@ -392,3 +392,79 @@ def test_qconv_layer_consistency(oracle):
     assert cs["q"].min() >= -4 and cs["q"].max() <= 3
     ref = oracle.dequant(cs["acc"], np.array([0.4], np.float32), cs["s_w"], b, cs["alpha"])
     assert np.array_equal(cs["y"], ref)
+
+
+# ------------------------------------------------------------------ width-axis convolution (Eq. 13-14 as stated)
+
+@pytest.mark.parametrize("W,n", [(8, 8), (16, 4), (32, 16), (12, 4)])
+def test_width_transform_is_the_row_transform_on_the_moved_axis(oracle, W, n):
+    """Transforming along w of NHWC must equal the (already pinned) last-axis transform of the tensor with w moved
+    last -- the reshape to (B*Cin*h) x w of the paper.  A wrong stride or a transposed H fails here."""
+    x = inputs.activations((2, 3, W, 5), outlier_count=1, outlier_scale=20.0, seed=W + n).astype(np.float64)
+    got = oracle.transform_width(x, n)
+    want = np.moveaxis(oracle.transform(np.moveaxis(x, 2, 3), n), 3, 2)
+    assert np.allclose(got, want, rtol=0, atol=1e-12)
+    assert np.allclose(oracle.transform_width(got, n), x, rtol=0, atol=1e-12)      # H_c H_c = I
+    with pytest.raises(ValueError):
+        oracle.transform_width(x, 2 * W)                                            # block does not divide w
+
+
+@pytest.mark.parametrize("W,n", [(8, 8), (16, 4), (32, 16)])
+def test_codes_inverse_width_closed_form_and_involution(oracle, W, n):
+    q = inputs.codes((2, 3, W, 4), 4, seed=W)
+    z = oracle.codes_inverse_width(q, n)
+    Hc = closed_form_H(n)
+    want = np.einsum("nhbic,ij->nhbjc", q.astype(np.int64).reshape(2, 3, W // n, n, 4), Hc).reshape(2, 3, W, 4)
+    assert np.array_equal(z, want)
+    assert np.abs(z).max() <= n * 8
+    # H_raw H_raw = n I: applying the integer factor twice returns n times the codes
+    zz = np.einsum("nhbic,ij->nhbjc", z.astype(np.int64).reshape(2, 3, W // n, n, 4), Hc).reshape(2, 3, W, 4)
+    assert np.array_equal(zz, n * q.astype(np.int64))
+
+
+def test_conv2d_int_z_equals_conv2d_int_on_small_values(oracle):
+    q = inputs.codes((2, 6, 5, 8), 4, seed=1)
+    B = inputs.codes((4, 3, 3, 8), 4, seed=2).astype(np.int32)
+    for stride, pad in ((1, 1), (2, 1), (1, 0)):
+        assert np.array_equal(oracle.conv2d_int_z(q.astype(np.int32), B, stride, pad), oracle.conv2d_int(q, B, stride, pad))
+
+
+def test_width_conv_layer_is_conv_of_dequantized_activations(oracle):
+    """Eq. 13 then Eq. 14: the layer output equals an ordinary float convolution of x_hat = S (XH)_int H_c with
+    W_hat = S_w W_int (im2col in numpy), and x_hat is within S/2 * sqrt(n) ... of x where nothing clamps."""
+    x = inputs.activations((2, 6, 16, 8), outlier_count=1, outlier_scale=10.0, seed=3).astype(np.float64)
+    w = inputs.weights((5, 3, 3, 8), seed=4)
+    b = inputs.bias(5, seed=5)
+    n, S = 8, 0.9
+    out = oracle.qconv_width(x, w, b, a_bits=4, w_bits=4, had_block_w=n, stride=1, pad=1, static_scale=S)
+    x_hat = np.float32(S) * oracle.transform_width(out["q"].astype(np.float64), n)      # S * q * H_c (orthonormal)
+    assert np.allclose(x_hat, np.float64(np.float32(S)) * 2.0 ** (-0.5 * np.log2(n)) * out["z"], rtol=0, atol=1e-12)
+    w_hat = out["s_w"].astype(np.float64)[:, None, None, None] * out["B"]
+    xp = np.pad(x_hat, ((0, 0), (1, 1), (1, 1), (0, 0)))
+    y = np.zeros((2, 6, 16, 5))
+    for r in range(3):
+        for s in range(3):
+            y += np.einsum("nhwc,oc->nhwo", xp[:, r:r + 6, s:s + 16, :], w_hat[:, r, s, :])
+    assert np.allclose(out["y"], y + b, rtol=1e-12, atol=1e-12)
+    # inside the clamp range the transformed values are within S/2 of their codes (Eq. 3), hence by Parseval the
+    # recovered activations are within S/2 * sqrt(n) of the originals per block
+    inside = np.abs(out["v"]) <= 7
+    assert np.all(np.abs(out["u"] - np.float32(S) * out["q"])[inside] <= 0.5 * np.float32(S) + 1e-12)
+
+
+def test_width_conv_recovers_plain_conv_when_quantization_is_fine(oracle):
+    """With 8-bit codes and a scale that nothing clamps at, the layer approaches Conv(x, W_hat): the error shrinks
+    with the scale (direction check of H_c H_c^T = I in Eq. 14)."""
+    x = inputs.activations((1, 5, 8, 4), seed=6).astype(np.float64)
+    w = inputs.weights((3, 3, 3, 4), seed=7)
+    errs = []
+    for S in (0.2, 0.05):
+        out = oracle.qconv_width(x, w, None, a_bits=8, w_bits=8, had_block_w=8, stride=1, pad=1, static_scale=S)
+        w_hat = out["s_w"].astype(np.float64)[:, None, None, None] * out["B"]
+        xp = np.pad(x, ((0, 0), (1, 1), (1, 1), (0, 0)))
+        y = np.zeros((1, 5, 8, 3))
+        for r in range(3):
+            for s in range(3):
+                y += np.einsum("nhwc,oc->nhwo", xp[:, r:r + 5, s:s + 8, :], w_hat[:, r, s, :])
+        errs.append(np.abs(out["y"] - y).max())
+    assert errs[1] < errs[0] and errs[1] < 0.02
