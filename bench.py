@@ -516,6 +516,39 @@ def main():
         d["gemm_ms"] += b.elapsed_time(c)
         d["n"] += 1
 
+    # ---- the same convolution with the width-axis transform (the paper's literal form; one weight limb) ----------
+    width = None
+    if rank == 0:
+        Lc = [L for L in layers if L["kind"] == "conv"][0]
+        c = CONV
+        pw_w = hq.hq_weight_prepare(inputs.config_conv_small(seed=rank, batch=1)["w"], W_BITS, 1, hq.HQ_W_PLAIN,
+                                    hq.HQ_CODES_INT8).to_device(device)
+        ws_w = torch.empty((hq.hq_workspace_size(Lc["rows"], Lc["cols"], hq.HQ_CODES_INT8),), dtype=torch.uint8, device=device)
+        zbuf = torch.empty((Lc["rows"], Lc["cols"]), dtype=torch.int8, device=device)
+
+        def width_layer():
+            hq.hq_qconv_width(Lc["x"], pw_w, c["R"], c["S"], c["stride"], c["pad"], Lc["bias"], A_BITS, 16,
+                              Lc["static_scale"], Lc["y"], ws_w, dev_status=status)
+
+        def width_quant():
+            hq.hq_hadamard_quant_width(Lc["x"], 16, A_BITS, Lc["static_scale"], zbuf.view(Lc["x"].shape))
+
+        res = []
+        for fn in (width_layer, width_quant):
+            for _ in range(3):
+                fn()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            for _ in range(args.steps):
+                fn()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            res.append(g0.elapsed_time(g1) / args.steps)
+        width = dict(layer_ms=res[0], quant_ms=res[1], tops_1limb=Lc["ops_1limb"] / (res[0] * 1e-3) / 1e12,
+                     quant_gbs=Lc["rows"] * Lc["cols"] * 5.0 / (res[1] * 1e-3) / 1e9,
+                     note="3x3 conv of the step with the transform along the width axis (16-point blocks), "
+                          "untransformed one-limb weights, int8 activations")
+
     # ---- end to end: pinned host input -> device -> fused call -> host output -----------------------
     e2e_steps = max(2, min(args.steps, 5))
     h2d = sum(L["x_host"].numel() * L["x_host"].element_size() for L in layers)
@@ -580,7 +613,8 @@ def main():
                     clocks=clocks, gpu_launches=2 * len(layers) * args.steps,
                     e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              steps=e2e_steps, ms_per_step=e2e_ms / e2e_steps),
-                    roofline=roofline, roofline_fwht_quant=roofline_quant, per_layer=per_layer)
+                    roofline=roofline, roofline_fwht_quant=roofline_quant, per_layer=per_layer,
+                    width_axis_conv=width)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline()
         print(json.dumps(line))

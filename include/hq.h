@@ -150,6 +150,30 @@ hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W
                    const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
                    int32_t* dev_status, void* stream);
 
+/* ---- Eq. 13 + Eq. 14 with the transform on the WIDTH axis, as the paper states the convolution ---------------------
+ * The paper reshapes X_c [B][Cin][h][w] to (B*Cin*h) x w and multiplies by the block-diagonal H_c (w x w): every
+ * image row of every channel is transformed along w.  The weights are quantized untransformed and the integer core
+ * is Conv((X~ H_c)_int * H_c, W_int) with ONE activation scale in front (a per-row scale would not factor out of the
+ * sum over channels and taps).
+ *
+ * hq_hadamard_quant_width: x device NHWC [Nb][H][W][C] (densely packed, C % 4 == 0) ->
+ *   z = clamp(rint(x H_c / S)) * H_raw   as int8 NHWC (device), the integer activations of the convolution, and
+ *   scale_out[0] = S * 2^(-k/2) (device, may be NULL), the scale that goes in front of it.
+ *   had_block_w = 2^k divides W (0/1: no transform); static_scale = S (device, 1 float); bits in {3,4,8}.
+ *   The integer factor must fit a signed byte: had_block_w * 2^(bits-1) <= 128 (16 positions at 4 bits, 32 at 3 bits),
+ *   otherwise HQ_ERR_OVERFLOW_RISK.
+ * hq_qconv_width: the whole layer.  desc / w_dev: PLAIN one-limb weights prepared for the INT8 container
+ *   (had_block of the descriptor is ignored); workspace as for hq_qconv with the INT8 container;
+ *   y = 2^(-k/2) * S * S_w[o] * Conv(z, W_int) + bias[o]. */
+hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                  int had_block_w, int bits, const float* static_scale, void* z_codes,
+                                  float* scale_out, void* stream);
+hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                         const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                         const float* scale_w, const float* bias, int a_bits, int had_block_w,
+                         const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                         int32_t* dev_status, void* stream);
+
 /* ---- Fused linear layer that allocates nothing and takes no workspace (the paper has no counterpart: this is a
  * packaging of hq_qlinear for a particular kind of caller, not another operation). ---------------------------------
  * Who it is for: code that must not, or cannot, obtain device memory at the moment it runs a layer -- an inference

@@ -24,7 +24,7 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
-           "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc"]
+           "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -67,11 +67,15 @@ def _load():
                            p, p, i32, p, C.c_size_t, p, p]
     L.hq_qlinear_noalloc.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i32, i64,
                                      p, p]
+    L.hq_hadamard_quant_width.argtypes = [p, i32, i64, i64, i64, i64, i32, i32, p, p, p, p]
+    L.hq_qconv_width.argtypes = [p, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32, i32,
+                                 p, p, i32, p, C.c_size_t, p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
-                 "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc"):
+                 "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
+                 "hq_hadamard_quant_width", "hq_qconv_width"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -234,6 +238,23 @@ def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias,
                         pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y),
                         _dtype_code(y), _dptr(workspace), workspace.numel() * workspace.element_size(),
                         _dptr(dev_status), _stream(stream)), "hq_qconv")
+
+
+def hq_hadamard_quant_width(x, had_block_w: int, bits: int, static_scale, z, scale_out=None, stream=None) -> None:
+    """x NHWC (fp32/bf16, dense) -> z int8 NHWC = clamp(rint(x H_c / S)) * H_raw along the width axis (Eq. 13-14)."""
+    Nb, H, W, Cin = x.shape
+    _check(lib.hq_hadamard_quant_width(_dptr(x), _dtype_code(x), Nb, H, W, Cin, had_block_w, bits, _dptr(static_scale),
+                                       _dptr(z), _dptr(scale_out), _stream(stream)), "hq_hadamard_quant_width")
+
+
+def hq_qconv_width(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias, a_bits: int, had_block_w: int,
+                   static_scale, y, workspace, dev_status=None, stream=None) -> None:
+    """The convolution layer with the width-axis transform (Eq. 13-14); pw: PLAIN weights for the INT8 container."""
+    Nb, H, W, Cin = x.shape
+    _check(lib.hq_qconv_width(_dptr(x), _dtype_code(x), Nb, H, W, Cin, C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride,
+                              pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, had_block_w, _dptr(static_scale), _dptr(y),
+                              _dtype_code(y), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                              _dptr(dev_status), _stream(stream)), "hq_qconv_width")
 
 
 def hq_mma_i8_probe(ctas: int, iters: int, dev_status=None, stream=None) -> None:

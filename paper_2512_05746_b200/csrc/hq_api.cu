@@ -21,6 +21,10 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
                          const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias,
                          float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st);
 
+hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                      int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
+                                      cudaStream_t st);
+
 namespace {
 int64_t code_pitch(int64_t cols, hq_container cont) {
     const int64_t b = cont == HQ_CODES_NIBBLE ? cols / 2 : cols;
@@ -109,6 +113,34 @@ extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st);
+}
+
+// Convolution exactly as Eq. 13-14 state it: transform along the width axis, quantization with one static scale,
+// integer factor q * H_raw, integer convolution with untransformed (PLAIN, one-limb, INT8-container) weights.
+// The int8 activations z and the scale S * 2^(-k/2) live in `workspace` (hq_workspace_size(Nb*H*W, C, INT8)).
+extern "C" hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                    const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                                    const float* scale_w, const float* bias, int a_bits, int had_block_w,
+                                    const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                                    int32_t* dev_status, void* stream) {
+    using namespace hq;
+    if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (desc->mode != HQ_W_PLAIN || desc->limbs != 1 || desc->container != HQ_CODES_INT8) return HQ_ERR_SHAPE;
+    if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+    const int64_t rows = Nb * H * W;
+    size_t need = 0;
+    hq_status s = hq_workspace_size(rows, C, HQ_CODES_INT8, &need);
+    if (s != HQ_OK) return s;
+    if (ws_bytes < need) return HQ_ERR_WORKSPACE;
+    if (C % 16 != 0) return HQ_ERR_ALIGNMENT;              // densely packed pixels for the convolution's TMA boxes
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* z = static_cast<unsigned char*>(workspace);
+    float* scale = reinterpret_cast<float*>(z + scales_offset(rows, C, HQ_CODES_INT8));
+    s = launch_hadamard_quant_width(x, xdt, Nb, H, W, C, had_block_w, a_bits, static_scale, z, scale, st);
+    if (s != HQ_OK) return s;
+    // |z| <= 128: the accumulator bound is that of 8-bit codes; the 2^(-k/2) is already inside `scale`
+    return launch_qconv2d(z, HQ_CODES_INT8, 8, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale, 1, scale_w, bias, 1.0f,
+                          nullptr, y, ydt, dev_status, st);
 }
 
 namespace hq {

@@ -377,6 +377,99 @@ __global__ void __launch_bounds__(256) fwht_quant_generic(const QuantParams p, i
     }
 }
 
+// ---- width-axis variant (Eq. 13-14 as stated): transform along w, quantize, integer factor q * H_raw ---------
+// x is NHWC; a thread owns 4 consecutive channels of one block of NB positions along w (loads and stores of a warp
+// are contiguous over channels).  Per channel: NB-point transform in registers, static-scale quantization
+// (ties to even, clamp), then the +-1 transform again on the codes (exact small integers in fp32) and a byte store.
+struct WidthParams {
+    const void* x;
+    int64_t items;        // Nb * H * (W / NB) * (C / 4)
+    int64_t C;
+    int c4;               // C / 4
+    int wblocks;          // W / NB
+    int bits;
+    float norm;           // 2^(-k/2)
+    const float* static_scale;
+    int8_t* z;
+    float* scale_out;     // receives S * 2^(-k/2), the one activation scale of the integer convolution
+};
+
+template <int NB, typename InT>
+__global__ void __launch_bounds__(256) width_quant_kernel(const WidthParams p) {
+    const int64_t item = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const float S = __ldg(p.static_scale);
+    if (item == 0 && p.scale_out != nullptr) p.scale_out[0] = S * p.norm;
+    if (item >= p.items) return;
+    const int c4 = int(item % p.c4);
+    const int64_t rest = item / p.c4;
+    const int b = int(rest % p.wblocks);
+    const int64_t nh = rest / p.wblocks;
+    const int64_t base = ((nh * p.wblocks + b) * NB) * p.C + 4 * c4;      // element offset of (nh, w = b*NB, c)
+    const InT* src = reinterpret_cast<const InT*>(p.x) + base;
+
+    f32x2 v[NB][2];                                   // [position along w][channel pair]
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        const float4 f = load4(src + int64_t(i) * p.C);
+        v[i][0] = pk2(f.x, f.y);
+        v[i][1] = pk2(f.z, f.w);
+    }
+#pragma unroll
+    for (int h = 1; h < NB; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            if (!(i & h)) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const f32x2 a = v[i][c], bb = v[i | h][c];
+                    v[i][c] = add2(a, bb);
+                    v[i | h][c] = sub2(a, bb);
+                }
+            }
+        }
+    }
+    // codes as integer-valued floats: round by the magic add, clamp, take the magic off again
+    const float inv = p.norm / S;
+    const float lo = kMagic + float(-(1 << (p.bits - 1))), hi = kMagic + float((1 << (p.bits - 1)) - 1);
+    const f32x2 inv2 = pk2(inv, inv), mg2 = pk2(kMagic, kMagic);
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            float a, bb;
+            upk2(fma2(v[i][c], inv2, mg2), a, bb);
+            a = fminf(fmaxf(a, lo), hi) - kMagic;
+            bb = fminf(fmaxf(bb, lo), hi) - kMagic;
+            v[i][c] = pk2(a, bb);
+        }
+    }
+#pragma unroll
+    for (int h = 1; h < NB; h <<= 1) {
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            if (!(i & h)) {
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const f32x2 a = v[i][c], bb = v[i | h][c];
+                    v[i][c] = add2(a, bb);
+                    v[i | h][c] = sub2(a, bb);
+                }
+            }
+        }
+    }
+    int8_t* dst = p.z + base;
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        float a0, a1, a2, a3;
+        upk2(add2(v[i][0], mg2), a0, a1);
+        upk2(add2(v[i][1], mg2), a2, a3);
+        // the low byte of (magic + z) is z in two's complement
+        const uint32_t w01 = __byte_perm(__float_as_uint(a0), __float_as_uint(a1), 0x0040);
+        const uint32_t w23 = __byte_perm(__float_as_uint(a2), __float_as_uint(a3), 0x0040);
+        *reinterpret_cast<uint32_t*>(dst + int64_t(i) * p.C) = __byte_perm(w01, w23, 0x5410);
+    }
+}
+
 template <int KLOG, int E, typename InT>
 cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threads, size_t smem, cudaStream_t st) {
     const bool stat = p.static_scale != nullptr;
@@ -484,7 +577,52 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
+// Width-axis transform + quantization + integer factor of Eq. 13-14: x NHWC fp32/bf16 -> z int8 NHWC.
+hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                      int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
+                                      cudaStream_t st) {
+    if (x == nullptr || z == nullptr || static_scale == nullptr) return HQ_ERR_INVALID_ARG;
+    if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return HQ_ERR_INVALID_ARG;
+    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0) return HQ_ERR_SHAPE;
+    const int nb = had_block_w > 1 ? had_block_w : 1;
+    if (!is_pow2(nb) || W % nb != 0) return HQ_ERR_SHAPE;
+    // z = q * H_raw must fit a signed byte: nb * 2^(bits-1) <= 128 (16 positions at 4 bits, 32 at 3 bits)
+    if (int64_t(nb) << (bits - 1) > 128) return HQ_ERR_OVERFLOW_RISK;
+    if (C % 4 != 0) return HQ_ERR_UNSUPPORTED;
+    const int elt = xdt == HQ_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(x) % (4 * elt) != 0 || reinterpret_cast<uintptr_t>(z) % 4 != 0) return HQ_ERR_ALIGNMENT;
+
+    WidthParams p{};
+    p.x = x; p.C = C; p.c4 = int(C / 4); p.wblocks = int(W / nb); p.bits = bits;
+    p.items = Nb * H * (W / nb) * (C / 4);
+    p.norm = float(exp2(-0.5 * double(ilog2(nb))));
+    p.static_scale = static_scale; p.z = static_cast<int8_t*>(z); p.scale_out = scale_out;
+    const int threads = 256;
+    const int64_t grid64 = (p.items + threads - 1) / threads;
+    if (grid64 > 0x7FFFFFFF) return HQ_ERR_UNSUPPORTED;
+    const int grid = int(grid64);
+#define HQ_WIDTH_CASE(NBV)                                                                              \
+    case NBV:                                                                                           \
+        if (xdt == HQ_F32) width_quant_kernel<NBV, float><<<grid, threads, 0, st>>>(p);                 \
+        else width_quant_kernel<NBV, __nv_bfloat16><<<grid, threads, 0, st>>>(p);                       \
+        break;
+    switch (nb) {
+        HQ_WIDTH_CASE(1) HQ_WIDTH_CASE(2) HQ_WIDTH_CASE(4) HQ_WIDTH_CASE(8) HQ_WIDTH_CASE(16) HQ_WIDTH_CASE(32)
+        default: return HQ_ERR_UNSUPPORTED;
+    }
+#undef HQ_WIDTH_CASE
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
 }  // namespace hq
+
+extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                             int had_block_w, int bits, const float* static_scale, void* z_codes,
+                                             float* scale_out, void* stream) {
+    return hq::launch_hadamard_quant_width(x, xdt, Nb, H, W, C, had_block_w, bits, static_scale, z_codes, scale_out,
+                                           static_cast<cudaStream_t>(stream));
+}
 
 extern "C" hq_status hq_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx,
                                        int had_block, int bits, hq_scale_mode mode, const float* static_scale,

@@ -1,0 +1,110 @@
+"""GPU parity of the convolution with the width-axis transform (Eq. 13-14 as the paper states them) against the
+CPU oracle: the int8 activations z = clamp(rint(x H_c / S)) * H_raw, then the whole layer."""
+import numpy as np
+import pytest
+
+from paper_2512_05746_b200 import inputs
+from hq_testutil import CODE_MISMATCH_FRAC, CODE_TIE_REL, Y_BF16_RTOL, Y_F32_RTOL, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2512_05746_b200 import binding as hq
+    return torch, hq
+
+
+def codes_from_z(z, n, closed_H):
+    """z = q * H_raw  =>  q = z * H_raw / n (exact): recovers the device's codes from its int8 activations."""
+    Nb, H, W, C = z.shape
+    zz = np.einsum("nhbic,ij->nhbjc", z.astype(np.int64).reshape(Nb, H, W // n, n, C), closed_H).reshape(z.shape)
+    assert np.all(zz % n == 0)
+    return (zz // n).astype(np.int64)
+
+
+def closed_form_H(n):
+    i = np.arange(n)
+    pc = np.vectorize(lambda v: bin(v).count("1"))(i[:, None] & i[None, :])
+    return (1 - 2 * (pc & 1)).astype(np.int64)
+
+
+CASES = [
+    # Nb, H, W, C, had_block_w, bits, dtype
+    (2, 8, 32, 64, 16, 4, "f32"),
+    (3, 5, 48, 32, 16, 4, "f32"),       # three blocks along w
+    (2, 6, 32, 128, 32, 3, "f32"),      # 32-point blocks are allowed at 3 bits
+    (1, 7, 8, 20, 8, 4, "bf16"),        # C not a multiple of 16, bf16 input
+    (2, 4, 16, 64, 4, 8, "f32"),        # 8-bit codes: only 1-point ... 1*128: block must be 1
+    (2, 4, 16, 64, 1, 8, "f32"),
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,n,bits,dt", CASES)
+def test_width_quant_matches_oracle(env, oracle, Nb, H, W, C, n, bits, dt):
+    torch, hq = env
+    x = inputs.activations((Nb, H, W, C), outlier_count=max(1, C // 50), outlier_scale=20.0, seed=W + C + n)
+    xt = torch.from_numpy(x).cuda()
+    if dt == "bf16":
+        xt = xt.to(torch.bfloat16)
+        x = xt.float().cpu().numpy()
+    u = oracle.transform_width(x, n)
+    S = float(np.float32(np.abs(u).max() / oracle.qmax(bits) / 2.5))          # clamps the largest values
+    z = torch.full((Nb, H, W, C), 77, dtype=torch.int8, device="cuda")
+    so = torch.zeros((1,), dtype=torch.float32, device="cuda")
+    ss = torch.tensor([S], dtype=torch.float32, device="cuda")
+    if n * 2 ** (bits - 1) > 128:
+        with pytest.raises(hq.HqError) as e:
+            hq.hq_hadamard_quant_width(xt, n, bits, ss, z, so)
+        assert e.value.status == 6
+        return
+    hq.hq_hadamard_quant_width(xt, n, bits, ss, z, so)
+    torch.cuda.synchronize()
+    q_ref, _, v = oracle.quantize(u, bits, static_scale=S, want_v=True)
+    z_gpu = z.cpu().numpy()
+    q_gpu = codes_from_z(z_gpu, n, closed_form_H(n)) if n > 1 else z_gpu.astype(np.int64)
+    bad = q_gpu != q_ref
+    if bad.any():                                             # only rounding ties may differ, by one
+        assert np.abs(q_gpu - q_ref)[bad].max() == 1 and bad.mean() <= CODE_MISMATCH_FRAC
+        vc = np.clip(v, oracle.qmin(bits) - 0.25, oracle.qmax(bits) + 0.25)
+        full = max(float(np.abs(vc).max()), 1.0)
+        assert np.all(np.abs(vc - (np.floor(vc) + 0.5))[bad] <= CODE_TIE_REL * full * 8)
+    assert np.array_equal(z_gpu.astype(np.int64), oracle.codes_inverse_width(q_gpu.astype(np.int8), n).astype(np.int64))
+    assert q_gpu.min() == oracle.qmin(bits) and q_gpu.max() == oracle.qmax(bits)
+    assert np.isclose(float(so.cpu()[0]), np.float32(S) * 2.0 ** (-0.5 * np.log2(n)), rtol=1e-6)
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,R,stride,n,bits,odt", [
+    (8, 32, 32, 256, 256, 3, 1, 16, 4, "bf16"),      # the small conv configuration, transform along the width
+    (2, 16, 16, 128, 200, 3, 1, 16, 4, "f32"),
+    (2, 32, 32, 64, 64, 3, 2, 16, 3, "f32"),         # stride 2, W4A3
+    (2, 16, 16, 128, 128, 1, 1, 8, 4, "bf16"),       # 1x1
+])
+def test_qconv_width_layer_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, stride, n, bits, odt):
+    torch, hq = env
+    x = inputs.activations((Nb, H, W, C), outlier_count=max(1, C // 100), outlier_scale=20.0, seed=H + C)
+    w = inputs.weights((Cout, R, R, C), seed=Cout + R)
+    b = inputs.bias(Cout, seed=2)
+    pad = R // 2
+    S = float(np.float32(np.abs(oracle.transform_width(x, n)).max() / oracle.qmax(bits) / 2.0))
+    pw = hq.hq_weight_prepare(w, 4, 1, hq.HQ_W_PLAIN, hq.HQ_CODES_INT8).to_device()
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
+    y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16 if odt == "bf16" else torch.float32, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(Nb * H * W, C, hq.HQ_CODES_INT8),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qconv_width(torch.from_numpy(x).cuda(), pw, R, R, stride, pad, torch.from_numpy(b).cuda(), bits, n,
+                      torch.tensor([S], dtype=torch.float32, device="cuda"), y, ws, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    ref = oracle.qconv_width(x, w, b, a_bits=bits, w_bits=4, had_block_w=n, stride=stride, pad=pad, static_scale=S)
+    # the device's own integer activations (they may differ from the oracle's at rounding ties) -> oracle conv + rescale
+    z_gpu = ws[: Nb * H * W * C].view(torch.int8).cpu().numpy().reshape(Nb, H, W, C)
+    assert (z_gpu.astype(np.int64) != ref["z"]).mean() <= 16 * CODE_MISMATCH_FRAC
+    B = hq.decode_blob(pw).reshape(Cout, R, R, C)
+    assert np.array_equal(B, ref["B"]) and np.array_equal(pw.s_w, ref["s_w"])
+    y_own = oracle.dequant(oracle.conv2d_int_z(z_gpu.astype(np.int32), B, stride, pad), ref["s_a"], pw.s_w, b, ref["alpha"])
+    assert rel_err(y.float().cpu().numpy(), y_own) <= (Y_BF16_RTOL if odt == "bf16" else Y_F32_RTOL)
+    rms = np.sqrt(np.mean((y.float().cpu().numpy() - ref["y"]) ** 2)) / np.sqrt(np.mean(ref["y"] ** 2))
+    assert rms <= Y_BF16_RTOL
