@@ -255,16 +255,25 @@ def main_reference(args):
     print(json.dumps(line))
 
 
-def main_unet(args):
-    """All 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent), one after the other on one
-    stream, bf16 activations, W4A4 with folded two-limb weights.  3x3 convolutions use one static activation scale,
-    1x1 convolutions and linears per-row scales.  The bf16 glue between the layers is not part of this path."""
+def main_layer_list(args, which):
+    """All quantized layers of a network-shaped workload, one after the other on one stream, bf16 activations,
+    W4A4 with folded two-limb weights.  3x3 convolutions use one static activation scale, 1x1 convolutions and linears
+    per-row scales.  The bf16 glue between the layers is not part of this path.
+    unet: 121 layers of the UNet-shaped workload (batch 64, 64x64 latent); dit: 143 linears of a width-1152,
+    depth-28 diffusion transformer (batch 32, 256 tokens)."""
     import torch
     from paper_2512_05746_b200 import binding as hq
-    from paper_2512_05746_b200 import unet
+    from paper_2512_05746_b200 import dit, unet
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    layers = unet.quantized_layers()
+    if which == "unet":
+        layers = unet.quantized_layers()
+        label = "the 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent)"
+        wl = "configs[3] quantized layers only: 121 layers, 47 distinct shapes"
+    else:
+        layers = dit.quantized_layers()
+        label = "the 143 quantized linears of the DiT-XL/2-shaped workload (batch 32, 256 tokens, width 1152 = 9 x 128)"
+        wl = "DiT-XL/2-shaped quantized linears: 28 blocks x (adaLN, QKV, proj, FC1, FC2) + embedding MLP"
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
     cache = {}
@@ -355,11 +364,11 @@ def main_unet(args):
         d["tops"] = 2.0 * d["macs"] * d["limbs"] / (d["ms_each"] * 1e-3) / 1e12
     macs = sum(L["macs"] for L in layers)
     ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
-    print(json.dumps(dict(metric="forwards/s of the 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent)",
+    print(json.dumps(dict(metric="forwards/s of " + label,
                           value=1e3 / ms, unit="forwards/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=ms,
                           higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int8", data="synthetic",
-                          config=dict(workload="configs[3] quantized layers only: 121 layers, 47 distinct shapes, bf16 in/out, "
-                                               "W4A4 folded two-limb weights, nibble codes", layers=len(layers),
+                          config=dict(workload=wl + ", bf16 in/out, W4A4 folded two-limb weights, nibble codes",
+                                      layers=len(layers),
                                       layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
                                       l2="activations of the large layers exceed L2"),
@@ -447,8 +456,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "unet", "sweep"],
-                    help="step: the benchmark step (default); unet: the 121 quantized layers of the UNet-shaped workload; "
+    ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep"],
+                    help="step: the benchmark step (default); unet / dit: the quantized layers of the UNet- / DiT-shaped workload; "
                          "sweep: the M x K x N shape sweep")
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
@@ -458,8 +467,8 @@ def main():
         WORKLOAD = f"REDUCED to {M_TOKENS} rows per layer (profiling case, not a benchmark number): " + WORKLOAD
     if args.impl == "reference":
         return main_reference(args)
-    if args.workload == "unet":
-        return main_unet(args)
+    if args.workload in ("unet", "dit"):
+        return main_layer_list(args, args.workload)
     if args.workload == "sweep":
         return main_sweep(args)
 

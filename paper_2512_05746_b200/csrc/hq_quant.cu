@@ -166,7 +166,7 @@ __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, i
 //            KLOG = 12 needs one more stage than fits and takes it with a lane exchange.
 // Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
 template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC>
-__global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
+__global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     constexpr int N = 1 << KLOG;
     constexpr int LE = ilog2_c(E);
     constexpr int P = E / 2;                           // two-wide registers per thread
@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
     static_assert(R <= LE, "block too large for this thread shape");
     constexpr int J = PAIR ? E / 2 : E / 4;            // float4 slots a phase-B thread (pair) walks
     constexpr int S = ilog2_c(J);
-    static_assert(TB % J == 0 || TB == J, "exchange layout needs TB to be a multiple of J");
+    static_assert(TB % J == 0 || J % TB == 0, "exchange layout needs TB and J to divide one another");
     constexpr int GS = N / 4 + (N / 4) / J;            // padded float4 slots per Hadamard block
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4* xch = reinterpret_cast<float4*>(smem_raw);
@@ -210,9 +210,11 @@ __global__ void __launch_bounds__(256) fwht_quant_fast(const QuantParams p) {
 
     float4* grp = xch + (tid / TB) * GS;
     {
+        // slot f = tb + TB i sits at f + f / J; with TB and J dividing one another that is a per-thread base plus a
+        // compile-time offset
         ulonglong2* wr = reinterpret_cast<ulonglong2*>(grp + tb + (tb >> S));
 #pragma unroll
-        for (int i = 0; i < E / 4; ++i) wr[i * (TB + (TB >> S))] = make_ulonglong2(v[2 * i], v[2 * i + 1]);
+        for (int i = 0; i < E / 4; ++i) wr[TB * i + ((TB * i) >> S)] = make_ulonglong2(v[2 * i], v[2 * i + 1]);
     }
     if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
     if (!PAIR) {
@@ -492,6 +494,9 @@ template <typename InT>
 cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int grid, int threads, size_t smem,
                           cudaStream_t st) {
     switch (klog) {
+        case 5: return launch_fast<5, 32, InT>(p, int8_out, grid, threads, smem, st);
+        case 6: return launch_fast<6, 32, InT>(p, int8_out, grid, threads, smem, st);
+        case 7: return launch_fast<7, 32, InT>(p, int8_out, grid, threads, smem, st);
         case 8: return launch_fast<8, fast_e(8), InT>(p, int8_out, grid, threads, smem, st);
         case 9: return launch_fast<9, fast_e(9), InT>(p, int8_out, grid, threads, smem, st);
         case 10: return launch_fast<10, fast_e(10), InT>(p, int8_out, grid, threads, smem, st);
@@ -535,7 +540,7 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
 
     const int elt = xdt == HQ_F32 ? 4 : 2;
     const int E = fast_e(klog);
-    const bool fast_ok = klog >= 8 && klog <= 12 && cols / E <= 256 &&
+    const bool fast_ok = klog >= 5 && klog <= 12 && cols / E <= 256 &&
                          (reinterpret_cast<uintptr_t>(x) % (4 * elt) == 0) && (ldx % 4 == 0) &&
                          aligned16(codes) && (ld_codes % 16 == 0);
     if (fast_ok) {
@@ -549,6 +554,7 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
         p.threads_per_row = tr;
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
+        if (threads <= 320) {                               // otherwise the generic kernel below takes the row shape
         // exchange buffer: per Hadamard block n/4 float4 slots plus one slot of padding per J (J = E/2 or E/4)
         const int jslots = (klog - ilog2(E) >= ilog2(E) - 1) ? E / 2 : E / 4;
         const size_t smem = size_t(threads / (n / E)) * size_t(n / 4 + n / 4 / jslots) * 16 + size_t(rpc) * 4;
@@ -557,6 +563,7 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
                             ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
                             : dispatch_fast<__nv_bfloat16>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st);
         return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+        }
     }
     const size_t smem = size_t(cols) * 4;
     if (smem > 200 * 1024) return HQ_ERR_UNSUPPORTED;

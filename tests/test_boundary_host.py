@@ -138,3 +138,13 @@ def test_unet_layer_list_matches_the_workload_description():
     assert sum(1 for L in layers if L["kind"] == "conv" and L["stride"] == 2) == 3
     assert sum(1 for L in layers if L["kind"] == "conv" and L["R"] == 1) == 15
     assert max(L["C"] for L in layers if L["kind"] == "conv") == 2048       # skip concatenation at the deepest level
+
+
+def test_dit_layer_list():
+    """Width 1152 = 9 x 128, depth 28, MLP ratio 4, batch 32 x 256 tokens: 28 x 5 + 3 quantized linears."""
+    from paper_2512_05746_b200 import dit
+    layers = dit.quantized_layers()
+    assert len(layers) == 28 * 5 + 3
+    assert all(L["K"] % L["had_block"] == 0 and L["had_block"] == 128 for L in layers)
+    big = [L for L in layers if L["M"] == 32 * 256]
+    assert len(big) == 28 * 4 and {(L["K"], L["N"]) for L in big} == {(1152, 3456), (1152, 1152), (1152, 4608), (4608, 1152)}

@@ -79,6 +79,18 @@ def test_qlinear_full_size_sampled_rows(env, oracle, which):
     run_linear(torch, hq, oracle, cfg["x"], cfg["w"], cfg["bias"], 4, cfg["had_block"], "folded", 0, rows_checked=rows)
 
 
+@pytest.mark.parametrize("K,N", [(1152, 3456), (4608, 1152)])
+def test_qlinear_block_diagonal_128(env, oracle, K, N):
+    """Linears of a width-1152 transformer: 9 (or 36) Hadamard blocks of 128 channels per token, ragged row count."""
+    torch, hq = env
+    M = 700
+    x = inputs.activations((M, K), dist="student_t3", outlier_count=max(1, K // 200), outlier_scale=30.0, seed=K)
+    w = inputs.weights((N, K), seed=N)
+    b = inputs.bias(N, seed=3)
+    rows = np.sort(np.random.default_rng(2).choice(M, size=96, replace=False))
+    run_linear(torch, hq, oracle, x, w, b, 4, 128, "folded", 0, rows_checked=rows)
+
+
 @pytest.mark.parametrize("a_bits,static", [(4, False), (3, False), (4, True)])
 def test_qconv_small_configuration(env, oracle, a_bits, static):
     """NHWC [8,32,32,256] x [256,3,3,256], stride 1, pad 1, Hadamard over the input channels, per-pixel INT4 / INT3

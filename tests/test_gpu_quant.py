@@ -62,6 +62,11 @@ CASES = [
     (100, 24, 1, 4, 0),          # identity bypass
     (100, 96, 32, 3, 1),
     (5, 256, 256, 4, 0),
+    (300, 1152, 128, 4, 0),      # 9 blocks of 128 (a transformer of width 1152): 36 threads per row
+    (100, 4608, 128, 4, 1),      # 36 blocks of 128
+    (130, 1152, 64, 3, 0),
+    (257, 640, 32, 4, 0),        # one thread per block
+    (64, 3200, 128, 4, 0),       # 100 threads per row: too wide for whole-warp CTAs, generic kernel
 ]
 
 
