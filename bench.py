@@ -563,12 +563,40 @@ def main():
     h2d = sum(L["x_host"].numel() * L["x_host"].element_size() for L in layers)
     d2h = sum(L["y_host"].numel() * L["y_host"].element_size() for L in layers)
 
+    # Three streams: inputs go up on one, the layer calls run on the main one as each input lands, results come down
+    # on the third as each layer finishes; the timed region is bracketed on the main stream, which waits for the last
+    # download of a step before the next step's uploads may overwrite anything.
+    up, down = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+
     def e2e_step():
-        for L in layers:
-            L["x"].copy_(L["x_host"], non_blocking=True)
-        run_step(hq, layers, status)
-        for L in layers:
-            L["y_host"].copy_(L["y"], non_blocking=True)
+        ev_start = torch.cuda.Event()
+        ev_start.record(stream)
+        up.wait_event(ev_start)
+        landed, done = [], []
+        with torch.cuda.stream(up):
+            for L in layers:
+                L["x"].copy_(L["x_host"], non_blocking=True)
+                e = torch.cuda.Event()
+                e.record(up)
+                landed.append(e)
+        for L, e in zip(layers, landed):
+            stream.wait_event(e)
+            if L["kind"] == "linear":
+                hq.hq_qlinear(L["x"], L["pw"], L["bias"], A_BITS, L["y"], L["ws"], dev_status=status, stream=stream)
+            else:
+                c = CONV
+                hq.hq_qconv(L["x"], L["pw"], c["R"], c["S"], c["stride"], c["pad"], L["bias"], A_BITS, L["y"], L["ws"],
+                            static_scale=L["static_scale"], dev_status=status, stream=stream)
+            e2 = torch.cuda.Event()
+            e2.record(stream)
+            done.append(e2)
+        with torch.cuda.stream(down):
+            for L, e2 in zip(layers, done):
+                down.wait_event(e2)
+                L["y_host"].copy_(L["y"], non_blocking=True)
+            ev_end = torch.cuda.Event()
+            ev_end.record(down)
+        stream.wait_event(ev_end)
 
     e2e_step()
     barrier()
