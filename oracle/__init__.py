@@ -55,6 +55,7 @@ def lib():
             L.hqo_dequant.argtypes = [p, i64, i64, p, C.c_int, p, p, C.c_double, p]
             L.hqo_conv2d_dequant_perpixel.argtypes = [p, p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int,
                                                       C.c_int, C.c_int, p, p, C.c_double, p]
+            L.hqo_groupnorm_silu.argtypes = [p, i64, i64, i64, i64, C.c_int, p, p, C.c_double, p]
             L.hqo_transform_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
             L.hqo_codes_inverse_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
             L.hqo_conv2d_int_z.argtypes = [p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int, C.c_int, C.c_int, p]
@@ -237,6 +238,17 @@ def conv2d_dequant_perpixel(q, s_a, B, stride: int, pad: int, s_w, bias, alpha: 
     _chk(lib().hqo_conv2d_dequant_perpixel(_ptr(q), _ptr(s_a), _ptr(B), Nb, H, W, Cc, Cout, R, S, stride, pad,
                                            _ptr(s_w), _ptr(b), float(alpha), _ptr(y)), "conv2d_dequant_perpixel")
     return y
+
+
+def groupnorm_silu(x, groups: int, gamma, beta, eps: float = 1e-6) -> np.ndarray:
+    """GroupNorm over `groups` groups of consecutive channels of an NHWC tensor, affine, then SiLU (fp64)."""
+    x = _c(x, np.float64)
+    Nb, H, W, Cc = x.shape
+    gamma, beta = _c(gamma, np.float64), _c(beta, np.float64)
+    out = np.empty_like(x)
+    _chk(lib().hqo_groupnorm_silu(_ptr(x), Nb, H, W, Cc, groups, _ptr(gamma), _ptr(beta), float(eps), _ptr(out)),
+         "groupnorm_silu")
+    return out
 
 
 def transform_width(x, had_block: int) -> np.ndarray:

@@ -385,3 +385,33 @@ i64 hqo_conv2d_int_z(const int32_t* z, const int32_t* B, i64 Nb, i64 H, i64 W, i
     }
     return bad;
 }
+
+/* ---- GroupNorm + SiLU in front of a quantized convolution (the "in_layers" of a ResBlock) -------------------
+ * Not part of the paper's equations: the usual definitions, written out.  x NHWC [Nb][H][W][C], `groups` groups of
+ * C/groups consecutive channels; per sample and group: mean and biased variance over H*W*(C/groups) values;
+ * y = (x - mean) / sqrt(var + eps) * gamma[c] + beta[c];   out = y * sigmoid(y) = y / (1 + exp(-y)). */
+int hqo_groupnorm_silu(const double* x, i64 Nb, i64 H, i64 W, i64 C, int groups, const double* gamma,
+                       const double* beta, double eps, double* out) {
+    if (groups <= 0 || C % groups != 0) return -1;
+    const i64 cg = C / groups, HW = H * W;
+#pragma omp parallel for schedule(static)
+    for (i64 ng = 0; ng < Nb * groups; ++ng) {
+        const i64 n = ng / groups, g = ng % groups;
+        double sum = 0.0;
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) sum += x[(n * HW + p) * C + g * cg + c];
+        const double mean = sum / (double)(HW * cg);
+        double var = 0.0;
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) { const double d = x[(n * HW + p) * C + g * cg + c] - mean; var += d * d; }
+        var /= (double)(HW * cg);
+        const double rstd = 1.0 / sqrt(var + eps);
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) {
+                const i64 ch = g * cg + c, idx = (n * HW + p) * C + ch;
+                const double y = (x[idx] - mean) * rstd * gamma[ch] + beta[ch];
+                out[idx] = y / (1.0 + exp(-y));
+            }
+    }
+    return 0;
+}

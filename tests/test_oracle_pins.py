@@ -468,3 +468,23 @@ def test_width_conv_recovers_plain_conv_when_quantization_is_fine(oracle):
                 y += np.einsum("nhwc,oc->nhwo", xp[:, r:r + 5, s:s + 8, :], w_hat[:, r, s, :])
         errs.append(np.abs(out["y"] - y).max())
     assert errs[1] < errs[0] and errs[1] < 0.02
+
+
+# ------------------------------------------------------------------ GroupNorm + SiLU prologue
+
+def test_groupnorm_silu_against_library_routine(oracle):
+    """The written-out definition against torch's group_norm + silu on the CPU in fp64 (a library routine), plus two
+    closed forms: a constant input gives silu(beta); with gamma = 1, beta = 0 each group of the normalised tensor has
+    mean 0 and variance 1 / (1 + eps / var)."""
+    import torch
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((3, 5, 4, 24)) * 3.0 + 1.5
+    gamma, beta = rng.standard_normal(24), rng.standard_normal(24)
+    got = oracle.groupnorm_silu(x, 6, gamma, beta, eps=1e-5)
+    xt = torch.from_numpy(x).permute(0, 3, 1, 2)                                  # NCHW for the library
+    want = torch.nn.functional.silu(torch.nn.functional.group_norm(xt, 6, torch.from_numpy(gamma), torch.from_numpy(beta), 1e-5))
+    assert np.allclose(got, want.permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+    const = oracle.groupnorm_silu(np.full((1, 2, 2, 8), 7.0), 2, gamma[:8], beta[:8], eps=1e-6)
+    assert np.allclose(const, beta[:8] / (1 + np.exp(-beta[:8])), atol=1e-9)
+    with pytest.raises(ValueError):
+        oracle.groupnorm_silu(x, 5, gamma, beta)                                   # 24 channels do not split into 5 groups
