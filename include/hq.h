@@ -174,6 +174,21 @@ hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int
                          const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
                          int32_t* dev_status, void* stream);
 
+/* ---- GroupNorm + SiLU fused in front of the transform + quantization (no counterpart in the paper's equations:
+ * the normalisation and activation that precede the quantized 3x3 convolutions of a UNet ResBlock, applied while the
+ * activations are read, so that they make one trip through memory instead of three). ---------------------------------
+ * x        device NHWC [Nb][H][W][C] fp32/bf16, densely packed.
+ * groups   groups of C/groups consecutive channels (a multiple of 4 each); statistics per (sample, group) over
+ *          H*W*(C/groups) values: y = (x - mean) / sqrt(var + eps) * gamma[c] + beta[c]; then y * sigmoid(y).
+ * gamma, beta  device [C].   The rest as hq_hadamard_quant with rows = Nb*H*W, cols = C (transform over channels).
+ * scratch  device, 16-byte aligned, Nb * groups * 24 bytes: fp64 sums (cleared by the call) and the statistics.
+ * Restrictions: had_block in 32..4096 with at most 320 threads per CTA shape (else HQ_ERR_UNSUPPORTED), and the
+ * rows of a sample must be a multiple of the rows one CTA takes (any H*W that is a multiple of 32 is). */
+hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                           const float* gamma, const float* beta, float eps, int had_block, int bits,
+                           hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                           int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, void* stream);
+
 /* ---- Fused linear layer that allocates nothing and takes no workspace (the paper has no counterpart: this is a
  * packaging of hq_qlinear for a particular kind of caller, not another operation). ---------------------------------
  * Who it is for: code that must not, or cannot, obtain device memory at the moment it runs a layer -- an inference

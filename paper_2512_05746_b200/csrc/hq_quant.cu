@@ -32,9 +32,23 @@ struct QuantParams {
     uint8_t* codes;
     int64_t ld_codes;
     float* scales;
+    // optional GroupNorm + SiLU applied to the values as they are loaded (gn_stats == nullptr: off)
+    const float* gn_stats;   // [samples][groups][2]: mean, 1/sqrt(var + eps)
+    const float* gn_gamma;   // [cols]
+    const float* gn_beta;    // [cols]
+    int gn_groups;
+    int64_t gn_rows_per_sample;
 };
 
+__device__ __forceinline__ float silu(float y) { return __fdividef(y, 1.0f + __expf(-y)); }
+
 __device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4_keep(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4_keep(const __nv_bfloat16* p) {
+    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p));
+    return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u), __uint_as_float(raw.y << 16),
+                       __uint_as_float(raw.y & 0xFFFF0000u));
+}
 __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
     uint2 raw = __ldcs(reinterpret_cast<const uint2*>(p));
     float4 f;
@@ -194,12 +208,36 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
 
     if (!STATIC && tid < p.rows_per_cta) rowmax[tid] = 0u;
 
+    // GroupNorm + SiLU prologue: per-channel y = x * a[c] + b[c] with a = rstd * gamma, b = beta - mean * a of the
+    // sample this CTA's rows belong to (the host makes sure a CTA never straddles two samples), then y * sigmoid(y).
+    float* gn_a = reinterpret_cast<float*>(rowmax + ((p.rows_per_cta + 3) & ~3));
+    float* gn_b = gn_a + p.cols;
+    const bool gn = p.gn_stats != nullptr;
+    if (gn) {
+        const int64_t sample = (int64_t(blockIdx.x) * p.rows_per_cta) / p.gn_rows_per_sample;
+        const int cg = int(p.cols) / p.gn_groups;
+        for (int c = tid; c < int(p.cols); c += blockDim.x) {
+            const float2 st = *reinterpret_cast<const float2*>(p.gn_stats + (sample * p.gn_groups + c / cg) * 2);
+            const float a = st.y * __ldg(p.gn_gamma + c);
+            gn_a[c] = a;
+            gn_b[c] = fmaf(-st.x, a, __ldg(p.gn_beta + c));
+        }
+        __syncthreads();
+    }
+
     f32x2 v[P];
     {
         const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
 #pragma unroll
         for (int i = 0; i < E / 4; ++i) {
             float4 f = load4(src + 4 * (tb + TB * i));
+            if (gn) {
+                const int ch = blk * N + 4 * (tb + TB * i);
+                const float4 a4 = *reinterpret_cast<const float4*>(gn_a + ch);
+                const float4 b4 = *reinterpret_cast<const float4*>(gn_b + ch);
+                f.x = silu(fmaf(f.x, a4.x, b4.x)); f.y = silu(fmaf(f.y, a4.y, b4.y));
+                f.z = silu(fmaf(f.z, a4.z, b4.z)); f.w = silu(fmaf(f.w, a4.w, b4.w));
+            }
             if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
             v[2 * i] = pk2(f.x, f.y);
             v[2 * i + 1] = pk2(f.z, f.w);
@@ -472,6 +510,66 @@ __global__ void __launch_bounds__(256) width_quant_kernel(const WidthParams p) {
     }
 }
 
+// ---- GroupNorm statistics: sums and sums of squares per (sample, group), then mean and 1/sqrt(var + eps) --------
+// x NHWC; grid (chunks, samples); a thread owns channel quads (coalesced over channels) and walks the pixels of its
+// chunk, accumulating in fp64; per-CTA shared-memory reduction per group, one fp64 atomic pair per group and CTA.
+template <typename InT>
+__global__ void __launch_bounds__(256) gn_stats_kernel(const InT* x, int64_t hw, int C, int groups, int chunks,
+                                                       double* sums) {
+    extern __shared__ double s_acc[];                  // [groups][2]
+    for (int i = threadIdx.x; i < 2 * groups; i += blockDim.x) s_acc[i] = 0.0;
+    __syncthreads();
+    const int nq = C / 4 < 256 ? C / 4 : 256;          // channel quads walked side by side
+    const int ppl = 256 / nq;                          // pixels walked side by side
+    const int qd0 = threadIdx.x % nq, pl = threadIdx.x / nq;
+    const int64_t per = (hw + chunks - 1) / chunks;
+    const int64_t p0 = int64_t(blockIdx.x) * per, p1 = p0 + per < hw ? p0 + per : hw;
+    const int cg = C / groups;
+    const InT* base = x + int64_t(blockIdx.y) * hw * C;
+    if (pl < ppl) {
+        for (int qd = qd0; qd < C / 4; qd += nq) {
+            double s1 = 0.0, s2 = 0.0;
+            int64_t px = p0 + pl;
+            for (; px + 3 * ppl < p1; px += 4 * ppl) {     // four independent loads in flight
+                float4 f[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) f[u] = load4_keep(base + (px + u * ppl) * C + 4 * qd);   // read again by the quantize kernel: keep in L2
+                // sixteen values at a time in fp32 (relative error about 1e-7), then into the fp64 running sums:
+                // the fp32 -> fp64 conversions are the slow instructions here
+                float a1 = 0.f, a2 = 0.f;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    a1 += (f[u].x + f[u].y) + (f[u].z + f[u].w);
+                    a2 = fmaf(f[u].x, f[u].x, fmaf(f[u].y, f[u].y, fmaf(f[u].z, f[u].z, fmaf(f[u].w, f[u].w, a2))));
+                }
+                s1 += double(a1);
+                s2 += double(a2);
+            }
+            for (; px < p1; px += ppl) {
+                const float4 f = load4_keep(base + px * C + 4 * qd);
+                s1 += double(f.x) + double(f.y) + double(f.z) + double(f.w);
+                s2 += double(f.x) * f.x + double(f.y) * f.y + double(f.z) * f.z + double(f.w) * f.w;
+            }
+            const int g = 4 * qd / cg;                 // cg is a multiple of 4 (checked on the host)
+            atomicAdd(&s_acc[2 * g], s1);
+            atomicAdd(&s_acc[2 * g + 1], s2);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * groups; i += blockDim.x)
+        atomicAdd(&sums[int64_t(blockIdx.y) * 2 * groups + i], s_acc[i]);
+}
+
+__global__ void gn_finalize_kernel(const double* sums, int64_t count, double eps, int total, float* stats) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const double mean = sums[2 * i] / double(count);
+    double var = sums[2 * i + 1] / double(count) - mean * mean;
+    if (var < 0.0) var = 0.0;
+    stats[2 * i] = float(mean);
+    stats[2 * i + 1] = float(1.0 / sqrt(var + eps));
+}
+
 template <int KLOG, int E, typename InT>
 cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threads, size_t smem, cudaStream_t st) {
     const bool stat = p.static_scale != nullptr;
@@ -509,9 +607,12 @@ cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int gri
 }  // namespace
 
 // Launches the transform+quantize kernel; shared by the public entry point and the fused layer calls.
-hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
-                                int bits, hq_scale_mode mode, const float* static_scale, void* codes,
-                                hq_container cont, int64_t ld_codes, float* scales, cudaStream_t st) {
+struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; };
+
+static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
+                                   int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                   hq_container cont, int64_t ld_codes, float* scales, const GnArgs* gn,
+                                   cudaStream_t st) {
     if (rows == 0 && cols > 0) return HQ_OK;                       // nothing to do; pointers may be NULL
     if (x == nullptr || codes == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
@@ -537,6 +638,10 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
     p.codes = static_cast<uint8_t*>(codes);
     p.ld_codes = ld_codes;
     p.scales = scales;
+    if (gn != nullptr) {
+        p.gn_stats = gn->stats; p.gn_gamma = gn->gamma; p.gn_beta = gn->beta; p.gn_groups = gn->groups;
+        p.gn_rows_per_sample = gn->rows_per_sample;
+    }
 
     const int elt = xdt == HQ_F32 ? 4 : 2;
     const int E = fast_e(klog);
@@ -554,10 +659,12 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
         p.threads_per_row = tr;
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
+        if (gn != nullptr && gn->rows_per_sample % rpc != 0) return HQ_ERR_UNSUPPORTED;   // a CTA must stay in one sample
         if (threads <= 320) {                               // otherwise the generic kernel below takes the row shape
         // exchange buffer: per Hadamard block n/4 float4 slots plus one slot of padding per J (J = E/2 or E/4)
         const int jslots = (klog - ilog2(E) >= ilog2(E) - 1) ? E / 2 : E / 4;
-        const size_t smem = size_t(threads / (n / E)) * size_t(n / 4 + n / 4 / jslots) * 16 + size_t(rpc) * 4;
+        const size_t smem = size_t(threads / (n / E)) * size_t(n / 4 + n / 4 / jslots) * 16 + size_t((rpc + 3) & ~3) * 4 +
+                            (gn != nullptr ? size_t(cols) * 8 : 0);
         const int grid = int((rows + rpc - 1) / rpc);
         cudaError_t e = xdt == HQ_F32
                             ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
@@ -565,6 +672,7 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
         return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
         }
     }
+    if (gn != nullptr) return HQ_ERR_UNSUPPORTED;           // the prologue exists in the fast kernel only
     const size_t smem = size_t(cols) * 4;
     if (smem > 200 * 1024) return HQ_ERR_UNSUPPORTED;
     const int grid = int(rows < 148 * 8 ? rows : 148 * 8);
@@ -582,6 +690,56 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
     }
     e = cudaGetLastError();
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
+                                int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                hq_container cont, int64_t ld_codes, float* scales, cudaStream_t st) {
+    return launch_quant_impl(x, xdt, rows, cols, ldx, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales,
+                             nullptr, st);
+}
+
+// GroupNorm + SiLU of an NHWC tensor fused into the transform+quantize kernel: statistics per (sample, group) first
+// (fp64 sums in `scratch`, which is cleared here), then the quantize kernel applies x * a[c] + b[c] and SiLU as it
+// loads.  scratch: Nb * groups * (2 doubles + 2 floats).
+hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                               const float* gamma, const float* beta, float eps, int had_block, int bits,
+                               hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                               int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st) {
+    if (x == nullptr || gamma == nullptr || beta == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
+    if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
+    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0 || groups <= 0) return HQ_ERR_SHAPE;
+    if (C % groups != 0 || (C / groups) % 4 != 0) return HQ_ERR_SHAPE;      // whole channel quads per group
+    if (groups > 1024) return HQ_ERR_UNSUPPORTED;
+    const size_t need = size_t(Nb) * groups * (2 * sizeof(double) + 2 * sizeof(float));
+    if (scratch_bytes < need) return HQ_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(scratch) % 16 != 0) return HQ_ERR_ALIGNMENT;
+    const int elt = xdt == HQ_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(x) % (4 * elt) != 0) return HQ_ERR_ALIGNMENT;
+    double* sums = static_cast<double*>(scratch);
+    float* stats = reinterpret_cast<float*>(sums + size_t(Nb) * groups * 2);
+    const int64_t hw = H * W;
+    HQ_CUDA_OK(cudaMemsetAsync(sums, 0, size_t(Nb) * groups * 2 * sizeof(double), st));
+    // enough CTAs that a thread walks about 16 pixels per channel quad (short dependent chains, many loads in flight)
+    const int64_t ppl = C / 4 < 256 ? 256 / (C / 4) : 1;
+    int64_t chunks = hw / (ppl * 16);
+    if (chunks > 1024) chunks = 1024;
+    if (chunks < 1) chunks = 1;
+    if (Nb > 65535) return HQ_ERR_UNSUPPORTED;
+    const dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(Nb));
+    const size_t smem = size_t(groups) * 2 * sizeof(double);
+    if (xdt == HQ_F32)
+        gn_stats_kernel<float><<<grid, 256, smem, st>>>(static_cast<const float*>(x), hw, int(C), groups, int(chunks), sums);
+    else
+        gn_stats_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(x), hw, int(C), groups,
+                                                                 int(chunks), sums);
+    if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+    const int total = int(Nb * groups);
+    gn_finalize_kernel<<<(total + 127) / 128, 128, 0, st>>>(sums, hw * (C / groups), double(eps), total, stats);
+    if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
+    const GnArgs gn{stats, gamma, beta, groups, hw};
+    return launch_quant_impl(x, xdt, Nb * hw, C, C, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales, &gn,
+                             st);
 }
 
 // Width-axis transform + quantization + integer factor of Eq. 13-14: x NHWC fp32/bf16 -> z int8 NHWC.
@@ -623,6 +781,15 @@ hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, i
 }
 
 }  // namespace hq
+
+extern "C" hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                      int groups, const float* gamma, const float* beta, float eps, int had_block,
+                                      int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                      hq_container cont, int64_t ld_codes, float* scales, void* scratch,
+                                      size_t scratch_bytes, void* stream) {
+    return hq::launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, had_block, bits, mode, static_scale, codes,
+                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream));
+}
 
 extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                              int had_block_w, int bits, const float* static_scale, void* z_codes,
