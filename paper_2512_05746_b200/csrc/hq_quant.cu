@@ -179,7 +179,7 @@ __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, i
 //            two threads of a group interleave their bytes with one shuffle so that each stores contiguous bytes.
 //            KLOG = 12 needs one more stage than fits and takes it with a lane exchange.
 // Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
-template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC>
+template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC, bool GN>
 __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     constexpr int N = 1 << KLOG;
     constexpr int LE = ilog2_c(E);
@@ -212,8 +212,7 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     // sample this CTA's rows belong to (the host makes sure a CTA never straddles two samples), then y * sigmoid(y).
     float* gn_a = reinterpret_cast<float*>(rowmax + ((p.rows_per_cta + 3) & ~3));
     float* gn_b = gn_a + p.cols;
-    const bool gn = p.gn_stats != nullptr;
-    if (gn) {
+    if (GN) {
         const int64_t sample = (int64_t(blockIdx.x) * p.rows_per_cta) / p.gn_rows_per_sample;
         const int cg = int(p.cols) / p.gn_groups;
         for (int c = tid; c < int(p.cols); c += blockDim.x) {
@@ -231,7 +230,7 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
 #pragma unroll
         for (int i = 0; i < E / 4; ++i) {
             float4 f = load4(src + 4 * (tb + TB * i));
-            if (gn) {
+            if (GN) {
                 const int ch = blk * N + 4 * (tb + TB * i);
                 const float4 a4 = *reinterpret_cast<const float4*>(gn_a + ch);
                 const float4 b4 = *reinterpret_cast<const float4*>(gn_b + ch);
@@ -581,8 +580,12 @@ cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threa
         kern<<<grid, threads, smem, st>>>(p);
         return cudaGetLastError();
     };
-    if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true>) : go(fwht_quant_fast<KLOG, E, InT, true, false>);
-    return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true>) : go(fwht_quant_fast<KLOG, E, InT, false, false>);
+    if (p.gn_stats != nullptr) {
+        if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, true>) : go(fwht_quant_fast<KLOG, E, InT, true, false, true>);
+        return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, true>) : go(fwht_quant_fast<KLOG, E, InT, false, false, true>);
+    }
+    if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, false>) : go(fwht_quant_fast<KLOG, E, InT, true, false, false>);
+    return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, false>) : go(fwht_quant_fast<KLOG, E, InT, false, false, false>);
 }
 
 // Values per thread for a block of 2^klog channels.
