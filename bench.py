@@ -33,12 +33,25 @@ UNIT = "TOPS"
 M_TOKENS = 32768
 CONV = dict(Nb=32, H=32, W=32, C=256, Cout=256, R=3, S=3, stride=1, pad=1, had_block=256)
 WORKLOAD = ("configs[2] transformer-block linears (M=32768; QKV, out-proj, FF1, FF2) + configs[1] 3x3 conv at "
-            "batch 32 (M=32768, K=2304, N=256); W4A4, folded 2-limb weights, nibble codes, bf16 out")
+            "batch 32 (M=32768, K=2304, N=256); W4A4, folded 2-limb weights, bf16 out")
 A_BITS, W_BITS = 4, 4
+# Container of the 4-bit activation codes between the two kernels of a layer: 0 = HQ_CODES_NIBBLE (two per byte,
+# unpacked inside the GEMM kernel), 1 = HQ_CODES_INT8 (one per byte); set by --codes.
+CODES = [1]
+
+
+def code_pitch(cols):
+    """Bytes per row of `cols` codes in the selected container."""
+    return cols // 2 if CODES[0] == 0 else cols
+
+
+def codes_name():
+    return "nibble" if CODES[0] == 0 else "int8"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at the full size of the default step, from the one-pass ncu
 # capture of this command (a summary is kept under profiles/; taken with these kernel versions: set an entry to
 # None when its kernel changes).  Outputs partly stay in L2 past the end of a launch, so these are below the
 # algorithmic bytes.
+NCU_DRAM_CODES = 0      # container the counters below were taken with (0 = nibble)
 NCU_DRAM_BYTES = {"gemm": {"qkv": 54.2e6, "ff1": 88.8e6, "ff2": 36.0e6, "conv3x3": 5.4e6, "out_proj": None},
                   "quant": {"qkv": 67.5e6, "out_proj": 67.5e6, "ff1": 67.5e6, "ff2": 275.1e6, "conv3x3": None}}
 
@@ -128,7 +141,7 @@ def build_layers(torch, hq, device, seed):
             c = CONV
             cfg = inputs.config_conv_small(seed=seed, batch=c["Nb"])
             x_host, w, b = cfg["x"], cfg["w"], cfg["bias"]
-        pw = hq.hq_weight_prepare(w, W_BITS, L["had_block"], hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE).to_device(device)
+        pw = hq.hq_weight_prepare(w, W_BITS, L["had_block"], hq.HQ_W_FOLDED, CODES[0]).to_device(device)
         L["pw"] = pw
         L["limbs"] = pw.desc.limbs
         L["x_host"] = torch.from_numpy(x_host).pin_memory()
@@ -136,16 +149,17 @@ def build_layers(torch, hq, device, seed):
         L["bias"] = torch.from_numpy(b).to(device)
         rows, cols = (L["M"], L["K"]) if L["kind"] == "linear" else (L["M"], CONV["C"])
         L["rows"], L["cols"] = rows, cols
-        ws_bytes = hq.hq_workspace_size(rows, cols, hq.HQ_CODES_NIBBLE)
+        ws_bytes = hq.hq_workspace_size(rows, cols, CODES[0])
         L["ws"] = torch.empty((ws_bytes,), dtype=torch.uint8, device=device)
         oshape = (L["M"], L["N"]) if L["kind"] == "linear" else (CONV["Nb"], CONV["H"], CONV["W"], CONV["Cout"])
         L["y"] = torch.empty(oshape, dtype=torch.bfloat16, device=device)
         L["y_host"] = torch.empty(oshape, dtype=torch.bfloat16).pin_memory()
         L["ops"] = 2.0 * L["M"] * L["N"] * L["K"] * L["limbs"]
         L["ops_1limb"] = 2.0 * L["M"] * L["N"] * L["K"]
-        # algorithmic HBM bytes of the two kernels (fp32 in, nibble codes out + scales; codes + weights in, bf16 out)
-        L["quant_bytes"] = rows * cols * 4.0 + rows * cols * 0.5 + rows * 4.0
-        L["gemm_bytes"] = (L["M"] * L["K"] * 0.5 if L["kind"] == "linear" else rows * cols * 0.5) + \
+        # algorithmic HBM bytes of the two kernels (fp32 in, codes out + scales; codes + weights in, bf16 out)
+        cb = float(code_pitch(2)) / 2.0                                      # bytes per code
+        L["quant_bytes"] = rows * cols * 4.0 + rows * cols * cb + rows * 4.0
+        L["gemm_bytes"] = (L["M"] * L["K"] * cb if L["kind"] == "linear" else rows * cols * cb) + \
             L["N"] * L["K"] * L["limbs"] + L["M"] * L["N"] * 2.0 + 4.0 * L["M"] + 8.0 * L["N"]
         L["static_scale"] = None
     torch.cuda.synchronize()
@@ -154,10 +168,10 @@ def build_layers(torch, hq, device, seed):
     for L in layers:
         if L["kind"] == "conv":
             x2d = L["x"].view(L["rows"], L["cols"])
-            pitch = L["cols"] // 2
+            pitch = code_pitch(L["cols"])
             codes = torch.empty((L["rows"], pitch), dtype=torch.uint8, device=device)
             scales = torch.empty((L["rows"],), dtype=torch.float32, device=device)
-            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales)
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, CODES[0], scales=scales)
             L["static_scale"] = scales.max().reshape(1).contiguous()
     torch.cuda.synchronize()
     return layers
@@ -178,7 +192,7 @@ def run_step_split(torch, hq, layers, status, evs):
     stream = torch.cuda.current_stream()
     for L in layers:
         rows, cols = L["rows"], L["cols"]
-        pitch = cols // 2
+        pitch = code_pitch(cols)
         codes = L["ws"][: rows * pitch].view(rows, pitch)
         off = (rows * pitch + 255) // 256 * 256
         scales = L["ws"][off: off + rows * 4].view(torch.float32)
@@ -186,16 +200,16 @@ def run_step_split(torch, hq, layers, status, evs):
         e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         e0.record(stream)
         if L["kind"] == "linear":
-            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales)
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, CODES[0], scales=scales)
             e1.record(stream)
-            hq.hq_qgemm(codes, hq.HQ_CODES_NIBBLE, A_BITS, L["K"], L["pw"], scale_a=scales, bias=L["bias"],
+            hq.hq_qgemm(codes, CODES[0], A_BITS, L["K"], L["pw"], scale_a=scales, bias=L["bias"],
                         alpha=L["pw"].alpha, y=L["y"], dev_status=status)
         else:
             c = CONV
-            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=scales[:1],
+            hq.hq_hadamard_quant(x2d, L["had_block"], A_BITS, codes, CODES[0], scales=scales[:1],
                                  static_scale=L["static_scale"])
             e1.record(stream)
-            hq.hq_qconv2d(codes, hq.HQ_CODES_NIBBLE, A_BITS, c["Nb"], c["H"], c["W"], c["C"], L["pw"], c["R"], c["S"],
+            hq.hq_qconv2d(codes, CODES[0], A_BITS, c["Nb"], c["H"], c["W"], c["C"], L["pw"], c["R"], c["S"],
                           c["stride"], c["pad"], scale_a=L["static_scale"], bias=L["bias"], alpha=L["pw"].alpha,
                           y=L["y"], dev_status=status)
         e2.record(stream)
@@ -302,16 +316,16 @@ def main_layer_list(args, which):
         x[:, torch.randperm(cin, generator=gen, device=dev)[:nout]] *= 20.0          # outlier channels
         x = x.to(torch.bfloat16)
         pw = hq.hq_weight_prepare(inputs.weights(wshape, seed=len(cache)), W_BITS, L["had_block"], hq.HQ_W_FOLDED,
-                                  hq.HQ_CODES_NIBBLE).to_device(dev)
+                                  CODES[0]).to_device(dev)
         res = dict(x=x.view((L["Nb"], L["H"], L["W"], cin)) if L["kind"] == "conv" else x, pw=pw,
                    bias=torch.from_numpy(inputs.bias(cout, seed=len(cache))).to(dev),
                    y=torch.empty(oshape, dtype=torch.bfloat16, device=dev),
-                   ws=torch.empty((hq.hq_workspace_size(rows, cin, hq.HQ_CODES_NIBBLE),), dtype=torch.uint8, device=dev),
+                   ws=torch.empty((hq.hq_workspace_size(rows, cin, CODES[0]),), dtype=torch.uint8, device=dev),
                    static=None)
         if L["kind"] == "conv" and L["R"] == 3:           # calibrate the static scale with one dynamic pass
-            codes = torch.empty((rows, cin // 2), dtype=torch.uint8, device=dev)
+            codes = torch.empty((rows, code_pitch(cin)), dtype=torch.uint8, device=dev)
             sc = torch.empty((rows,), dtype=torch.float32, device=dev)
-            hq.hq_hadamard_quant(x, L["had_block"], A_BITS, codes, hq.HQ_CODES_NIBBLE, scales=sc)
+            hq.hq_hadamard_quant(x, L["had_block"], A_BITS, codes, CODES[0], scales=sc)
             res["static"] = sc.max().reshape(1).contiguous()
             del codes, sc
         cache[k] = res
@@ -367,7 +381,7 @@ def main_layer_list(args, which):
     print(json.dumps(dict(metric="forwards/s of " + label,
                           value=1e3 / ms, unit="forwards/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=ms,
                           higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int8", data="synthetic",
-                          config=dict(workload=wl + ", bf16 in/out, W4A4 folded two-limb weights, nibble codes",
+                          config=dict(workload=wl + ", bf16 in/out, W4A4 folded two-limb weights, " + codes_name() + " codes",
                                       layers=len(layers),
                                       layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
@@ -459,9 +473,14 @@ def main():
     ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep"],
                     help="step: the benchmark step (default); unet / dit: the quantized layers of the UNet- / DiT-shaped workload; "
                          "sweep: the M x K x N shape sweep")
+    ap.add_argument("--codes", default="int8", choices=["nibble", "int8"],
+                    help="container of the 4-bit activation codes between the transform and the GEMM kernel: one per "
+                         "byte (default, the faster one) or two per byte (half the workspace)")
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     args = ap.parse_args()
+    CODES[0] = 0 if args.codes == "nibble" else 1
+    WORKLOAD = WORKLOAD + f", {args.codes} codes"
     if args.rows != M_TOKENS:
         M_TOKENS = int(args.rows)
         WORKLOAD = f"REDUCED to {M_TOKENS} rows per layer (profiling case, not a benchmark number): " + WORKLOAD
@@ -623,10 +642,10 @@ def main():
         L = dom["L"]
         gemm_ms = dom["gemm_ms"] / dom["n"]
         ach = L["ops"] / (gemm_ms * 1e-3) / 1e12
-        roofline = dict(bound="tensor", kernel=f"qgemm_kernel<nibble> ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
+        roofline = dict(bound="tensor", kernel=f"qgemm_kernel<{codes_name()}> ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
                                                 f"limbs={L['limbs']})",
                         achieved=ach, peak=int8_peak, unit="TOPS", frac=ach / int8_peak,
-                        traffic=NCU_DRAM_BYTES["gemm"].get(L["name"]) if M_TOKENS == 32768 else None,
+                        traffic=NCU_DRAM_BYTES["gemm"].get(L["name"]) if (M_TOKENS == 32768 and CODES[0] == NCU_DRAM_CODES) else None,
                         algorithmic_bytes=L["gemm_bytes"],
                         peak_source=f"2 x bf16 sustained ({pk['source']})", launch_ms=gemm_ms)
         qd = max(per.values(), key=lambda d: d["quant_ms"])
@@ -634,7 +653,7 @@ def main():
         q_gbs = qd["L"]["quant_bytes"] / (q_ms * 1e-3) / 1e9
         roofline_quant = dict(bound="hbm", kernel=f"fwht_quant_fast ({qd['L']['name']}: {qd['L']['rows']}x{qd['L']['cols']})",
                               achieved=q_gbs, peak=pk["hbm_gbs"], unit="GB/s", frac=q_gbs / pk["hbm_gbs"],
-                              traffic=NCU_DRAM_BYTES["quant"].get(qd["L"]["name"]) if M_TOKENS == 32768 else None,
+                              traffic=NCU_DRAM_BYTES["quant"].get(qd["L"]["name"]) if (M_TOKENS == 32768 and CODES[0] == NCU_DRAM_CODES) else None,
                               algorithmic_bytes=qd["L"]["quant_bytes"],
                               peak_source=f"copy bandwidth ({pk['source']})", launch_ms=q_ms)
         per_layer = {k: dict(quant_ms=d["quant_ms"] / d["n"], gemm_ms=d["gemm_ms"] / d["n"],
