@@ -98,17 +98,17 @@ bool encode_4d(CUtensorMap* tm, const void* base, const uint64_t dims_in[4], con
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Output tensor map for the epilogue's bulk stores: bf16 [rows][N] with pitch ldy, boxes of 32 rows x `box_cols`
-// columns (32: 64-byte swizzle, 16: 32-byte swizzle), the layout the staging buffers are written in.
-bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy, uint32_t box_cols) {
+// Output tensor map for the epilogue's bulk stores: bf16 [rows][N] with pitch ldy, boxes of 32 rows x 32 columns
+// in the 64-byte swizzle the staging buffers are written in.
+bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[2] = {N, rows};
     cuuint64_t strides[1] = {ldy * 2};
-    cuuint32_t box[2] = {box_cols, 32};
+    cuuint32_t box[2] = {32, 32};
     cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(y), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -125,11 +125,11 @@ int sm_count() {
 }
 
 // Ring depth and weight residency for a problem; fills p.stages / p.b_resident and returns the shared-memory size.
-size_t plan_smem(GemmParams& p, int epi) {
+size_t plan_smem(GemmParams& p) {
     const int num_kb = p.kb_per_tap * p.taps;
     p.b_resident = num_kb <= kResidentKb ? 1 : 0;
     for (int stages = kMaxStages; stages >= 2; --stages) {
-        const SmemLayout L = smem_layout(stages, p.b_resident != 0, num_kb, epi);
+        const SmemLayout L = smem_layout(stages, p.b_resident != 0, num_kb);
         if (L.total <= kSmemLimit) { p.stages = stages; return size_t(L.total); }
     }
     return 0;
@@ -137,14 +137,13 @@ size_t plan_smem(GemmParams& p, int epi) {
 
 hq_status launch(bool nibble, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmParams& p,
                  cudaStream_t st) {
-    // the kernel's fast epilogue assumes exactly these conditions
-    const bool fast = p.tma_store && !p.per_tap && p.y != nullptr && p.acc_out == nullptr && p.combine_fast;
-    const int mode = p.per_tap ? kModePerTap : fast ? kModeFast : kModeGeneric;
-    if ((p.epi_wide != 0) != wide_epilogue(nibble, fast, p.kb_per_tap * p.taps)) return HQ_ERR_UNSUPPORTED;
-    const size_t smem = plan_smem(p, epi_warps(p.epi_wide != 0));
+    const size_t smem = plan_smem(p);
     if (smem == 0) return HQ_ERR_UNSUPPORTED;
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < sm_count() ? tiles : sm_count();
+    // the kernel's fast epilogue assumes exactly these conditions
+    const bool fast = p.tma_store && !p.per_tap && p.y != nullptr && p.acc_out == nullptr && p.combine_fast;
+    const int mode = p.per_tap ? kModePerTap : fast ? kModeFast : kModeGeneric;
     cudaError_t e;
     if (nibble) e = p.conv ? launch_nibble_conv(mode, grid, smem, st, tmA, tmB, tmY, p)
                            : launch_nibble_gemm(mode, grid, smem, st, tmA, tmB, tmY, p);
@@ -221,9 +220,7 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
         return HQ_ERR_CUDA;
     // bf16 output: the epilogue hands 32 x 32 blocks to the copy engine (rows of a GEMM tile are consecutive)
     p.tma_store = (y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast) ? 1 : 0;
-    p.epi_wide = wide_epilogue(nib, p.tma_store != 0, p.kb_per_tap * p.taps) ? 1 : 0;
-    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy),
-                                 uint32_t(staging_bytes(epi_warps(p.epi_wide != 0)) / 64))) return HQ_ERR_CUDA;
+    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad);
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, kBN, true)) return HQ_ERR_CUDA;
     return launch(nib, tmA, tmB, tmY, p, st);
@@ -284,9 +281,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     const bool rows_consecutive = p.bw == Wo && p.bw * p.bh * p.bn == kBM && (p.bh == Ho || (p.bn == 1 && Ho % p.bh == 0));
     p.per_tap = per_tap ? 1 : 0;
     p.tma_store = (!per_tap && y != nullptr && acc_out == nullptr && p.y_bf16 && p.y_vec_ok && p.combine_fast && rows_consecutive) ? 1 : 0;
-    p.epi_wide = wide_epilogue(nib, p.tma_store != 0, p.kb_per_tap * p.taps) ? 1 : 0;
-    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(Nb * Ho * Wo), uint64_t(desc->N),
-                                 uint32_t(staging_bytes(epi_warps(p.epi_wide != 0)) / 64))) return HQ_ERR_CUDA;
+    if (p.tma_store && !encode_y(&tmY, y, uint64_t(desc->N), uint64_t(Nb * Ho * Wo), uint64_t(desc->N))) return HQ_ERR_CUDA;
     const uint64_t dims[4] = {uint64_t(row_bytes), uint64_t(W), uint64_t(H), uint64_t(Nb)};
     // With a traversal stride the box extent is given in input elements: stride * (pixels wanted).
     const uint32_t box[4] = {uint32_t(nib ? kBK / 2 : kBK), uint32_t(p.bw * stride), uint32_t(p.bh * stride), uint32_t(p.bn)};

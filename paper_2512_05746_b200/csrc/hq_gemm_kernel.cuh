@@ -20,17 +20,9 @@ constexpr int kABytes = kBM * kBK;           // 16 KB
 constexpr int kBBytes = kBN * kBK;           // 32 KB
 constexpr int kRawBytes = kBM * kBK / 2;     // 8 KB packed activation tile (lands in the upper half of its A stage)
 constexpr int kTmemCols = 512;
-// Epilogue warps: a warp may read only the TMEM lane quarter (warp index % 4), so there are 4 * P of them and each
-// takes 1/P of the tile's columns.  P = 2 normally; P = 4 ("wide") is offered for the fast output mode with the
-// one-code-per-byte container (no unpack warps, so the CTA has room and the register budget holds) and chosen by the
-// host for K_pad <= 256, where the epilogue is by far the longer half of a tile: measured 18 % faster at K = 256,
-// within +-3 % at K = 512 (slower inside whole networks), and 3-6 % slower with streamed weights.
-__host__ __device__ constexpr int epi_warps(bool wide) { return wide ? 16 : 8; }
-__host__ __device__ constexpr int cta_threads(bool nibble, bool wide) { return (2 + epi_warps(wide) + (nibble ? 4 : 0)) * 32; }
-inline bool wide_epilogue(bool nibble, bool fast, int num_kb) { return !nibble && fast && num_kb <= 2; }
-// Staging buffer of an epilogue warp: 32 rows x 64 bytes with 8 epilogue warps, 32 rows x 32 bytes with 16.
-__host__ __device__ constexpr int staging_bytes(int epi) { return epi == 16 ? 1024 : 2048; }
-constexpr int kParamBytes = 4 * 2 * kBN * 4; // all epilogue warps together: per lane quarter [scale_w | bias][kBN columns]
+constexpr int kEpiWarps = 8;            // two per TMEM lane quarter, each taking half of the tile's columns
+constexpr int kStagingBytes = 2048;          // per epilogue warp: 32 rows x 64 bytes
+constexpr int kParamBytes = kEpiWarps * 2 * (kBN / 2) * 4;   // per epilogue warp: [scale_w | bias][its columns]
 constexpr int kSmemLimit = 232448;           // 227 KB
 
 struct GemmParams {
@@ -55,7 +47,6 @@ struct GemmParams {
     int y_vec_ok, acc_vec_ok;
     int per_tap;          // convolution with one activation scale per input pixel: the accumulator is drained per filter tap
     int col_pass;         // per_tap with one weight limb: which 64 of a warp's 128 columns this launch produces
-    int epi_wide;         // sixteen epilogue warps (see epi_warps)
     int tma_store;        // bf16 output goes out through bulk tensor stores (rows of a tile are consecutive output rows)
     int32_t* dev_status;
 };
@@ -75,12 +66,12 @@ struct SharedCtl {
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout { int b_off, a_off, staging_off, param_off, ctl_off, total; };
-__host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int num_kb, int epi) {
+__host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int num_kb) {
     SmemLayout L;
     L.b_off = 0;
     L.a_off = (resident ? num_kb : stages) * kBBytes;
     L.staging_off = L.a_off + stages * kABytes;
-    L.param_off = L.staging_off + epi * staging_bytes(epi);
+    L.param_off = L.staging_off + kEpiWarps * kStagingBytes;
     L.ctl_off = L.param_off + kParamBytes;
     L.total = L.ctl_off + int(sizeof(SharedCtl)) + 1024;      // + slack for the base alignment
     return L;
@@ -256,19 +247,17 @@ __device__ __forceinline__ void store_row16(void* out_row, const uint32_t (&v)[1
 
 // Epilogue of one warp for the common case: bf16 output written by bulk tensor stores, limbs recombined as
 // 256*hi + lo without overflow.  Per 16 columns: two TMEM loads, one integer multiply-add, int->float, two float
-// operations per value, bf16 packing and two 16-byte stores into the warp's staging buffer, which is laid out in the
-// swizzle of the output tensor map: 32 rows x 64 bytes (SC = 32 columns, 64-byte swizzle, handed to the copy engine
-// every second step) or 32 rows x 32 bytes (SC = 16, 32-byte swizzle, handed over every step).  The copy engine
-// clips rows and columns beyond the output, and the warp carries on with the next columns; before the buffer is
-// written again one lane waits until the engine has read it.
-template <int LIMBS, int CPW, int SC>
+// operations per value, bf16 packing and two 16-byte stores into the warp's staging buffer (32 rows x 64 bytes, laid
+// out in the 64-byte swizzle of the output tensor map); every 32 columns one lane hands the buffer to the copy
+// engine, which clips rows and columns beyond the output, and the warp carries on with the next columns.  Before
+// the buffer is written again the lane waits until the engine has read it.
+template <int LIMBS>
 __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
                                               const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0,
                                               int row0, uint64_t* tempty_bar) {
-    constexpr int NSTEPS = CPW / 16;               // CPW: output columns of this warp (a multiple of 32)
-    constexpr int SPB = SC / 16;                   // steps per staging buffer
-    const uint32_t wsw = SC == 32 ? (lane >> 1) & 3 : (lane >> 2) & 1;
-    unsigned char* wr = stg + lane * (SC * 2);
+    constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
+    const uint32_t wsw = (lane >> 1) & 3;
+    unsigned char* wr = stg + lane * 64;
     uint32_t hi[16], lo[16];
     tmem_ld_32x16(t_row, hi);
     if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
@@ -292,7 +281,7 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar);
         }
-        if (st % SPB == 0) {                           // the copy engine must be done reading the staging buffer
+        if ((st & 1) == 0) {                           // the copy engine must be done reading the staging buffer
             if (lane == 0) bulk_wait_read_all();
             __syncwarp();
         }
@@ -306,13 +295,13 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
             o.y = pack_bf16x2(fmaf(float(w[8 * j + 2]) * s0.z, sa_eff, c0.z), fmaf(float(w[8 * j + 3]) * s0.w, sa_eff, c0.w));
             o.z = pack_bf16x2(fmaf(float(w[8 * j + 4]) * s1.x, sa_eff, c1.x), fmaf(float(w[8 * j + 5]) * s1.y, sa_eff, c1.y));
             o.w = pack_bf16x2(fmaf(float(w[8 * j + 6]) * s1.z, sa_eff, c1.z), fmaf(float(w[8 * j + 7]) * s1.w, sa_eff, c1.w));
-            *reinterpret_cast<uint4*>(wr + (((2 * (st % SPB) + j) ^ wsw) << 4)) = o;
+            *reinterpret_cast<uint4*>(wr + (((2 * (st & 1) + j) ^ wsw) << 4)) = o;
         }
-        if (st % SPB == SPB - 1) {
+        if (st & 1) {
             fence_proxy_async_smem();                  // the lanes' writes become visible to the copy engine
             __syncwarp();
             if (lane == 0) {
-                tma_store_2d(tmY, stg, col0 + (st / SPB) * SC, row0);
+                tma_store_2d(tmY, stg, col0 + (st >> 1) * 32, row0);
                 bulk_commit_group();
             }
         }
@@ -327,22 +316,19 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
 //   CONV     implicit-GEMM convolution (4-D activation boxes, pixel geometry) or plain GEMM,
 //   LIMBS_T  weight limbs (1 or 2), or 0 = read at run time,
 //   RES_T    weights resident (1) / streamed (0), or -1 = read at run time,
-//   WIDE     sixteen epilogue warps instead of eight (fast mode, one code per byte only),
 // because the hot loop of each role is short and runs once per tile: run-time branches over these choices and the
 // code of the paths not taken cost 10-15 % on the K <= 512 shapes (instruction fetch and bookkeeping per tile).
-template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T, bool WIDE>
-__global__ void __launch_bounds__(cta_threads(NIBBLE, WIDE), 1)
+template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T>
+__global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const GemmParams p) {
     constexpr bool PERTAP = MODE == kModePerTap;
-    constexpr int EPI = epi_warps(WIDE);              // epilogue warps
-    constexpr int CPARTS = EPI / 4;                   // column parts of a tile, one per epilogue warp of a lane quarter
     const int limbs = LIMBS_T != 0 ? LIMBS_T : p.limbs;
     const bool resident = RES_T >= 0 ? (RES_T != 0) : (p.b_resident != 0);
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int num_kb = p.kb_per_tap * p.taps;
-    const SmemLayout L = smem_layout(p.stages, resident, num_kb, EPI);
+    const SmemLayout L = smem_layout(p.stages, resident, num_kb);
     unsigned char* sB = smem + L.b_off;
     unsigned char* sA = smem + L.a_off;
     unsigned char* sStage = smem + L.staging_off;
@@ -362,7 +348,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         for (int k = 0; k < kResidentKb; ++k) mbar_init(&ctl->bfull[k], 1);
         mbar_init(&ctl->bfree, 1);
-        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], EPI); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], kEpiWarps); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
@@ -468,15 +454,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (ok && resident && i + 1 < walk.count && cur.m_tile + 1 == p.tiles_m) mma_commit(&ctl->bfree);
             }
         }
-    } else if (warp < 2 + EPI) {
+    } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------------ epilogue (warps 2-9)
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        const int cpart = (warp - 2) >> 2;            // which part of the tile's columns this warp takes
-        unsigned char* stg = sStage + (warp - 2) * staging_bytes(EPI);
-        float* prm_sw = sParam + (warp - 2) * 2 * (kBN / CPARTS);
-        float* prm_b = prm_sw + kBN / CPARTS;
+        const int chalf = (warp - 2) >> 2;            // which half of the tile's columns this warp takes
+        unsigned char* stg = sStage + (warp - 2) * kStagingBytes;
+        float* prm_sw = sParam + (warp - 2) * 2 * (kBN / 2);
+        float* prm_b = prm_sw + kBN / 2;
         const int cols_per_tile = limbs == 2 ? kBN / 2 : kBN;
-        const int cols_per_warp = cols_per_tile / CPARTS;
+        const int cols_per_warp = cols_per_tile / 2;
         const bool want_y = MODE == kModeFast ? true : p.y != nullptr;
         const bool want_acc = MODE == kModeFast ? false : p.acc_out != nullptr;
         bool ok = true;
@@ -490,7 +476,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int col_base = tc.n_tile * cols_per_tile;
             // This warp's columns [wc0, wc0 + cols_per_warp) of the tile; their scale_w / bias go to the warp's own
             // slice of shared memory (read back as broadcasts), so no CTA-wide barrier is needed.
-            const int wc0 = cpart * cols_per_warp;
+            const int wc0 = chalf * cols_per_warp;
             if (want_y && tc.n_tile != last_n) {       // consecutive tiles under resident weights share their columns
                 last_n = tc.n_tile;
                 __syncwarp();
@@ -611,7 +597,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 // rows of the tile are consecutive output rows (checked on the host); this warp owns 32 of them
                 const int row0 = out_row_of<CONV>(p, tc, 0) + q * 32;
                 const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
-                epilogue_fast<LIMBS_T, (LIMBS_T == 2 ? kBN / 2 : kBN) / CPARTS, staging_bytes(EPI) / 64>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
+                epilogue_fast<LIMBS_T>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
                 continue;
             }
 
@@ -707,7 +693,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // The packed tile (128 rows x 64 bytes) lands in the upper half of the 16 KB operand stage; every thread
         // first takes its share into registers, then (after a barrier of the four warps) the stage is rewritten
         // in place as 128 rows x 128 bytes with the 128-byte swizzle the MMA descriptor expects.
-        const int t = threadIdx.x - (2 + EPI) * 32;    // 0..127
+        const int t = threadIdx.x - (2 + kEpiWarps) * 32;    // 0..127
         int stage = 0; uint32_t phase = 0;
         bool ok = true;
         for (int i = 0; i < walk.count && ok; ++i) {
@@ -747,11 +733,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 
 // Launches one instantiation; the first launch per device raises its dynamic shared-memory limit.
-template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T, bool WIDE = false>
+template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T>
 cudaError_t launch_one(int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                        const CUtensorMap& tmY, const GemmParams& p) {
     static bool attr_set[64] = {};
-    auto kern = qgemm_kernel<NIBBLE, MODE, CONV, LIMBS_T, RES_T, WIDE>;
+    auto kern = qgemm_kernel<NIBBLE, MODE, CONV, LIMBS_T, RES_T>;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -760,7 +746,7 @@ cudaError_t launch_one(int grid, size_t smem, cudaStream_t st, const CUtensorMap
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<grid, cta_threads(NIBBLE, WIDE), smem, st>>>(tmA, tmB, tmY, p);
+    kern<<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
     return cudaGetLastError();
 }
 
@@ -769,13 +755,6 @@ template <bool NIBBLE, bool CONV>
 cudaError_t dispatch(int mode, int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                      const CUtensorMap& tmY, const GemmParams& p) {
     if (mode == kModeFast) {
-        if constexpr (!NIBBLE) {
-            if (p.epi_wide) {          // short reductions only, so the weights are resident
-                if (!p.b_resident) return cudaErrorInvalidValue;
-                return p.limbs == 2 ? launch_one<NIBBLE, kModeFast, CONV, 2, 1, true>(grid, smem, st, tmA, tmB, tmY, p)
-                                    : launch_one<NIBBLE, kModeFast, CONV, 1, 1, true>(grid, smem, st, tmA, tmB, tmY, p);
-            }
-        }
         if (p.limbs == 2)
             return p.b_resident ? launch_one<NIBBLE, kModeFast, CONV, 2, 1>(grid, smem, st, tmA, tmB, tmY, p)
                                 : launch_one<NIBBLE, kModeFast, CONV, 2, 0>(grid, smem, st, tmA, tmB, tmY, p);
