@@ -125,11 +125,11 @@ int sm_count() {
 }
 
 // Ring depth and weight residency for a problem; fills p.stages / p.b_resident and returns the shared-memory size.
-size_t plan_smem(GemmParams& p) {
+size_t plan_smem(GemmParams& p, bool frag) {
     const int num_kb = p.kb_per_tap * p.taps;
     p.b_resident = num_kb <= kResidentKb ? 1 : 0;
     for (int stages = kMaxStages; stages >= 2; --stages) {
-        const SmemLayout L = smem_layout(stages, p.b_resident != 0, num_kb);
+        const SmemLayout L = smem_layout(stages, p.b_resident != 0, num_kb, frag);
         if (L.total <= kSmemLimit) { p.stages = stages; return size_t(L.total); }
     }
     return 0;
@@ -137,13 +137,14 @@ size_t plan_smem(GemmParams& p) {
 
 hq_status launch(bool nibble, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY, GemmParams& p,
                  cudaStream_t st) {
-    const size_t smem = plan_smem(p);
-    if (smem == 0) return HQ_ERR_UNSUPPORTED;
-    const int tiles = p.tiles_m * p.tiles_n;
-    const int grid = tiles < sm_count() ? tiles : sm_count();
     // the kernel's fast epilogue assumes exactly these conditions
     const bool fast = p.tma_store && !p.per_tap && p.y != nullptr && p.acc_out == nullptr && p.combine_fast;
     const int mode = p.per_tap ? kModePerTap : fast ? kModeFast : kModeGeneric;
+    p.frag = use_frag(nibble, fast, p.limbs, p.kb_per_tap * p.taps) ? 1 : 0;
+    const size_t smem = plan_smem(p, p.frag != 0);
+    if (smem == 0) return HQ_ERR_UNSUPPORTED;
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
     cudaError_t e;
     if (nibble) e = p.conv ? launch_nibble_conv(mode, grid, smem, st, tmA, tmB, tmY, p)
                            : launch_nibble_gemm(mode, grid, smem, st, tmA, tmB, tmY, p);

@@ -9,7 +9,6 @@
 namespace hq {
 namespace gemm {
 
-enum : int { kModeFast = 0, kModeGeneric = 1, kModePerTap = 2 };
 
 constexpr int kBM = 128;             // rows per tile (TMEM lanes)
 constexpr int kBN = 256;             // operand-B rows per tile (TMEM columns)
@@ -24,6 +23,16 @@ constexpr int kEpiWarps = 8;            // two per TMEM lane quarter, each takin
 constexpr int kStagingBytes = 2048;          // per epilogue warp: 32 rows x 64 bytes
 constexpr int kParamBytes = kEpiWarps * 2 * (kBN / 2) * 4;   // per epilogue warp: [scale_w | bias][its columns]
 constexpr int kSmemLimit = 232448;           // 227 KB
+enum : int { kModeFast = 0, kModeGeneric = 1, kModePerTap = 2 };
+// warps: producer, MMA issuer, 8 epilogue, then 4 unpack warps (nibble container) or a second MMA issuer (fast mode
+// with one code per byte)
+__host__ __device__ constexpr int cta_threads(bool nibble, bool frag) { return nibble ? 448 : (frag ? 352 : 320); }
+// Whether the fragment-layout epilogue with its second MMA issuer is used (fast mode, one code per byte): for K_pad
+// <= 256, and for one weight limb with resident weights (K_pad <= 512).  Measured there 10-22 % faster; with two limbs
+// and K_pad >= 512 it is level, and with streamed weights 2-4 % slower on most shapes.
+inline bool use_frag(bool nibble, bool fast, int limbs, int num_kb) {
+    return !nibble && fast && (num_kb <= 2 || (limbs == 1 && num_kb <= kResidentKb));
+}
 
 struct GemmParams {
     int64_t M;            // GEMM rows (unused for conv)
@@ -47,12 +56,14 @@ struct GemmParams {
     int y_vec_ok, acc_vec_ok;
     int per_tap;          // convolution with one activation scale per input pixel: the accumulator is drained per filter tap
     int col_pass;         // per_tap with one weight limb: which 64 of a warp's 128 columns this launch produces
+    int frag;             // fragment-layout epilogue + second MMA issuer (see use_frag)
     int tma_store;        // bf16 output goes out through bulk tensor stores (rows of a tile are consecutive output rows)
     int32_t* dev_status;
 };
 
 struct SharedCtl {
     uint64_t full[kMaxStages];
+    uint64_t full2[kMaxStages];       // the same stages when filled for the second MMA issuer (see the kernel)
     uint64_t empty[kMaxStages];
     uint64_t rawread[kMaxStages];     // all unpack threads hold their share of the packed tile in registers
     uint64_t unpacked[kMaxStages];
@@ -66,13 +77,14 @@ struct SharedCtl {
 
 // Shared-memory carve-up (all offsets from a 1024-byte aligned base).
 struct SmemLayout { int b_off, a_off, staging_off, param_off, ctl_off, total; };
-__host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int num_kb) {
+// `frag`: the fragment-layout fast epilogue (two staging buffers per warp, column parameters in registers).
+__host__ __device__ inline SmemLayout smem_layout(int stages, bool resident, int num_kb, bool frag) {
     SmemLayout L;
     L.b_off = 0;
     L.a_off = (resident ? num_kb : stages) * kBBytes;
     L.staging_off = L.a_off + stages * kABytes;
-    L.param_off = L.staging_off + kEpiWarps * kStagingBytes;
-    L.ctl_off = L.param_off + kParamBytes;
+    L.param_off = L.staging_off + kEpiWarps * kStagingBytes * (frag ? 2 : 1);
+    L.ctl_off = L.param_off + (frag ? 0 : kParamBytes);
     L.total = L.ctl_off + int(sizeof(SharedCtl)) + 1024;      // + slack for the base alignment
     return L;
 }
@@ -308,6 +320,135 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
     }
 }
 
+// Epilogue warp of the fast output mode with accumulators read in the 16x256b fragment layout: a lane holds, for its
+// four rows (lane/4 + 8 j of the warp's 32), the column pairs 8 n + 2 (lane%4) + {0, 1}.  So the scale_w / bias of a
+// lane's columns are 1/4 of the warp's and stay in registers while the weight tile stays (no shared-memory reads at
+// all), and a bf16 pair goes to the staging buffer as one 32-bit store that is free of bank conflicts in the 64-byte
+// swizzle of the output tensor map.  The shared-memory data pipe, which also feeds the tensor core its operands, is
+// the busiest unit of this kernel: with row-per-lane loads the broadcast reads of the column parameters and the 16-byte
+// staging stores took more of it than the MMAs themselves.
+// Per 32 columns: four TMEM loads (two 16-lane slabs x two limbs), recombination, rescale, 16 stores, one bulk store.
+template <bool CONV, int LIMBS>
+__device__ __forceinline__ void fast_epilogue_warp(const GemmParams& p, const TileCursor& walk, bool resident,
+                                                   SharedCtl* ctl, uint32_t tmem_base, unsigned char* stg,
+                                                   const CUtensorMap* tmY, int warp, int lane) {
+    constexpr int CPT = LIMBS == 2 ? kBN / 2 : kBN;      // output columns per tile
+    constexpr int CPW = CPT / 2;                         // ... per warp
+    constexpr int NCH = CPW / 32;                        // 32-column chunks: one staging buffer and one bulk store each
+    const int q = warp & 3;                              // TMEM lane quarter this warp may read
+    const int wc0 = ((warp - 2) >> 2) * CPW;             // first column (in the tile) of this warp
+    const int tq = lane & 3, tr = lane >> 2;
+    const uint32_t rsw = uint32_t(tr >> 1) & 3u;         // swizzle term of this lane's staging rows (same for all four)
+    const int64_t total_rows = CONV ? int64_t(p.Nb) * p.Ho * p.Wo : p.M;
+    const float a_eff = p.alpha / float(1 << p.a_shift); // the accumulators carry the container's shift
+    float sw[CPW / 4], bb[CPW / 4];
+    float sa[4] = {0.f, 0.f, 0.f, 0.f};
+    TileCursor cur = walk;
+    int last_n = -1;
+    for (int i = 0; i < walk.count; ++i, tile_next(p, cur, resident)) {
+        const int as = i & 1;
+        const TileCoord tc = tile_coord<CONV>(p, cur);
+        const int col_base = tc.n_tile * CPT + wc0;
+        if (tc.n_tile != last_n) {                       // consecutive tiles under resident weights share their columns
+            last_n = tc.n_tile;
+#pragma unroll
+            for (int c = 0; c < CPW / 4; ++c) {
+                const int col = col_base + 8 * (c >> 1) + 2 * tq + (c & 1);
+                sw[c] = col < p.N ? __ldg(p.scale_w + col) : 0.f;
+                bb[c] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
+            }
+        }
+        // rows of the tile are consecutive output rows (checked on the host); this warp owns 32 of them
+        const int row0 = out_row_of<CONV>(p, tc, 0) + q * 32;
+        if (i == 0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t row = int64_t(row0) + tr + 8 * j;
+                sa[j] = p.sa_scalar ? __ldg(p.scale_a) : (row < total_rows ? __ldg(p.scale_a + row) : 0.f);
+            }
+        }
+        int row0_next = -1;
+        if (i + 1 < walk.count && !p.sa_scalar) {
+            TileCursor nx = cur;
+            tile_next(p, nx, resident);
+            row0_next = out_row_of<CONV>(p, tile_coord<CONV>(p, nx), 0) + q * 32;
+        }
+        if (!wait_or_abort(&ctl->tfull[as], uint32_t(i >> 1) & 1u, ctl, p.dev_status, kStatusAccumWait)) break;
+        tc_fence_after();
+        float sa_eff[4], sa_nx[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            sa_eff[j] = a_eff * sa[j];
+            sa_nx[j] = sa[j];
+            if (row0_next >= 0) {                        // the next tile's row scales fly while this tile is processed
+                const int64_t row = int64_t(row0_next) + tr + 8 * j;
+                sa_nx[j] = row < total_rows ? __ldg(p.scale_a + row) : 0.f;
+            }
+        }
+        const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
+        const uint32_t t1 = t0 + (16u << 16);            // the second 16-lane slab
+        uint32_t h0[16], h1[16], l0[16], l1[16];
+        tmem_ld_16x256_x4(t0, h0);
+        tmem_ld_16x256_x4(t1, h1);
+        if (LIMBS == 2) { tmem_ld_16x256_x4(t0 + uint32_t(kBN / 2), l0); tmem_ld_16x256_x4(t1 + uint32_t(kBN / 2), l1); }
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            float f0[16], f1[16];
+            tmem_ld_wait_16(h0);
+            tmem_ld_wait_16(h1);
+            if (LIMBS == 2) {
+                tmem_ld_wait_16(l0);
+                tmem_ld_wait_16(l1);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    f0[e] = float(int32_t(h0[e]) * 256 + int32_t(l0[e]));
+                    f1[e] = float(int32_t(h1[e]) * 256 + int32_t(l1[e]));
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) { f0[e] = float(int32_t(h0[e])); f1[e] = float(int32_t(h1[e])); }
+            }
+            if (ch + 1 < NCH) {                          // the next chunk's loads fly while this one is processed
+                const uint32_t c = uint32_t((ch + 1) * 32);
+                tmem_ld_16x256_x4(t0 + c, h0);
+                tmem_ld_16x256_x4(t1 + c, h1);
+                if (LIMBS == 2) { tmem_ld_16x256_x4(t0 + c + uint32_t(kBN / 2), l0); tmem_ld_16x256_x4(t1 + c + uint32_t(kBN / 2), l1); }
+            } else {                                     // accumulator fully read: hand it back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->tempty[as]);
+            }
+            // two staging buffers, used in turn: the copy engine must be done reading the one written two chunks ago
+            unsigned char* buf = stg + ((i * NCH + ch) & 1) * kStagingBytes;
+            if (lane == 0) bulk_wait_read_1();
+            __syncwarp();
+#pragma unroll
+            for (int n = 0; n < 4; ++n) {
+                const int c = 2 * (ch * 4 + n);          // index of this repeat's column pair in sw / bb
+                unsigned char* wr = buf + tr * 64 + ((uint32_t(n) ^ rsw) << 4) + 4 * tq;
+                // slab 0: rows tr, tr + 8; slab 1: rows tr + 16, tr + 24
+                *reinterpret_cast<uint32_t*>(wr) = pack_bf16x2(fmaf(f0[4 * n + 0] * sw[c], sa_eff[0], bb[c]),
+                                                               fmaf(f0[4 * n + 1] * sw[c + 1], sa_eff[0], bb[c + 1]));
+                *reinterpret_cast<uint32_t*>(wr + 8 * 64) = pack_bf16x2(fmaf(f0[4 * n + 2] * sw[c], sa_eff[1], bb[c]),
+                                                                        fmaf(f0[4 * n + 3] * sw[c + 1], sa_eff[1], bb[c + 1]));
+                *reinterpret_cast<uint32_t*>(wr + 16 * 64) = pack_bf16x2(fmaf(f1[4 * n + 0] * sw[c], sa_eff[2], bb[c]),
+                                                                         fmaf(f1[4 * n + 1] * sw[c + 1], sa_eff[2], bb[c + 1]));
+                *reinterpret_cast<uint32_t*>(wr + 24 * 64) = pack_bf16x2(fmaf(f1[4 * n + 2] * sw[c], sa_eff[3], bb[c]),
+                                                                         fmaf(f1[4 * n + 3] * sw[c + 1], sa_eff[3], bb[c + 1]));
+            }
+            fence_proxy_async_smem();                    // the lanes' writes become visible to the copy engine
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(tmY, buf, col_base + ch * 32, row0);
+                bulk_commit_group();
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sa[j] = sa_nx[j];
+    }
+    if (lane == 0) bulk_wait_read_all();                 // shared memory must outlive the copy engine's reads
+}
+
 // The kernel is compiled once per combination of
 //   NIBBLE   container of the activation codes (the nibble container adds the four unpack warps),
 //   MODE     kModeFast: bf16 output through bulk tensor stores, limbs recombined as 256*hi + lo without overflow (the
@@ -316,19 +457,24 @@ __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg
 //   CONV     implicit-GEMM convolution (4-D activation boxes, pixel geometry) or plain GEMM,
 //   LIMBS_T  weight limbs (1 or 2), or 0 = read at run time,
 //   RES_T    weights resident (1) / streamed (0), or -1 = read at run time,
+//   FRAG     fragment-layout epilogue and a second MMA issuer (fast mode with one code per byte only; see use_frag),
 // because the hot loop of each role is short and runs once per tile: run-time branches over these choices and the
 // code of the paths not taken cost 10-15 % on the K <= 512 shapes (instruction fetch and bookkeeping per tile).
-template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T>
-__global__ void __launch_bounds__(NIBBLE ? 448 : 320, 1)
+template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T, bool FRAG>
+__global__ void __launch_bounds__(cta_threads(NIBBLE, FRAG), 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmY, const GemmParams p) {
     constexpr bool PERTAP = MODE == kModePerTap;
+    static_assert(!FRAG || (MODE == kModeFast && !NIBBLE), "the fragment-layout epilogue exists for the fast mode with one code per byte");
+    // MMA-issuing warps: two (warp 1 and the CTA's last warp) together with the fragment-layout epilogue, else one
+    constexpr int ISSUERS = FRAG ? 2 : 1;
+    constexpr int kIssuer2 = 2 + kEpiWarps;
     const int limbs = LIMBS_T != 0 ? LIMBS_T : p.limbs;
     const bool resident = RES_T >= 0 ? (RES_T != 0) : (p.b_resident != 0);
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int num_kb = p.kb_per_tap * p.taps;
-    const SmemLayout L = smem_layout(p.stages, resident, num_kb);
+    const SmemLayout L = smem_layout(p.stages, resident, num_kb, FRAG);
     unsigned char* sB = smem + L.b_off;
     unsigned char* sA = smem + L.a_off;
     unsigned char* sStage = smem + L.staging_off;
@@ -342,12 +488,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->full2[s], 1);
             mbar_init(&ctl->empty[s], 1);
             mbar_init(&ctl->rawread[s], 128);
             mbar_init(&ctl->unpacked[s], 128);
         }
         for (int k = 0; k < kResidentKb; ++k) mbar_init(&ctl->bfull[k], 1);
-        mbar_init(&ctl->bfree, 1);
+        mbar_init(&ctl->bfree, ISSUERS);
         for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], kEpiWarps); }
         ctl->abort_flag = 0;
         fence_barrier_init();
@@ -367,6 +514,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             int stage = 0; uint32_t phase = 0;
             int cur_n = -1, reloads = 0;
             long long armed = 0;
+            uint32_t par_a = 0, par_b = 0;     // per stage: parity of the next phase of full[] / full2[]
+            uint32_t last_fill = 0;            // per stage: which of the two barriers its latest fill was armed on
             bool ok = true;
             TileCursor cur = walk;
             for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur, resident)) {
@@ -383,18 +532,22 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 }
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_or_abort(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
-                    mbar_expect_tx(&ctl->full[stage], p.a_box_bytes + (resident ? 0u : uint32_t(kBBytes)));
+                    // the stage's arrival is signalled on the barrier of the issuer that takes this tile
+                    uint64_t* fbar = (ISSUERS == 2 && (i & 1)) ? &ctl->full2[stage] : &ctl->full[stage];
+                    if (ISSUERS == 2 && (i & 1)) { last_fill |= 1u << stage; par_b ^= 1u << stage; }
+                    else { last_fill &= ~(1u << stage); par_a ^= 1u << stage; }
+                    mbar_expect_tx(fbar, p.a_box_bytes + (resident ? 0u : uint32_t(kBBytes)));
                     unsigned char* a_dst = sA + stage * kABytes + (NIBBLE ? kABytes - kRawBytes : 0);
                     const int a_k = (NIBBLE ? kBK / 2 : kBK);
                     if (CONV) {
                         const int tap = kb / p.kb_per_tap, kc = kb - tap * p.kb_per_tap;
                         const int r = tap / p.S, s = tap - r * p.S;
-                        tma_load_4d(a_dst, &tmA, &ctl->full[stage], kc * a_k, tc.w0 * p.stride + s - p.pad,
+                        tma_load_4d(a_dst, &tmA, fbar, kc * a_k, tc.w0 * p.stride + s - p.pad,
                                     tc.h0 * p.stride + r - p.pad, tc.n0);
                     } else {
-                        tma_load_2d(a_dst, &tmA, &ctl->full[stage], kb * a_k, tc.m_tile * kBM);
+                        tma_load_2d(a_dst, &tmA, fbar, kb * a_k, tc.m_tile * kBM);
                     }
-                    if (!resident) tma_load_2d(sB + stage * kBBytes, &tmB, &ctl->full[stage], kb * kBK, tc.n_tile * kBN);
+                    if (!resident) tma_load_2d(sB + stage * kBBytes, &tmB, fbar, kb * kBK, tc.n_tile * kBN);
                     ++armed;
                     if (++stage == nstages) { stage = 0; phase ^= 1; }
                 }
@@ -405,18 +558,28 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     for (int kb = 0; kb < num_kb; ++kb) mbar_wait(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, nullptr, 0);
                 const int back = armed < nstages ? int(armed) : nstages;
                 for (int j = 0; j < back; ++j) {
-                    if (--stage < 0) { stage = nstages - 1; phase ^= 1; }
-                    mbar_wait(&ctl->full[stage], phase, nullptr, 0);
+                    if (--stage < 0) stage = nstages - 1;
+                    const bool second = (last_fill >> stage) & 1u;
+                    const uint32_t armed_parity = (((second ? par_b : par_a) >> stage) & 1u) ^ 1u;   // the phase armed last
+                    mbar_wait(second ? &ctl->full2[stage] : &ctl->full[stage], armed_parity, nullptr, 0);
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || (ISSUERS == 2 && warp == kIssuer2)) {
+        // ------------------------------------------------------------------ MMA issuer(s)
+        // One lane needs about as long to get a K block issued (barrier wait, fence, four MMAs, commit) as the tensor
+        // pipe needs to run it, so with a single issuer every wait at a tile change leaves the pipe idle.  With two,
+        // warp 1 takes the even tiles (accumulator 0) and the CTA's last warp the odd ones (accumulator 1).  They share
+        // the ring of operand stages; the producer signals a stage on full[] or full2[] according to the tile it
+        // belongs to, so each barrier has one waiter who sees all of its phases in order.
         if (lane == 0) {
+            const int me = warp == 1 ? 0 : 1;
+            uint64_t* fullbar = me ? ctl->full2 : ctl->full;
             const uint32_t idesc = make_idesc_i8(kBM, kBN);
-            int stage = 0; uint32_t phase = 0;
+            int stage = 0; uint32_t phase = 0;            // position in the ring (phase: the unpack barriers' parity)
+            uint32_t par = 0;                             // per stage: parity of the next phase of this issuer's barrier
             int cur_n = -1, reloads = 0;
-            bool ok = true;
+            bool ok = true, pending_b = false;
             TileCursor cur = walk;
             // One accumulator per tile, or (per-tap mode) one per filter tap of a tile; they alternate between the
             // two TMEM buffers in the order they are produced.
@@ -424,36 +587,58 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int kb_per_group = num_kb / groups;
             int seq = 0;
             for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur, resident)) {
-                const bool new_b = resident && cur.n_tile != cur_n;
-                if (new_b) { cur_n = cur.n_tile; ++reloads; }
-                for (int g = 0; g < groups && ok; ++g, ++seq) {
-                    const int as = seq & 1;
-                    const uint32_t aphase = (seq >> 1) & 1;
-                    if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
-                    for (int kk = 0; kk < kb_per_group; ++kk) {
-                        const int kb = g * kb_per_group + kk;
-                        if (new_b && !wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                        if (!wait_or_abort(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
-                        if (NIBBLE) {
-                            if (!wait_or_abort(&ctl->unpacked[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
-                        }
-                        tc_fence_after();
-                        const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
-                        const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + (resident ? kb : stage) * kBBytes));
-#pragma unroll
-                        for (int k = 0; k < kBK / 32; ++k)
-                            mma_i8(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kk | k) != 0 ? 1u : 0u);
-                        mma_commit(&ctl->empty[stage]);
-                        if (++stage == nstages) { stage = 0; phase ^= 1; }
+                if (resident && cur.n_tile != cur_n) { cur_n = cur.n_tile; ++reloads; pending_b = true; }
+                const bool mine = ISSUERS == 1 || (i & 1) == me;
+                if (!mine) {
+                    // The other issuer's tile: step over its stages.  New weights are waited for here all the same, so
+                    // that this lane sees every phase of the weight barriers (a parity wait cannot tell phase r from r+2).
+                    if (pending_b) {
+                        for (int kb = 0; kb < num_kb && ok; ++kb)
+                            if (!wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) ok = false;
+                        pending_b = false;
                     }
-                    if (ok) mma_commit(&ctl->tfull[as]);
+                    stage += num_kb;
+                    while (stage >= nstages) { stage -= nstages; phase ^= 1; }
+                } else {
+                    const bool new_b = pending_b;          // first use of these weights: wait per K block before its MMAs
+                    pending_b = false;
+                    for (int g = 0; g < groups && ok; ++g, ++seq) {
+                        const int as = ISSUERS == 2 ? me : (seq & 1);
+                        const uint32_t aphase = ISSUERS == 2 ? uint32_t(i >> 1) & 1u : uint32_t(seq >> 1) & 1u;
+                        if (!wait_or_abort(&ctl->tempty[as], aphase ^ 1, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                        for (int kk = 0; kk < kb_per_group; ++kk) {
+                            const int kb = g * kb_per_group + kk;
+                            if (new_b && !wait_or_abort(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                            if (!wait_or_abort(&fullbar[stage], (par >> stage) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                            par ^= 1u << stage;
+                            if (NIBBLE) {
+                                if (!wait_or_abort(&ctl->unpacked[stage], phase, ctl, p.dev_status, kStatusUnpackWait)) { ok = false; break; }
+                            }
+                            tc_fence_after();
+                            const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
+                            const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + (resident ? kb : stage) * kBBytes));
+#pragma unroll
+                            for (int k = 0; k < kBK / 32; ++k)
+                                mma_i8(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kk | k) != 0 ? 1u : 0u);
+                            mma_commit(&ctl->empty[stage]);
+                            if (++stage == nstages) { stage = 0; phase ^= 1; }
+                        }
+                        if (ok) mma_commit(&ctl->tfull[as]);
+                    }
                 }
-                // the next tile of the range starts a new weight tile: tell the producer when this one is done with
+                // The next tile of the range starts a new weight tile: tell the producer when this issuer's MMAs on the
+                // old one are done (the barrier counts one arrival per issuer; an issuer with nothing in flight
+                // arrives at once).
                 if (ok && resident && i + 1 < walk.count && cur.m_tile + 1 == p.tiles_m) mma_commit(&ctl->bfree);
             }
         }
+    } else if (FRAG && warp < 2 + kEpiWarps) {
+        // ------------------------------------------------------------------ epilogue (warps 2-9), fragment layout
+        if constexpr (FRAG)
+            fast_epilogue_warp<CONV, LIMBS_T>(p, walk, resident, ctl, tmem_base, sStage + (warp - 2) * 2 * kStagingBytes, &tmY,
+                                              warp, lane);
     } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------------ epilogue (warps 2-9)
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
@@ -733,11 +918,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 
 // Launches one instantiation; the first launch per device raises its dynamic shared-memory limit.
-template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T>
+template <bool NIBBLE, int MODE, bool CONV, int LIMBS_T, int RES_T, bool FRAG = false>
 cudaError_t launch_one(int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                        const CUtensorMap& tmY, const GemmParams& p) {
     static bool attr_set[64] = {};
-    auto kern = qgemm_kernel<NIBBLE, MODE, CONV, LIMBS_T, RES_T>;
+    auto kern = qgemm_kernel<NIBBLE, MODE, CONV, LIMBS_T, RES_T, FRAG>;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -746,7 +931,7 @@ cudaError_t launch_one(int grid, size_t smem, cudaStream_t st, const CUtensorMap
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<grid, NIBBLE ? 448 : 320, smem, st>>>(tmA, tmB, tmY, p);
+    kern<<<grid, cta_threads(NIBBLE, FRAG), smem, st>>>(tmA, tmB, tmY, p);
     return cudaGetLastError();
 }
 
@@ -755,6 +940,13 @@ template <bool NIBBLE, bool CONV>
 cudaError_t dispatch(int mode, int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                      const CUtensorMap& tmY, const GemmParams& p) {
     if (mode == kModeFast) {
+        if constexpr (!NIBBLE) {
+            if (p.frag) {
+                if (!p.b_resident) return cudaErrorInvalidValue;       // chosen for resident weights only
+                return p.limbs == 1 ? launch_one<NIBBLE, kModeFast, CONV, 1, 1, true>(grid, smem, st, tmA, tmB, tmY, p)
+                                    : launch_one<NIBBLE, kModeFast, CONV, 2, 1, true>(grid, smem, st, tmA, tmB, tmY, p);
+            }
+        }
         if (p.limbs == 2)
             return p.b_resident ? launch_one<NIBBLE, kModeFast, CONV, 2, 1>(grid, smem, st, tmA, tmB, tmY, p)
                                 : launch_one<NIBBLE, kModeFast, CONV, 2, 0>(grid, smem, st, tmA, tmB, tmY, p);
