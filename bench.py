@@ -51,9 +51,9 @@ def codes_name():
 # capture of this command (a summary is kept under profiles/; taken with these kernel versions: set an entry to
 # None when its kernel changes).  Outputs partly stay in L2 past the end of a launch, so these are below the
 # algorithmic bytes.
-NCU_DRAM_CODES = 0      # container the counters below were taken with (0 = nibble)
-NCU_DRAM_BYTES = {"gemm": {"qkv": 54.2e6, "ff1": 88.8e6, "ff2": 36.0e6, "conv3x3": 5.4e6, "out_proj": None},
-                  "quant": {"qkv": 67.5e6, "out_proj": 67.5e6, "ff1": 67.5e6, "ff2": 275.1e6, "conv3x3": None}}
+NCU_DRAM_CODES = 1      # container the counters below were taken with (1 = one code per byte)
+NCU_DRAM_BYTES = {"gemm": {"qkv": 66.2e6, "ff1": 100.7e6, "ff2": 73.4e6, "conv3x3": 9.6e6, "out_proj": 17.5e6},
+                  "quant": {"qkv": 67.3e6, "out_proj": 67.2e6, "ff1": 68.7e6, "ff2": 278.2e6, "conv3x3": 33.6e6}}
 
 
 def layer_list():
