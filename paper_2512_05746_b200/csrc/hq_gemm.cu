@@ -3,16 +3,10 @@
 //   acc[m][o] = sum_k a[m][k] * B[o][k]   int8 x int8 -> int32 on the 5th-generation tensor cores
 //   y[m][o]   = alpha * S_a[m] * S_w[o] * acc[m][o] + bias[o]
 //
-// One persistent CTA per SM walks output tiles of 128 rows x 256 operand rows (256 output channels with
-// one weight limb, 128 with two).  Roles:
-//   warp 0      TMA producer: activation tile (2-D box for a GEMM, 4-D NHWC box per filter tap for a
-//               convolution, out-of-bounds = zero padding) and weight tile
-//   warp 1      issues tcgen05.mma.kind::i8 (128x256x32) into one of two 256-column TMEM accumulators
-//   warps 2-5   epilogue: tcgen05.ld, limb recombination (256*hi + lo), rescale, and row-contiguous 16-byte stores
-//               through a small swizzled staging buffer; runs on accumulator t while the MMA warp fills t+1
-//   warps 6-9   (NIBBLE container only) unpack 4-bit codes from a raw TMA tile into the swizzled int8 operand
-//               tile.  A code q is written as the byte q<<4 (= 16q, no sign extension needed), so the accumulator
-//               is 16x the true one; the factor is removed exactly in the epilogue.
+// Host side: argument checks, tensor maps, shared-memory planning and the choice of kernel instantiation.  The kernel
+// itself (one persistent CTA per SM walking output tiles of 128 rows x 256 operand rows, warp-specialised into a TMA
+// producer, one or two MMA issuers, eight epilogue warps and, for the nibble container, four unpack warps) is in
+// hq_gemm_kernel.cuh; hq_gemm_inst_*.cu instantiate it per container and problem kind.
 // Weights: when the whole reduction fits (K_pad <= 512 bytes per operand row, 128 KB per tile) the weight tile
 // stays resident in shared memory and the CTA walks a contiguous range of row tiles under it (only activations
 // stream); otherwise weights stream through the same ring as the activations.
