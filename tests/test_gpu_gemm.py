@@ -43,6 +43,9 @@ def gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, conta
     hq.hq_qgemm(a_dev, container, a_bits, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, acc_out=acc, y=y16,
                 dev_status=status)
     hq.hq_qgemm(a_dev, container, a_bits, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y32, dev_status=status)
+    # bf16 output alone: the launch configuration the layers and the benchmark use (bulk-store epilogue)
+    y16_only = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    hq.hq_qgemm(a_dev, container, a_bits, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y16_only, dev_status=status)
     torch.cuda.synchronize()
     hq.hq_check_status(status)
     acc_ref = oracle.gemm_int(q, B_ref)
@@ -50,6 +53,7 @@ def gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, conta
     y_ref = oracle.dequant(acc_ref, s_a, pw.s_w, b, pw.alpha)
     assert rel_err(y32.cpu().numpy(), y_ref) <= Y_F32_RTOL
     assert rel_err(y16.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+    assert rel_err(y16_only.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
     return pw
 
 
@@ -68,6 +72,12 @@ GEMM_CASES = [
     (4096, 1024, 1280, 4, 4, 1024, "folded", 0),  # several tiles per CTA
     (64, 4096, 256, 4, 4, 4096, "folded", 1),
     (1, 256, 256, 4, 4, 256, "double", 0),
+    # one code per byte with short reductions / one resident limb: the fragment-layout epilogue and its second issuer
+    (1000, 256, 200, 4, 4, 256, "folded", 1),     # two limbs, K = 2 blocks, ragged M, N = 1.56 tiles
+    (777, 512, 328, 4, 4, 512, "plain", 1),       # one limb, resident weights, several weight tiles per CTA range
+    (130, 128, 72, 4, 4, 128, "folded", 1),       # K = 1 block
+    (40000, 256, 384, 4, 4, 256, "double", 1),    # many tiles per CTA, weight tile changes inside a CTA's range
+    (5000, 1152, 136, 4, 4, 128, "plain", 1),     # one limb with streamed weights (row-per-lane epilogue)
 ]
 
 
@@ -135,6 +145,8 @@ CONV_CASES = [
     (1, 20, 12, 128, 64, 3, 1, 4, "plain", 1),       # width that does not divide 128
     (2, 16, 16, 256, 256, 1, 0, 4, "folded", 0),     # 1x1
     (1, 10, 10, 160, 96, 3, 0, 4, "plain", 1),       # no padding, channel tail (160 = 1.25 blocks)
+    (4, 16, 16, 256, 320, 1, 0, 4, "folded", 1),     # 1x1, K = 2 blocks: fragment-layout epilogue on a convolution
+    (5, 8, 8, 384, 200, 1, 0, 4, "plain", 1),        # 1x1, one limb, tiles span two images, last tile partly empty
 ]
 
 
@@ -160,6 +172,13 @@ def test_qconv2d_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, a_bits, 
     assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
     y_ref = oracle.dequant(acc_ref, np.array([0.05], np.float32), pw.s_w, b, pw.alpha)
     assert rel_err(y.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+    # bf16 output alone: the launch configuration the layers and the benchmark use
+    y2 = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
+    hq.hq_qconv2d(to_container(torch, hq, q, container), container, a_bits, Nb, H, W, C, pw, R, R, 1, pad, scale_a=s_a,
+                  bias=torch.from_numpy(b).cuda(), alpha=pw.alpha, y=y2, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    assert rel_err(y2.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
 
 
 STRIDE2_CASES = [
