@@ -15,11 +15,12 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
 hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64_t M, int64_t K, int64_t lda,
                        const hq_weight_desc* desc, const void* w_dev, const float* scale_a, int scale_a_is_scalar,
                        const float* scale_w, const float* bias, float alpha, int32_t* acc_out, void* y,
-                       hq_dtype ydt, int64_t ldy, int32_t* dev_status, cudaStream_t st);
+                       hq_dtype ydt, int64_t ldy, int32_t* dev_status, cudaStream_t st, bool after_quant);
 hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
                          int64_t C, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
                          const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias,
-                         float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st);
+                         float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st,
+                         bool after_quant);
 
 hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                       int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
@@ -87,7 +88,7 @@ extern "C" hq_status hq_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t 
     s = launch_hadamard_quant(x, xdt, M, K, ldx, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
     if (s != HQ_OK) return s;
     return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, mode == HQ_SCALE_STATIC, scale_w, bias,
-                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st);
+                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st, true);
 }
 
 extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
@@ -112,7 +113,7 @@ extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H
     s = launch_hadamard_quant(x, xdt, rows, C, C, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
-                          mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st);
+                          mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st, true);
 }
 
 // Convolution exactly as Eq. 13-14 state it: transform along the width axis, quantization with one static scale,
@@ -140,7 +141,7 @@ extern "C" hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int
     if (s != HQ_OK) return s;
     // |z| <= 128: the accumulator bound is that of 8-bit codes; the 2^(-k/2) is already inside `scale`
     return launch_qconv2d(z, HQ_CODES_INT8, 8, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale, 1, scale_w, bias, 1.0f,
-                          nullptr, y, ydt, dev_status, st);
+                          nullptr, y, ydt, dev_status, st, true);
 }
 
 namespace hq {
@@ -187,5 +188,5 @@ extern "C" hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, 
     s = launch_hadamard_quant(x, xdt, M, K, ldx, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
     if (s != HQ_OK) return s;
     return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, mode == HQ_SCALE_STATIC, scale_w, bias,
-                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st);
+                        hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st, true);
 }

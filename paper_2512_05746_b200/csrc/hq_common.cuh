@@ -100,6 +100,12 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, const void* smem_
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the bulk stores committed by this thread have finished READING shared memory (not writing global).
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start while the
+// kernel before it in the stream is still running; griddep_wait() then blocks until that kernel has completed and its
+// writes are visible (a no-op for a normally launched kernel).  griddep_launch() in the earlier kernel lets the later
+// one be scheduled once every CTA has called it or exited.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 // at most one bulk store group of this thread may still be reading shared memory
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }

@@ -187,7 +187,7 @@ hq_status check_common(const void* a_codes, hq_container cont, int a_bits, const
 hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64_t M, int64_t K, int64_t lda,
                        const hq_weight_desc* desc, const void* w_dev, const float* scale_a, int scale_a_is_scalar,
                        const float* scale_w, const float* bias, float alpha, int32_t* acc_out, void* y,
-                       hq_dtype ydt, int64_t ldy, int32_t* dev_status, cudaStream_t st) {
+                       hq_dtype ydt, int64_t ldy, int32_t* dev_status, cudaStream_t st, bool after_quant) {
     hq_status s = check_common(a_codes, cont, a_bits, desc, w_dev, scale_a, scale_w, acc_out, y, ydt, K);
     if (s != HQ_OK) return s;
     if (desc->RS != 1 || desc->C != K) return HQ_ERR_SHAPE;
@@ -206,6 +206,7 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     p.tiles_n = int(desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
     p.a_box_bytes = cont == HQ_CODES_NIBBLE ? kRawBytes : kABytes;
     p.conv = 0;
+    p.pdl = after_quant ? 1 : 0;
     fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
                   dev_status);
 
@@ -224,7 +225,8 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
 hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
                          int64_t C, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
                          const float* scale_a, int scale_a_is_scalar, const float* scale_w, const float* bias,
-                         float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st) {
+                         float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st,
+                         bool after_quant) {
     hq_status s = check_common(a_codes, cont, a_bits, desc, w_dev, scale_a, scale_w, acc_out, y, ydt,
                                int64_t(R) * S * C);
     if (s != HQ_OK) return s;
@@ -243,7 +245,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     if (per_tap && acc_out != nullptr) {
         // the whole-window integer sums never exist in that mode: produce them with a launch of their own
         s = launch_qconv2d(a_codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, nullptr, 1, nullptr,
-                           nullptr, 1.0f, acc_out, nullptr, ydt, dev_status, st);
+                           nullptr, 1.0f, acc_out, nullptr, ydt, dev_status, st, after_quant);
         if (s != HQ_OK) return s;
         acc_out = nullptr;
     }
@@ -251,6 +253,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     GemmParams p{};
     p.N = int(desc->N); p.limbs = desc->limbs;
     p.kb_per_tap = int(desc->C_pad / kBK); p.taps = R * S;
+    p.pdl = (after_quant && !per_tap) ? 1 : 0;       // a per-tap layer may take several launches: keep those plain
     p.conv = 1; p.Nb = int(Nb); p.H = int(H); p.W = int(W); p.Ho = int(Ho); p.Wo = int(Wo);
     p.R = R; p.S = S; p.stride = stride; p.pad = pad;
     p.bw = int(Wo < kBM ? Wo : kBM);
@@ -300,7 +303,7 @@ extern "C" hq_status hq_qgemm(const void* a_codes, hq_container cont, int a_bits
                               int32_t* acc_out, void* y, hq_dtype ydt, int64_t ldy, int32_t* dev_status,
                               void* stream) {
     return hq::launch_qgemm(a_codes, cont, a_bits, M, K, lda, desc, w_dev, scale_a, scale_a_is_scalar, scale_w, bias,
-                            alpha, acc_out, y, ydt, ldy, dev_status, static_cast<cudaStream_t>(stream));
+                            alpha, acc_out, y, ydt, ldy, dev_status, static_cast<cudaStream_t>(stream), false);
 }
 
 extern "C" hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t Nb, int64_t H, int64_t W,
@@ -310,7 +313,7 @@ extern "C" hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bi
                                 int32_t* dev_status, void* stream) {
     return hq::launch_qconv2d(a_codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale_a,
                               scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, dev_status,
-                              static_cast<cudaStream_t>(stream));
+                              static_cast<cudaStream_t>(stream), false);
 }
 
 extern "C" hq_status hq_mma_i8_probe(int ctas, int iters, int32_t* dev_status, void* stream) {

@@ -56,6 +56,7 @@ struct GemmParams {
     int y_vec_ok, acc_vec_ok;
     int per_tap;          // convolution with one activation scale per input pixel: the accumulator is drained per filter tap
     int col_pass;         // per_tap with one weight limb: which 64 of a warp's 128 columns this launch produces
+    int pdl;              // launched ahead of the completion of the kernel that produces the codes and scale_a
     int frag;             // fragment-layout epilogue + second MMA issuer (see use_frag)
     int tma_store;        // bf16 output goes out through bulk tensor stores (rows of a tile are consecutive output rows)
     int32_t* dev_status;
@@ -343,6 +344,7 @@ __device__ __forceinline__ void fast_epilogue_warp(const GemmParams& p, const Ti
     const float a_eff = p.alpha / float(1 << p.a_shift); // the accumulators carry the container's shift
     float sw[CPW / 4], bb[CPW / 4];
     float sa[4] = {0.f, 0.f, 0.f, 0.f};
+    griddep_wait();                                      // scale_a comes from the kernel before this one
     TileCursor cur = walk;
     int last_n = -1;
     for (int i = 0; i < walk.count; ++i, tile_next(p, cur, resident)) {
@@ -530,6 +532,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     }
                     cur_n = tc.n_tile; ++reloads;
                 }
+                // Weights do not depend on the kernel before this one, activation codes do: with a programmatic
+                // dependent launch the first weight tile is on its way while that kernel finishes.
+                if (i == 0) griddep_wait();
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_or_abort(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
                     // the stage's arrival is signalled on the barrier of the issuer that takes this tile
@@ -654,6 +659,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         TileCursor cur = walk;
         int last_n = -1;
         float sa_next = 0.f;
+        griddep_wait();                               // scale_a comes from the kernel before this one
         for (int i = 0; i < walk.count && ok; ++i, tile_next(p, cur, resident)) {
             const int as = i & 1;
             const uint32_t aphase = (i >> 1) & 1;
@@ -930,6 +936,16 @@ cudaError_t launch_one(int grid, size_t smem, cudaStream_t st, const CUtensorMap
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    if (p.pdl) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(unsigned(grid)); cfg.blockDim = dim3(unsigned(cta_threads(NIBBLE, FRAG)));
+        cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
     }
     kern<<<grid, cta_threads(NIBBLE, FRAG), smem, st>>>(tmA, tmB, tmY, p);
     return cudaGetLastError();

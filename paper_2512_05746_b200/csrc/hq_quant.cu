@@ -181,6 +181,7 @@ __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, i
 // Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
 template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC, bool GN>
 __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
+    griddep_launch();      // a GEMM launched as a programmatic dependent may start its prologue as this grid drains
     constexpr int N = 1 << KLOG;
     constexpr int LE = ilog2_c(E);
     constexpr int P = E / 2;                           // two-wide registers per thread
@@ -346,6 +347,7 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
 // Generic path: one CTA per row (grid-stride), the row lives in shared memory, one __syncthreads per stage.
 template <typename InT>
 __global__ void __launch_bounds__(256) fwht_quant_generic(const QuantParams p, int had_block, int int8_out) {
+    griddep_launch();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* buf = reinterpret_cast<float*>(smem_raw);
     __shared__ float red[8];
@@ -435,6 +437,7 @@ struct WidthParams {
 
 template <int NB, typename InT>
 __global__ void __launch_bounds__(256) width_quant_kernel(const WidthParams p) {
+    griddep_launch();
     const int64_t item = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const float S = __ldg(p.static_scale);
     if (item == 0 && p.scale_out != nullptr) p.scale_out[0] = S * p.norm;
