@@ -391,8 +391,8 @@ def main_layer_list(args, which):
 
 def main_sweep(args):
     """Shape sweep of transform+quantize followed by the integer GEMM: M x K x N grid, Hadamard block = K, for
-    W4A4 with the folded two-limb weights (nibble codes), W4A4 with plain one-limb weights (nibble codes) and W8A8
-    (int8 codes, plain weights).  W4A3 runs the same kernels as W4A4 (only the quantizer range differs).  One JSON
+    W4A4 with the folded two-limb weights, W4A4 with plain one-limb weights (codes in the container --codes selects) and
+    W8A8 (plain weights).  W4A3 runs the same kernels as W4A4 (only the quantizer range differs).  One JSON
     line with one record per point: int TOPS of the GEMM, GB/s of the quantize stage, and the roofline fraction of
     the GEMM (slower of tensor peak and algorithmic bytes over the measured copy bandwidth)."""
     import torch
@@ -404,8 +404,8 @@ def main_sweep(args):
     Ms, Ks, Ns = (4096, 16384, 65536), (256, 512, 1024, 2048, 4096), (512, 1280, 4096)
     if args.rows != M_TOKENS:
         Ms = (int(args.rows),)
-    variants = (("W4A4 folded", 4, 4, hq.HQ_W_FOLDED, hq.HQ_CODES_NIBBLE),
-                ("W4A4 plain", 4, 4, hq.HQ_W_PLAIN, hq.HQ_CODES_NIBBLE),
+    variants = (("W4A4 folded", 4, 4, hq.HQ_W_FOLDED, CODES[0]),
+                ("W4A4 plain", 4, 4, hq.HQ_W_PLAIN, CODES[0]),
                 ("W8A8 plain", 8, 8, hq.HQ_W_PLAIN, hq.HQ_CODES_INT8))
     status = torch.zeros((1,), dtype=torch.int32, device=dev)
     gen = torch.Generator(device=dev)
@@ -458,7 +458,7 @@ def main_sweep(args):
     print(json.dumps(dict(metric="shape sweep: int TOPS of the GEMM and GB/s of transform+quantize per point", value=best["gemm_tops"],
                           unit="TOPS (best point)", n_gpus=1, steps=reps, warmup=3, higher_is_better=True, dtype="int8",
                           data="synthetic", vs_baseline=None,
-                          config=dict(workload="configs[4] shape sweep", int8_peak_tops=int8_peak, hbm_gbs=pk["hbm_gbs"],
+                          config=dict(workload="configs[4] shape sweep, " + codes_name() + " codes for W4A4", int8_peak_tops=int8_peak, hbm_gbs=pk["hbm_gbs"],
                                       peak_source=pk["source"]), points=points)))
 
 
