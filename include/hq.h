@@ -31,6 +31,11 @@
 #ifdef __cplusplus
 extern "C" {
 #endif
+/* The library is built with hidden visibility (two builds loaded into one process must not bind to one another's
+ * internals); the entry points declared here are its only exported symbols. */
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)
+#endif
 
 typedef enum {
     HQ_OK = 0,
@@ -224,6 +229,9 @@ float hq_alpha_for(const hq_weight_desc* desc);
  * The caller times it with events; ops = ctas * iters * 2*128*256*32.  dev_status as above. */
 hq_status hq_mma_i8_probe(int ctas, int iters, int32_t* dev_status, void* stream);
 
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cflags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
+    cflags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
     if verbose:
         cflags += ["-Xptxas", "-v"]
     objdir = os.path.join(_DIR, "_build")
