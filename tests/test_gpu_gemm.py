@@ -87,6 +87,21 @@ def test_qgemm_matches_oracle(env, oracle, M, K, N, a_bits, w_bits, had_block, m
     gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, container, seed=M + K + N)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_qgemm_random_shapes(env, oracle, seed):
+    """Seeded random draws over reduction length, Hadamard block, ragged M / N, weight mode and container: every launch
+    form of gemm_case (accumulators + bf16, fp32, bf16 alone) against the oracle."""
+    torch, hq = env
+    rng = np.random.default_rng(1000 + seed)
+    K = int(rng.choice([128, 256, 384, 512, 640, 1024, 1152]))
+    hb = int(rng.choice([h for h in (32, 128, 256, 512) if K % h == 0]))
+    N = int(rng.choice([8, 72, 128, 136, 200, 256, 384, 520]))
+    M = int(rng.choice([1, 127, 128, 129, 1000, 2500]))
+    mode = ["folded", "plain", "double"][int(rng.integers(3))]
+    container = int(rng.integers(2))
+    gemm_case(torch, hq, oracle, M, K, N, 4, 4, hb, mode, container, seed=seed, with_bias=bool(rng.integers(2)))
+
+
 def test_qgemm_extreme_magnitudes(env, oracle):
     """Largest accumulators the path can produce: (a) folded weights with a constant channel (B = -8*n at one index,
     so the high limb is at its extreme) against sign-matched extreme codes; (b) W8A8 with every product at 127*128."""
