@@ -382,6 +382,57 @@ def main_layer_list(args, which):
     for d in per_shape.values():
         d["ms_each"] = d["ms"] / d["count"]
         d["tops"] = 2.0 * d["macs"] * d["limbs"] / (d["ms_each"] * 1e-3) / 1e12
+    # The UNet's residual-block convolutions take SiLU(GroupNorm32(h)) as input: the same forward with that prologue
+    # fused into the transform kernel of those layers (statistics pass + normalise-on-load), reported beside the main figure.
+    gn_extra = None
+    if which == "unet":
+        gn_layers = [L for L in layers if L["kind"] == "conv" and L["R"] == 3 and L["stride"] == 1 and
+                     (".conv1" in L["name"] or ".conv2" in L["name"])]
+        for L in gn_layers:
+            r = L["res"]
+            if "gn" in r:
+                continue
+            cin, rows = L["C"], L["Nb"] * L["H"] * L["W"]
+            g = dict(gamma=torch.ones((cin,), device=dev), beta=torch.zeros((cin,), device=dev),
+                     scratch=torch.empty((L["Nb"] * 32 * 24,), dtype=torch.uint8, device=dev))
+            codes, sc = hq.workspace_views(r["ws"], rows, cin, CODES[0])
+            hq.hq_gn_silu_quant(r["x"], 32, g["gamma"], g["beta"], 1e-5, L["had_block"], A_BITS, codes, CODES[0], g["scratch"],
+                                scales=sc)
+            g["static"] = sc.max().reshape(1).contiguous()          # one static scale, calibrated on the normalised input
+            r["gn"] = g
+        torch.cuda.synchronize()
+        gn_names = {L["name"] for L in gn_layers}
+
+        def forward_gn():
+            for L in layers:
+                r = L["res"]
+                if L["name"] in gn_names:
+                    g = r["gn"]
+                    rows = L["Nb"] * L["H"] * L["W"]
+                    codes, sc = hq.workspace_views(r["ws"], rows, L["C"], CODES[0])
+                    hq.hq_gn_silu_quant(r["x"], 32, g["gamma"], g["beta"], 1e-5, L["had_block"], A_BITS, codes, CODES[0],
+                                        g["scratch"], scales=sc[:1], static_scale=g["static"])
+                    hq.hq_qconv2d(codes, CODES[0], A_BITS, L["Nb"], L["H"], L["W"], L["C"], r["pw"], L["R"], L["R"], L["stride"],
+                                  L["pad"], scale_a=g["static"], bias=r["bias"], alpha=r["pw"].alpha, y=r["y"], dev_status=status)
+                elif L["kind"] == "conv":
+                    hq.hq_qconv(r["x"], r["pw"], L["R"], L["R"], L["stride"], L["pad"], r["bias"], A_BITS, r["y"], r["ws"],
+                                static_scale=r["static"], dev_status=status)
+                else:
+                    hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
+
+        for _ in range(3):
+            forward_gn()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(steps):
+            forward_gn()
+        g1.record()
+        torch.cuda.synchronize()
+        hq.hq_check_status(status)
+        gn_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(gn_layers),
+                        note="GroupNorm(32) + SiLU fused in front of the residual-block 3x3 convolutions "
+                             "(hq_gn_silu_quant + hq_qconv2d for those layers)")
     macs = sum(L["macs"] for L in layers)
     ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
     print(json.dumps(dict(metric="forwards/s of " + label,
@@ -392,7 +443,8 @@ def main_layer_list(args, which):
                                       layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
                                       l2="activations of the large layers exceed L2"),
-                          clocks=clocks, gpu_launches=2 * len(layers) * steps, per_shape=per_shape)))
+                          clocks=clocks, gpu_launches=2 * len(layers) * steps, per_shape=per_shape,
+                          with_groupnorm_prologue=gn_extra)))
 
 
 def main_sweep(args):
