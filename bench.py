@@ -520,6 +520,50 @@ def main_sweep(args):
                                       peak_source=pk["source"]), points=points)))
 
 
+def main_gn(args):
+    """GroupNorm(32) + SiLU + transform + quantize on one NHWC bf16 tensor (64 x 64 x 64 x 256, the input of a UNet
+    residual-block convolution), beside the plain transform + quantize of the same tensor."""
+    import torch
+    from paper_2512_05746_b200 import binding as hq
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Nb, H, W, Cc = 64, 64, 64, 256
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    x = (torch.randn((Nb, H, W, Cc), generator=gen, device=dev) * 1.5 + 0.3).to(torch.bfloat16)
+    gamma = torch.rand((Cc,), generator=gen, device=dev) + 0.5
+    beta = torch.randn((Cc,), generator=gen, device=dev) * 0.1
+    rows = Nb * H * W
+    codes = torch.empty((rows, code_pitch(Cc)), dtype=torch.uint8, device=dev)
+    sc = torch.empty((rows,), dtype=torch.float32, device=dev)
+    scratch = torch.empty((Nb * 32 * 24,), dtype=torch.uint8, device=dev)
+    steps, warmup = max(1, min(args.steps, 20)), max(3, min(args.warmup, 5))
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    gn_ms = timed(lambda: hq.hq_gn_silu_quant(x, 32, gamma, beta, 1e-5, 256, A_BITS, codes, CODES[0], scratch, scales=sc))
+    plain_ms = timed(lambda: hq.hq_hadamard_quant(x.view(rows, Cc), 256, A_BITS, codes, CODES[0], scales=sc))
+    cb = code_pitch(2) / 2.0
+    gbytes = x.numel() * (2 * 2.0 + cb) + rows * 4.0                     # x read twice, codes and scales written
+    pk = peaks()
+    print(json.dumps(dict(metric="GB/s of GroupNorm+SiLU+transform+quantize (x read twice + codes written)",
+                          value=gbytes / gn_ms / 1e6, unit="GB/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=gn_ms,
+                          higher_is_better=True, dtype="f32", data="synthetic", vs_baseline=None,
+                          config=dict(workload=f"GroupNorm(32)+SiLU prologue on {Nb}x{H}x{W}x{Cc} bf16, {codes_name()} codes"),
+                          plain_transform_quantize_ms=plain_ms, frac_of_copy_bandwidth=gbytes / gn_ms / 1e6 / pk["hbm_gbs"],
+                          gpu_launches=3 * steps)))
+
+
 def main():
     global M_TOKENS, WORKLOAD
     ap = argparse.ArgumentParser()
@@ -528,9 +572,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep"],
+    ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep", "gn"],
                     help="step: the benchmark step (default); unet / dit: the quantized layers of the UNet- / DiT-shaped workload; "
-                         "sweep: the M x K x N shape sweep")
+                         "sweep: the M x K x N shape sweep; gn: the GroupNorm+SiLU prologue on one tensor")
     ap.add_argument("--codes", default="int8", choices=["nibble", "int8"],
                     help="container of the 4-bit activation codes between the transform and the GEMM kernel: one per "
                          "byte (default, the faster one) or two per byte (half the workspace)")
@@ -548,6 +592,8 @@ def main():
         return main_layer_list(args, args.workload)
     if args.workload == "sweep":
         return main_sweep(args)
+    if args.workload == "gn":
+        return main_gn(args)
 
     import torch
     import torch.distributed as dist
