@@ -438,7 +438,7 @@ def main_layer_list(args, which):
     print(json.dumps(dict(metric="forwards/s of " + label,
                           value=1e3 / ms, unit="forwards/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=ms,
                           higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int8", data="synthetic",
-                          config=dict(workload=wl + ", bf16 in/out, W4A4 folded two-limb weights, " + codes_name() + " codes",
+                          config=dict(workload=wl + f", bf16 in/out, W4A{A_BITS} folded two-limb weights, " + codes_name() + " codes",
                                       layers=len(layers),
                                       layers_per_s=len(layers) * 1e3 / ms, tops_limbs=ops_limbs / ms / 1e9,
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
@@ -565,7 +565,7 @@ def main_gn(args):
 
 
 def main():
-    global M_TOKENS, WORKLOAD
+    global M_TOKENS, WORKLOAD, A_BITS, METRIC
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
@@ -575,6 +575,8 @@ def main():
     ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep", "gn"],
                     help="step: the benchmark step (default); unet / dit: the quantized layers of the UNet- / DiT-shaped workload; "
                          "sweep: the M x K x N shape sweep; gn: the GroupNorm+SiLU prologue on one tensor")
+    ap.add_argument("--a-bits", type=int, default=4, choices=[3, 4],
+                    help="activation bits of the step / unet / dit workloads (INT3 codes travel in the same containers)")
     ap.add_argument("--codes", default="int8", choices=["nibble", "int8"],
                     help="container of the 4-bit activation codes between the transform and the GEMM kernel: one per "
                          "byte (default, the faster one) or two per byte (half the workspace)")
@@ -583,6 +585,10 @@ def main():
     args = ap.parse_args()
     CODES[0] = 0 if args.codes == "nibble" else 1
     WORKLOAD = WORKLOAD + f", {args.codes} codes"
+    if args.a_bits != 4:
+        A_BITS = int(args.a_bits)
+        WORKLOAD = WORKLOAD.replace("W4A4", f"W4A{A_BITS}")
+        METRIC = METRIC.replace("W4A4", f"W4A{A_BITS}")
     if args.rows != M_TOKENS:
         M_TOKENS = int(args.rows)
         WORKLOAD = f"REDUCED to {M_TOKENS} rows per layer (profiling case, not a benchmark number): " + WORKLOAD
