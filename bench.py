@@ -468,11 +468,11 @@ def main_sweep(args):
     status = torch.zeros((1,), dtype=torch.int32, device=dev)
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
-    reps = max(3, min(args.steps, 10))
+    reps = max(3, min(args.steps, 50))
     points = []
 
     def timed(fn):
-        for _ in range(3):
+        for _ in range(10):
             fn()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -514,7 +514,7 @@ def main_sweep(args):
     hq.hq_check_status(status)
     best = max(points, key=lambda d: d["gemm_tops"])
     print(json.dumps(dict(metric="shape sweep: int TOPS of the GEMM and GB/s of transform+quantize per point", value=best["gemm_tops"],
-                          unit="TOPS (best point)", n_gpus=1, steps=reps, warmup=3, higher_is_better=True, dtype="int8",
+                          unit="TOPS (best point)", n_gpus=1, steps=reps, warmup=10, higher_is_better=True, dtype="int8",
                           data="synthetic", vs_baseline=None,
                           config=dict(workload="configs[4] shape sweep, " + codes_name() + " codes for W4A4", int8_peak_tops=int8_peak, hbm_gbs=pk["hbm_gbs"],
                                       peak_source=pk["source"]), points=points)))
