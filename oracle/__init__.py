@@ -56,6 +56,7 @@ def lib():
             L.hqo_conv2d_dequant_perpixel.argtypes = [p, p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int,
                                                       C.c_int, C.c_int, p, p, C.c_double, p]
             L.hqo_groupnorm_silu.argtypes = [p, i64, i64, i64, i64, C.c_int, p, p, C.c_double, p]
+            L.hqo_layernorm_affine.argtypes = [p, i64, i64, p, p, i64, C.c_double, p]
             L.hqo_transform_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
             L.hqo_codes_inverse_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
             L.hqo_conv2d_int_z.argtypes = [p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int, C.c_int, C.c_int, p]
@@ -248,6 +249,24 @@ def groupnorm_silu(x, groups: int, gamma, beta, eps: float = 1e-6) -> np.ndarray
     out = np.empty_like(x)
     _chk(lib().hqo_groupnorm_silu(_ptr(x), Nb, H, W, Cc, groups, _ptr(gamma), _ptr(beta), float(eps), _ptr(out)),
          "groupnorm_silu")
+    return out
+
+
+def layernorm_affine(x, weight=None, bias=None, rows_per_group: int = 0, eps: float = 1e-6) -> np.ndarray:
+    """LayerNorm over the last axis of x [rows, cols] (biased variance), then y * weight[g] + bias[g] with
+    g = row // rows_per_group (one vector pair for all rows when rows_per_group <= 0); fp64."""
+    x = _c(x, np.float64)
+    rows, cols = x.shape
+    w = None if weight is None else _c(np.asarray(weight, np.float64).reshape(-1, cols), np.float64)
+    b = None if bias is None else _c(np.asarray(bias, np.float64).reshape(-1, cols), np.float64)
+    groups = (rows + rows_per_group - 1) // rows_per_group if rows_per_group > 0 else 1
+    for v in (w, b):
+        if v is not None and v.shape[0] != groups:
+            raise ValueError("one affine vector per group of rows is needed")
+    out = np.empty_like(x)
+    _chk(lib().hqo_layernorm_affine(_ptr(x), rows, cols, _ptr(w) if w is not None else None,
+                                    _ptr(b) if b is not None else None, int(rows_per_group), float(eps), _ptr(out)),
+         "layernorm_affine")
     return out
 
 

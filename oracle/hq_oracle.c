@@ -386,6 +386,34 @@ i64 hqo_conv2d_int_z(const int32_t* z, const int32_t* B, i64 Nb, i64 H, i64 W, i
     return bad;
 }
 
+/* ---- LayerNorm with a per-sample affine in front of a quantized linear (the "modulate(norm(x), shift, scale)" of a
+ * diffusion-transformer block) ---------------------------------------------------------------------------------
+ * Not part of the paper's equations: the usual definition, written out.  x [rows][cols]; per row: mean and biased
+ * variance over the cols values; y = (x - mean) / sqrt(var + eps) * w[g][c] + b[g][c], where g = row / rows_per_group
+ * selects the affine vectors of the row's sample (rows_per_group <= 0: one vector pair for all rows).
+ * w == NULL means 1, b == NULL means 0. */
+int hqo_layernorm_affine(const double* x, i64 rows, i64 cols, const double* w, const double* b, i64 rows_per_group,
+                         double eps, double* out) {
+    if (rows < 0 || cols <= 0) return -1;
+#pragma omp parallel for schedule(static)
+    for (i64 r = 0; r < rows; ++r) {
+        const double* xr = x + r * cols;
+        double sum = 0.0;
+        for (i64 c = 0; c < cols; ++c) sum += xr[c];
+        const double mean = sum / (double)cols;
+        double var = 0.0;
+        for (i64 c = 0; c < cols; ++c) { const double d = xr[c] - mean; var += d * d; }
+        var /= (double)cols;
+        const double rstd = 1.0 / sqrt(var + eps);
+        const i64 g = rows_per_group > 0 ? r / rows_per_group : 0;
+        for (i64 c = 0; c < cols; ++c) {
+            const double wc = w ? w[g * cols + c] : 1.0, bc = b ? b[g * cols + c] : 0.0;
+            out[r * cols + c] = (xr[c] - mean) * rstd * wc + bc;
+        }
+    }
+    return 0;
+}
+
 /* ---- GroupNorm + SiLU in front of a quantized convolution (the "in_layers" of a ResBlock) -------------------
  * Not part of the paper's equations: the usual definitions, written out.  x NHWC [Nb][H][W][C], `groups` groups of
  * C/groups consecutive channels; per sample and group: mean and biased variance over H*W*(C/groups) values;

@@ -488,3 +488,30 @@ def test_groupnorm_silu_against_library_routine(oracle):
     assert np.allclose(const, beta[:8] / (1 + np.exp(-beta[:8])), atol=1e-9)
     with pytest.raises(ValueError):
         oracle.groupnorm_silu(x, 5, gamma, beta)                                   # 24 channels do not split into 5 groups
+
+
+# ------------------------------------------------------------------ LayerNorm + per-sample affine prologue
+
+def test_layernorm_affine_against_library_routine(oracle):
+    """The written-out definition against torch's layer_norm on the CPU in fp64 (a library routine) followed by the
+    modulation y * (1 + scale) + shift of a diffusion-transformer block, plus closed forms: without an affine every row
+    has mean 0 and variance 1 / (1 + eps / var); a constant row gives the bias; a per-row shift and a positive per-row
+    scale of x leave the result unchanged (up to the eps term)."""
+    import torch
+    rng = np.random.default_rng(1)
+    rows, cols, rpg = 12, 40, 4
+    x = rng.standard_normal((rows, cols)) * 2.5 + 0.7
+    scale, shift = rng.standard_normal((3, cols)) * 0.3, rng.standard_normal((3, cols))
+    got = oracle.layernorm_affine(x, 1.0 + scale, shift, rows_per_group=rpg, eps=1e-6)
+    ln = torch.nn.functional.layer_norm(torch.from_numpy(x), (cols,), None, None, 1e-6).numpy()
+    want = ln * (1.0 + np.repeat(scale, rpg, axis=0)) + np.repeat(shift, rpg, axis=0)
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    plain = oracle.layernorm_affine(x, eps=1e-6)
+    assert np.allclose(plain.mean(axis=1), 0.0, atol=1e-12)
+    assert np.allclose(plain.var(axis=1), 1.0 / (1.0 + 1e-6 / x.var(axis=1)), rtol=1e-12)
+    const = oracle.layernorm_affine(np.full((2, cols), 3.0), np.ones((1, cols)), shift[:1], eps=1e-6)
+    assert np.allclose(const, np.repeat(shift[:1], 2, axis=0), atol=1e-12)
+    moved = oracle.layernorm_affine(x * 3.0 + rng.standard_normal((rows, 1)), 1.0 + scale, shift, rows_per_group=rpg, eps=1e-12)
+    assert np.allclose(moved, oracle.layernorm_affine(x, 1.0 + scale, shift, rows_per_group=rpg, eps=1e-12), atol=1e-9)
+    with pytest.raises(ValueError):
+        oracle.layernorm_affine(x, scale[:2], shift, rows_per_group=rpg)          # 12 rows in groups of 4 need 3 vectors
