@@ -433,6 +433,65 @@ def main_layer_list(args, which):
         gn_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(gn_layers),
                         note="GroupNorm(32) + SiLU fused in front of the residual-block 3x3 convolutions "
                              "(hq_gn_silu_quant + hq_qconv2d for those layers)")
+    # The transformer's QKV and FC1 linears take modulate(LayerNorm(x), shift, scale) as input: the same forward with that
+    # prologue fused into the transform kernel of those layers (row statistics from the registers that hold the row).
+    ln_extra = None
+    if which == "dit":
+        ln_names = {L["name"] for L in layers if L["name"].endswith(".qkv") or L["name"].endswith(".fc1")}
+        tokens = 256
+        for L in layers:
+            r = L["res"]
+            if L["name"] in ln_names and "ln" not in r:
+                groups = L["M"] // tokens
+                r["ln"] = dict(w=1.0 + 0.1 * torch.randn((groups, L["K"]), generator=gen, device=dev),
+                               b=0.1 * torch.randn((groups, L["K"]), generator=gen, device=dev))
+
+        def forward_ln():
+            for L in layers:
+                r = L["res"]
+                if L["name"] in ln_names:
+                    codes, sc = hq.workspace_views(r["ws"], L["M"], L["K"], CODES[0])
+                    hq.hq_ln_quant(r["x"], r["ln"]["w"], r["ln"]["b"], tokens, 1e-6, L["had_block"], A_BITS, codes, CODES[0],
+                                   scales=sc)
+                    hq.hq_qgemm(codes, CODES[0], A_BITS, L["K"], r["pw"], scale_a=sc, bias=r["bias"], alpha=r["pw"].alpha,
+                                y=r["y"], dev_status=status)
+                else:
+                    hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
+
+        for _ in range(3):
+            forward_ln()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(steps):
+            forward_ln()
+        g1.record()
+        torch.cuda.synchronize()
+        hq.hq_check_status(status)
+        # the prologue alone against the plain transform on the block input (8192 x 1152 bf16)
+        Lq = next(L for L in layers if L["name"].endswith(".qkv"))
+        rq = Lq["res"]
+        cq, sq = hq.workspace_views(rq["ws"], Lq["M"], Lq["K"], CODES[0])
+
+        def t_of(fn):
+            for _ in range(5):
+                fn()
+            torch.cuda.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for _ in range(20):
+                fn()
+            a1.record()
+            torch.cuda.synchronize()
+            return a0.elapsed_time(a1) / 20
+
+        ln_us = 1e3 * t_of(lambda: hq.hq_ln_quant(rq["x"], rq["ln"]["w"], rq["ln"]["b"], tokens, 1e-6, Lq["had_block"], A_BITS,
+                                                  cq, CODES[0], scales=sq))
+        pl_us = 1e3 * t_of(lambda: hq.hq_hadamard_quant(rq["x"], Lq["had_block"], A_BITS, cq, CODES[0], scales=sq))
+        ln_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(ln_names),
+                        ln_quant_us=ln_us, plain_quant_us=pl_us,
+                        note="LayerNorm + per-sample modulation fused in front of the QKV and FC1 linears (hq_ln_quant + "
+                             "hq_qgemm for those layers; without the dependent launch of the fused layer call)")
     macs = sum(L["macs"] for L in layers)
     ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
     print(json.dumps(dict(metric="forwards/s of " + label,
@@ -444,7 +503,7 @@ def main_layer_list(args, which):
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
                                       l2="activations of the large layers exceed L2"),
                           clocks=clocks, gpu_launches=2 * len(layers) * steps, per_shape=per_shape,
-                          with_groupnorm_prologue=gn_extra)))
+                          with_groupnorm_prologue=gn_extra, with_layernorm_prologue=ln_extra)))
 
 
 def main_sweep(args):

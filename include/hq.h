@@ -179,6 +179,22 @@ hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int
                          const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
                          int32_t* dev_status, void* stream);
 
+/* ---- LayerNorm with a per-sample affine fused in front of the transform + quantization (no counterpart in the paper's
+ * equations: the "modulate(norm(x), shift, scale)" that precedes the quantized linears of a diffusion-transformer block;
+ * the row statistics are taken from the registers that hold the row for the transform, so the activations make one trip
+ * through memory). --------------------------------------------------------------------------------------------------
+ * x        device [rows][ldx] fp32/bf16.   Per row: mean and biased variance over the cols values,
+ *          y = (x - mean) / sqrt(var + eps) * weight[g][c] + bias[g][c],   g = row / rows_per_group
+ *          (rows_per_group = 0: one vector pair for all rows).  For adaLN pass weight = 1 + scale, bias = shift.
+ * weight, bias   device [groups][cols] fp32, 16-byte aligned, or NULL (1 and 0).   The rest as hq_hadamard_quant.
+ * Restrictions: the row shapes of the fast kernel only (had_block in 32..4096, cols / 32 (64 above 512-wide blocks)
+ * <= 256 threads per row and a CTA of at most 320 threads; 16-byte aligned codes and pitches), else HQ_ERR_UNSUPPORTED;
+ * rows_per_group must be a multiple of the rows one CTA takes (any multiple of 32 is). */
+hq_status hq_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
+                      const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
+                      hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                      int64_t ld_codes, float* scales, void* stream);
+
 /* ---- GroupNorm + SiLU fused in front of the transform + quantization (no counterpart in the paper's equations:
  * the normalisation and activation that precede the quantized 3x3 convolutions of a UNet ResBlock, applied while the
  * activations are read, so that they make one trip through memory instead of three). ---------------------------------

@@ -24,7 +24,8 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
-           "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant"]
+           "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
+           "hq_ln_quant"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -72,12 +73,13 @@ def _load():
                                  p, p, i32, p, C.c_size_t, p, p]
     L.hq_gn_silu_quant.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, i32, i32, i32, p, p, i32, i64, p, p,
                                    C.c_size_t, p]
+    L.hq_ln_quant.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, i32, i32, i32, p, p, i32, i64, p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
                  "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
-                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant"):
+                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -251,6 +253,17 @@ def hq_gn_silu_quant(x, groups: int, gamma, beta, eps: float, had_block: int, bi
                                 bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
                                 _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)),
            "hq_gn_silu_quant")
+
+
+def hq_ln_quant(x, weight, bias, rows_per_group: int, eps: float, had_block: int, bits: int, codes, container: int,
+                scales=None, static_scale=None, stream=None) -> None:
+    """LayerNorm over each row of x [rows, cols] with the affine vectors weight/bias [groups, cols] (or None) of the row's
+    group, then transform + quantization into codes [rows, pitch]."""
+    rows, cols = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_ln_quant(_dptr(x), _dtype_code(x), rows, cols, x.stride(0), _dptr(weight), _dptr(bias), rows_per_group,
+                           eps, had_block, bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0),
+                           _dptr(scales), _stream(stream)), "hq_ln_quant")
 
 
 def hq_hadamard_quant_width(x, had_block_w: int, bits: int, static_scale, z, scale_out=None, stream=None) -> None:

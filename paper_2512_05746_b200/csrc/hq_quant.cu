@@ -38,6 +38,12 @@ struct QuantParams {
     const float* gn_beta;    // [cols]
     int gn_groups;
     int64_t gn_rows_per_sample;
+    // optional LayerNorm over each row with a per-sample affine, applied before the transform (ln_on != 0)
+    int ln_on;
+    const float* ln_w;       // [groups][cols] or nullptr (= 1)
+    const float* ln_b;       // [groups][cols] or nullptr (= 0)
+    int64_t ln_rows_per_group;   // rows that share one affine vector pair; 0: all rows
+    float ln_eps;
 };
 
 __device__ __forceinline__ float silu(float y) { return __fdividef(y, 1.0f + __expf(-y)); }
@@ -108,6 +114,7 @@ __device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) { asm("mov.b
 __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 
 // Butterflies over pair-index bits: element distance 2*h for h = LO .. HI (pairs stay pairs).
 template <int P, int LO, int HI>
@@ -179,8 +186,12 @@ __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, i
 //            two threads of a group interleave their bytes with one shuffle so that each stores contiguous bytes.
 //            KLOG = 12 needs one more stage than fits and takes it with a lane exchange.
 // Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
-template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC, bool GN>
+// PRO: prologue applied to the values before the transform: 0 none, 1 GroupNorm + SiLU (statistics given), 2 LayerNorm
+// over the row (statistics taken here: the row is in the registers of its threads) with a per-sample affine.
+template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC, int PRO>
 __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
+    constexpr bool GN = PRO == 1;
+    constexpr bool LN = PRO == 2;
     griddep_launch();      // a GEMM launched as a programmatic dependent may start its prologue as this grid drains
     constexpr int N = 1 << KLOG;
     constexpr int LE = ilog2_c(E);
@@ -224,6 +235,13 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
         }
         __syncthreads();
     }
+    // LayerNorm prologue: two sums per row, gathered in shared memory (the affine vectors of the CTA's sample are read
+    // from global memory as they are used: a CTA holds only a few rows, a table of its own would cost more than it saves)
+    float* lnacc = gn_a;                               // [rows_per_cta][2]
+    if (LN) {
+        if (tid < 2 * p.rows_per_cta) lnacc[tid] = 0.f;
+        __syncthreads();
+    }
 
     f32x2 v[P];
     {
@@ -241,6 +259,45 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
             if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
             v[2 * i] = pk2(f.x, f.y);
             v[2 * i + 1] = pk2(f.z, f.w);
+        }
+    }
+    if (LN) {
+        // mean, then the sum of squared deviations (two passes over the registers), each gathered per row through a
+        // shared-memory sum; y = (x - mean) * rstd * w[c] + b[c]
+        // four neighbouring lanes belong to one row when the row's thread count is a multiple of 4: add them up by
+        // shuffles first, so that a quarter of the threads go to shared memory
+        const bool quad = (p.threads_per_row & 3) == 0;
+        f32x2 acc = v[0];
+#pragma unroll
+        for (int i = 1; i < P; ++i) acc = add2(acc, v[i]);
+        float lo, hi;
+        upk2(acc, lo, hi);
+        float part = lo + hi;
+        if (quad) { part += __shfl_xor_sync(0xffffffffu, part, 1); part += __shfl_xor_sync(0xffffffffu, part, 2); }
+        if (!quad || (tid & 3) == 0) atomicAdd(&lnacc[2 * row_in_cta], part);
+        __syncthreads();
+        const float mean = lnacc[2 * row_in_cta] / float(p.cols);
+        const f32x2 mean2 = pk2(mean, mean);
+        acc = pk2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < P; ++i) { v[i] = sub2(v[i], mean2); acc = fma2(v[i], v[i], acc); }
+        upk2(acc, lo, hi);
+        part = lo + hi;
+        if (quad) { part += __shfl_xor_sync(0xffffffffu, part, 1); part += __shfl_xor_sync(0xffffffffu, part, 2); }
+        if (!quad || (tid & 3) == 0) atomicAdd(&lnacc[2 * row_in_cta + 1], part);
+        __syncthreads();
+        const float rstd = rsqrtf(lnacc[2 * row_in_cta + 1] / float(p.cols) + p.ln_eps);
+        const f32x2 rstd2 = pk2(rstd, rstd);
+        const int64_t g = p.ln_rows_per_group > 0 ? (int64_t(blockIdx.x) * p.rows_per_cta) / p.ln_rows_per_group : 0;
+        const float* wrow = p.ln_w != nullptr ? p.ln_w + g * p.cols : nullptr;
+        const float* brow = p.ln_b != nullptr ? p.ln_b + g * p.cols : nullptr;
+#pragma unroll
+        for (int i = 0; i < E / 4; ++i) {
+            const int ch = blk * N + 4 * (tb + TB * i);
+            const float4 a4 = wrow != nullptr ? __ldg(reinterpret_cast<const float4*>(wrow + ch)) : make_float4(1.f, 1.f, 1.f, 1.f);
+            const float4 b4 = brow != nullptr ? __ldg(reinterpret_cast<const float4*>(brow + ch)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[2 * i] = valid ? fma2(mul2(v[2 * i], rstd2), pk2(a4.x, a4.y), pk2(b4.x, b4.y)) : pk2(0.f, 0.f);
+            v[2 * i + 1] = valid ? fma2(mul2(v[2 * i + 1], rstd2), pk2(a4.z, a4.w), pk2(b4.z, b4.w)) : pk2(0.f, 0.f);
         }
     }
     butterfly_within_pairs<P>(v);                      // index bit 0
@@ -584,11 +641,15 @@ cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threa
         return cudaGetLastError();
     };
     if (p.gn_stats != nullptr) {
-        if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, true>) : go(fwht_quant_fast<KLOG, E, InT, true, false, true>);
-        return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, true>) : go(fwht_quant_fast<KLOG, E, InT, false, false, true>);
+        if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 1>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 1>);
+        return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, 1>) : go(fwht_quant_fast<KLOG, E, InT, false, false, 1>);
     }
-    if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, false>) : go(fwht_quant_fast<KLOG, E, InT, true, false, false>);
-    return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, false>) : go(fwht_quant_fast<KLOG, E, InT, false, false, false>);
+    if (p.ln_on) {
+        if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 2>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 2>);
+        return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, 2>) : go(fwht_quant_fast<KLOG, E, InT, false, false, 2>);
+    }
+    if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 0>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 0>);
+    return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, 0>) : go(fwht_quant_fast<KLOG, E, InT, false, false, 0>);
 }
 
 // Values per thread for a block of 2^klog channels.
@@ -614,11 +675,12 @@ cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int gri
 
 // Launches the transform+quantize kernel; shared by the public entry point and the fused layer calls.
 struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; };
+struct LnArgs { const float* w; const float* b; int64_t rows_per_group; float eps; };
 
 static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
                                    int bits, hq_scale_mode mode, const float* static_scale, void* codes,
                                    hq_container cont, int64_t ld_codes, float* scales, const GnArgs* gn,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, const LnArgs* ln = nullptr) {
     if (rows == 0 && cols > 0) return HQ_OK;                       // nothing to do; pointers may be NULL
     if (x == nullptr || codes == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
@@ -648,6 +710,9 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
         p.gn_stats = gn->stats; p.gn_gamma = gn->gamma; p.gn_beta = gn->beta; p.gn_groups = gn->groups;
         p.gn_rows_per_sample = gn->rows_per_sample;
     }
+    if (ln != nullptr) {
+        p.ln_on = 1; p.ln_w = ln->w; p.ln_b = ln->b; p.ln_rows_per_group = ln->rows_per_group; p.ln_eps = ln->eps;
+    }
 
     const int elt = xdt == HQ_F32 ? 4 : 2;
     const int E = fast_e(klog);
@@ -666,11 +731,12 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
         if (gn != nullptr && gn->rows_per_sample % rpc != 0) return HQ_ERR_UNSUPPORTED;   // a CTA must stay in one sample
+        if (ln != nullptr && ln->rows_per_group > 0 && ln->rows_per_group % rpc != 0) return HQ_ERR_UNSUPPORTED;
         if (threads <= 320) {                               // otherwise the generic kernel below takes the row shape
         // exchange buffer: per Hadamard block n/4 float4 slots plus one slot of padding per J (J = E/2 or E/4)
         const int jslots = (klog - ilog2(E) >= ilog2(E) - 1) ? E / 2 : E / 4;
         const size_t smem = size_t(threads / (n / E)) * size_t(n / 4 + n / 4 / jslots) * 16 + size_t((rpc + 3) & ~3) * 4 +
-                            (gn != nullptr ? size_t(cols) * 8 : 0);
+                            (gn != nullptr ? size_t(cols) * 8 : 0) + (ln != nullptr ? size_t(rpc) * 8 : 0);
         const int grid = int((rows + rpc - 1) / rpc);
         cudaError_t e = xdt == HQ_F32
                             ? dispatch_fast<float>(klog, p, cont == HQ_CODES_INT8, grid, threads, smem, st)
@@ -678,7 +744,7 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
         return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
         }
     }
-    if (gn != nullptr) return HQ_ERR_UNSUPPORTED;           // the prologue exists in the fast kernel only
+    if (gn != nullptr || ln != nullptr) return HQ_ERR_UNSUPPORTED;   // the prologues exist in the fast kernel only
     const size_t smem = size_t(cols) * 4;
     if (smem > 200 * 1024) return HQ_ERR_UNSUPPORTED;
     const int grid = int(rows < 148 * 8 ? rows : 148 * 8);
@@ -748,6 +814,19 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
                              st);
 }
 
+// LayerNorm over each row with a per-sample affine, fused into the transform+quantize kernel (one pass: the row's
+// statistics are taken from the registers that already hold it).
+hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
+                          const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
+                          hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
+                          float* scales, cudaStream_t st) {
+    if (rows_per_group < 0 || !(eps >= 0.f)) return HQ_ERR_INVALID_ARG;
+    if ((weight != nullptr && !aligned16(weight)) || (bias != nullptr && !aligned16(bias)) || cols % 4 != 0) return HQ_ERR_ALIGNMENT;
+    const LnArgs ln{weight, bias, rows_per_group, eps};
+    return launch_quant_impl(x, xdt, rows, cols, ldx, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales,
+                             nullptr, st, &ln);
+}
+
 // Width-axis transform + quantization + integer factor of Eq. 13-14: x NHWC fp32/bf16 -> z int8 NHWC.
 hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                       int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
@@ -787,6 +866,14 @@ hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, i
 }
 
 }  // namespace hq
+
+extern "C" hq_status hq_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
+                                 const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
+                                 hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                                 int64_t ld_codes, float* scales, void* stream) {
+    return hq::launch_ln_quant(x, xdt, rows, cols, ldx, weight, bias, rows_per_group, eps, had_block, bits, mode,
+                               static_scale, codes, cont, ld_codes, scales, static_cast<cudaStream_t>(stream));
+}
 
 extern "C" hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                       int groups, const float* gamma, const float* beta, float eps, int had_block,

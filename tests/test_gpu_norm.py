@@ -71,3 +71,69 @@ def test_gn_silu_quant_matches_oracle(env, oracle, Nb, H, W, C, G, n, bits, dt, 
     s_gpu = scales.cpu().numpy()[:, None] if not static else np.float32(s0)
     inside = np.abs(v) < oracle.qmax(bits)
     assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)
+
+
+LN_TIE_REL = 1e-5          # fp32 row statistics (sums of up to 4608 values) and rsqrt in front of the plain kernel's window
+LN_MISMATCH_FRAC = 1e-3
+LN_SCALE_RTOL = 1e-5
+
+
+@pytest.mark.parametrize("rows,cols,n,rpg,bits,dt,cont,static,affine", [
+    (512, 1152, 128, 256, 4, "bf16", 1, False, True),    # the diffusion-transformer width: nine 128-blocks, two samples
+    (300, 1152, 128, 0, 4, "f32", 0, False, True),       # ragged row count, one affine pair for all rows
+    (256, 512, 512, 32, 3, "f32", 1, False, True),       # one block per row, eight samples
+    (192, 4608, 128, 64, 4, "bf16", 1, False, True),     # the MLP's hidden width (36 blocks)
+    (128, 256, 256, 0, 4, "f32", 0, True, False),        # static scale, no affine
+    (96, 2048, 2048, 32, 4, "f32", 1, False, True),      # 64 values per thread
+])
+def test_ln_quant_matches_oracle(env, oracle, rows, cols, n, rpg, bits, dt, cont, static, affine):
+    torch, hq = env
+    rng = np.random.default_rng(rows + cols)
+    x = inputs.activations((rows, cols), outlier_count=max(1, cols // 100), outlier_scale=8.0, seed=cols + n) * np.float32(1.7) \
+        + np.float32(0.4)
+    groups = (rows + rpg - 1) // rpg if rpg > 0 else 1
+    w = (1.0 + 0.3 * rng.standard_normal((groups, cols))).astype(np.float32) if affine else None
+    b = (0.5 * rng.standard_normal((groups, cols))).astype(np.float32) if affine else None
+    xt = torch.from_numpy(x).cuda()
+    if dt == "bf16":
+        xt = xt.to(torch.bfloat16)
+        x = xt.float().cpu().numpy()
+    eps = 1e-6
+    pitch = cols // 2 if cont == 0 else cols
+    codes = torch.full((rows, pitch), 0x5A, dtype=torch.uint8, device="cuda")
+    scales = torch.full((rows,), -1.0, dtype=torch.float32, device="cuda")
+    y_ref = oracle.layernorm_affine(x, w, b, rows_per_group=rpg, eps=eps)
+    u = oracle.transform(y_ref, n)
+    s0 = float(np.float32(np.abs(u).max() / oracle.qmax(bits) / 2.0)) if static else None
+    ss = torch.tensor([s0], dtype=torch.float32, device="cuda") if static else None
+    hq.hq_ln_quant(xt, None if w is None else torch.from_numpy(w).cuda(), None if b is None else torch.from_numpy(b).cuda(),
+                   rpg, eps, n, bits, codes, cont, scales=scales, static_scale=ss)
+    torch.cuda.synchronize()
+    q = unpack_nibbles_np(codes.cpu().numpy()) if cont == 0 else codes.cpu().numpy().view(np.int8)
+    q_ref, s_ref, v = oracle.quantize(u, bits, static_scale=s0, want_v=True)
+    if static:
+        assert float(scales.cpu()[0]) == np.float32(s0)
+        v = np.clip(v, oracle.qmin(bits) - 0.25, oracle.qmax(bits) + 0.25)
+    else:
+        assert np.allclose(scales.cpu().numpy(), s_ref, rtol=LN_SCALE_RTOL, atol=0)
+    bad = q != q_ref
+    if bad.any():
+        assert np.abs(q.astype(np.int32) - q_ref)[bad].max() == 1
+        assert bad.mean() <= LN_MISMATCH_FRAC
+        full = np.maximum(np.abs(v).max(axis=1, keepdims=True), 1.0)
+        dist = np.abs(v - (np.floor(v) + 0.5))
+        assert np.all(dist[bad] <= (LN_TIE_REL * np.broadcast_to(full, v.shape))[bad])
+    s_gpu = scales.cpu().numpy()[:, None] if not static else np.float32(s0)
+    inside = np.abs(v) < oracle.qmax(bits)
+    assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)
+
+
+def test_ln_quant_refuses_what_it_cannot_do(env):
+    torch, hq = env
+    x = torch.zeros((64, 1152), device="cuda")
+    codes = torch.zeros((64, 1152), dtype=torch.uint8, device="cuda")
+    sc = torch.zeros((64,), device="cuda")
+    with pytest.raises(hq.HqError):                       # groups of 10 rows cannot be split over whole CTAs
+        hq.hq_ln_quant(x, None, None, 10, 1e-6, 128, 4, codes, 1, scales=sc)
+    with pytest.raises(hq.HqError):                       # a block size the fast kernel does not take
+        hq.hq_ln_quant(x, None, None, 0, 1e-6, 16, 4, codes, 1, scales=sc)
