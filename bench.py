@@ -450,11 +450,8 @@ def main_layer_list(args, which):
             for L in layers:
                 r = L["res"]
                 if L["name"] in ln_names:
-                    codes, sc = hq.workspace_views(r["ws"], L["M"], L["K"], CODES[0])
-                    hq.hq_ln_quant(r["x"], r["ln"]["w"], r["ln"]["b"], tokens, 1e-6, L["had_block"], A_BITS, codes, CODES[0],
-                                   scales=sc)
-                    hq.hq_qgemm(codes, CODES[0], A_BITS, L["K"], r["pw"], scale_a=sc, bias=r["bias"], alpha=r["pw"].alpha,
-                                y=r["y"], dev_status=status)
+                    hq.hq_ln_qlinear(r["x"], r["ln"]["w"], r["ln"]["b"], tokens, 1e-6, r["pw"], r["bias"], A_BITS, r["y"], r["ws"],
+                                     dev_status=status)
                 else:
                     hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
 
@@ -490,8 +487,7 @@ def main_layer_list(args, which):
         pl_us = 1e3 * t_of(lambda: hq.hq_hadamard_quant(rq["x"], Lq["had_block"], A_BITS, cq, CODES[0], scales=sq))
         ln_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(ln_names),
                         ln_quant_us=ln_us, plain_quant_us=pl_us,
-                        note="LayerNorm + per-sample modulation fused in front of the QKV and FC1 linears (hq_ln_quant + "
-                             "hq_qgemm for those layers; without the dependent launch of the fused layer call)")
+                        note="LayerNorm + per-sample modulation fused in front of the QKV and FC1 linears (hq_ln_qlinear)")
     macs = sum(L["macs"] for L in layers)
     ops_limbs = sum(2.0 * L["macs"] * L["res"]["pw"].desc.limbs for L in layers)
     print(json.dumps(dict(metric="forwards/s of " + label,

@@ -195,6 +195,13 @@ hq_status hq_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, i
                       hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                       int64_t ld_codes, float* scales, void* stream);
 
+/* The fused layer with that prologue: LayerNorm + affine -> transform -> quantize (one activation scale per row) ->
+ * integer product -> rescale.  Arguments as hq_ln_quant and hq_qlinear. */
+hq_status hq_ln_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx, const float* ln_weight,
+                        const float* ln_bias, int64_t rows_per_group, float eps, const hq_weight_desc* desc,
+                        const void* w_dev, const float* scale_w, const float* bias, int a_bits, void* y, hq_dtype ydt,
+                        int64_t ldy, void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* ---- GroupNorm + SiLU fused in front of the transform + quantization (no counterpart in the paper's equations:
  * the normalisation and activation that precede the quantized 3x3 convolutions of a UNet ResBlock, applied while the
  * activations are read, so that they make one trip through memory instead of three). ---------------------------------

@@ -25,7 +25,7 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
-           "hq_ln_quant"]
+           "hq_ln_quant", "hq_ln_qlinear"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -74,12 +74,14 @@ def _load():
     L.hq_gn_silu_quant.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, i32, i32, i32, p, p, i32, i64, p, p,
                                    C.c_size_t, p]
     L.hq_ln_quant.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, i32, i32, i32, p, p, i32, i64, p, p]
+    L.hq_ln_qlinear.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, C.POINTER(WeightDesc), p, p, p, i32, p, i32, i64,
+                                p, C.c_size_t, p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
                  "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
-                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant"):
+                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -264,6 +266,16 @@ def hq_ln_quant(x, weight, bias, rows_per_group: int, eps: float, had_block: int
     _check(lib.hq_ln_quant(_dptr(x), _dtype_code(x), rows, cols, x.stride(0), _dptr(weight), _dptr(bias), rows_per_group,
                            eps, had_block, bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0),
                            _dptr(scales), _stream(stream)), "hq_ln_quant")
+
+
+def hq_ln_qlinear(x, ln_weight, ln_bias, rows_per_group: int, eps: float, pw: PreparedWeight, bias, a_bits: int, y,
+                  workspace, dev_status=None, stream=None) -> None:
+    """The fused linear layer with LayerNorm + per-sample affine in front (per-row activation scales)."""
+    M, K = x.shape
+    _check(lib.hq_ln_qlinear(_dptr(x), _dtype_code(x), M, K, x.stride(0), _dptr(ln_weight), _dptr(ln_bias), rows_per_group,
+                             eps, C.byref(pw.desc), _dptr(pw.blob_dev), _dptr(pw.s_w_dev), _dptr(bias), a_bits, _dptr(y),
+                             _dtype_code(y), y.stride(0), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                             _dptr(dev_status), _stream(stream)), "hq_ln_qlinear")
 
 
 def hq_hadamard_quant_width(x, had_block_w: int, bits: int, static_scale, z, scale_out=None, stream=None) -> None:

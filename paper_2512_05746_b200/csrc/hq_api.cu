@@ -22,6 +22,10 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
                          float alpha, int32_t* acc_out, void* y, hq_dtype ydt, int32_t* dev_status, cudaStream_t st,
                          bool after_quant);
 
+hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
+                          const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
+                          hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
+                          float* scales, cudaStream_t st);
 hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                       int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
                                       cudaStream_t st);
@@ -89,6 +93,30 @@ extern "C" hq_status hq_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t 
     if (s != HQ_OK) return s;
     return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, mode == HQ_SCALE_STATIC, scale_w, bias,
                         hq_alpha_for(desc), nullptr, y, ydt, ldy, dev_status, st, true);
+}
+
+extern "C" hq_status hq_ln_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx, const float* ln_weight,
+                                   const float* ln_bias, int64_t rows_per_group, float eps, const hq_weight_desc* desc,
+                                   const void* w_dev, const float* scale_w, const float* bias, int a_bits, void* y,
+                                   hq_dtype ydt, int64_t ldy, void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                   void* stream) {
+    using namespace hq;
+    if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+    const hq_container cont = hq_container(desc->container);
+    size_t need = 0;
+    hq_status s = hq_workspace_size(M, K, cont, &need);
+    if (s != HQ_OK) return s;
+    if (ws_bytes < need) return HQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* codes = static_cast<unsigned char*>(workspace);
+    float* scales = reinterpret_cast<float*>(codes + scales_offset(M, K, cont));
+    const int64_t ldc = code_pitch(K, cont);
+    s = launch_ln_quant(x, xdt, M, K, ldx, ln_weight, ln_bias, rows_per_group, eps, desc->had_block, a_bits, HQ_SCALE_PER_ROW,
+                        nullptr, codes, cont, ldc, scales, st);
+    if (s != HQ_OK) return s;
+    return launch_qgemm(codes, cont, a_bits, M, K, ldc, desc, w_dev, scales, 0, scale_w, bias, hq_alpha_for(desc), nullptr,
+                        y, ydt, ldy, dev_status, st, true);
 }
 
 extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,

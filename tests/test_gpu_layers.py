@@ -128,3 +128,33 @@ def test_qconv_small_configuration(env, oracle, a_bits, static):
         y_own = oracle.conv2d_dequant_perpixel(qg, s_gpu, B, 1, 1, pw.s_w, b, pw.alpha)
     assert rel_err(y.float().cpu().numpy(), y_own) <= Y_BF16_RTOL
     assert rms_rel(y.float().cpu().numpy(), ref["y"]) <= Y_BF16_RTOL
+
+
+@pytest.mark.parametrize("M,K,N,n,rpg,container", [(512, 1152, 384, 128, 256, 1), (320, 512, 200, 512, 32, 0)])
+def test_ln_qlinear_layer(env, oracle, M, K, N, n, rpg, container):
+    """LayerNorm + per-sample affine -> transform -> quantize -> integer product -> rescale in one call: the output
+    equals the oracle's rescale of the integer product of the codes and scales the call left in its workspace, and the
+    whole layer follows the oracle chain (normalise, quantize, multiply) to the layers' end-to-end bound."""
+    torch, hq = env
+    rng = np.random.default_rng(M + K)
+    x = inputs.activations((M, K), outlier_count=max(1, K // 100), outlier_scale=8.0, seed=K) + np.float32(0.3)
+    groups = (M + rpg - 1) // rpg
+    lw = (1.0 + 0.2 * rng.standard_normal((groups, K))).astype(np.float32)
+    lb = (0.3 * rng.standard_normal((groups, K))).astype(np.float32)
+    w, b = inputs.weights((N, K), seed=N), inputs.bias(N, seed=N)
+    pw = hq.hq_weight_prepare(w, 4, n, hq.HQ_W_FOLDED, container).to_device()
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(M, K, container),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_ln_qlinear(torch.from_numpy(x).cuda(), torch.from_numpy(lw).cuda(), torch.from_numpy(lb).cuda(), rpg, 1e-6, pw,
+                     torch.from_numpy(b).cuda(), 4, y, ws, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, M, K, container)
+    B = hq.decode_blob(pw).reshape(N, K)
+    y_own = oracle.dequant(oracle.gemm_int(q_gpu, B), s_gpu, pw.s_w, b, pw.alpha)
+    y_gpu = y.float().cpu().numpy()
+    assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
+    xn = oracle.layernorm_affine(x, lw, lb, rows_per_group=rpg, eps=1e-6)
+    ref = oracle.qlinear(xn.astype(np.float32), w, b, a_bits=4, w_bits=4, had_block=n, weight_mode="folded")
+    assert rms_rel(y_gpu, ref["y"]) <= 1e-2
