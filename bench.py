@@ -408,12 +408,9 @@ def main_layer_list(args, which):
                 r = L["res"]
                 if L["name"] in gn_names:
                     g = r["gn"]
-                    rows = L["Nb"] * L["H"] * L["W"]
-                    codes, sc = hq.workspace_views(r["ws"], rows, L["C"], CODES[0])
-                    hq.hq_gn_silu_quant(r["x"], 32, g["gamma"], g["beta"], 1e-5, L["had_block"], A_BITS, codes, CODES[0],
-                                        g["scratch"], scales=sc[:1], static_scale=g["static"])
-                    hq.hq_qconv2d(codes, CODES[0], A_BITS, L["Nb"], L["H"], L["W"], L["C"], r["pw"], L["R"], L["R"], L["stride"],
-                                  L["pad"], scale_a=g["static"], bias=r["bias"], alpha=r["pw"].alpha, y=r["y"], dev_status=status)
+                    hq.hq_gn_silu_qconv(r["x"], 32, g["gamma"], g["beta"], 1e-5, r["pw"], L["R"], L["R"], L["stride"], L["pad"],
+                                        r["bias"], A_BITS, r["y"], r["ws"], g["scratch"], static_scale=g["static"],
+                                        dev_status=status)
                 elif L["kind"] == "conv":
                     hq.hq_qconv(r["x"], r["pw"], L["R"], L["R"], L["stride"], L["pad"], r["bias"], A_BITS, r["y"], r["ws"],
                                 static_scale=r["static"], dev_status=status)
@@ -432,7 +429,7 @@ def main_layer_list(args, which):
         hq.hq_check_status(status)
         gn_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(gn_layers),
                         note="GroupNorm(32) + SiLU fused in front of the residual-block 3x3 convolutions "
-                             "(hq_gn_silu_quant + hq_qconv2d for those layers)")
+                             "(hq_gn_silu_qconv)")
     # The transformer's QKV and FC1 linears take modulate(LayerNorm(x), shift, scale) as input: the same forward with that
     # prologue fused into the transform kernel of those layers (row statistics from the registers that hold the row).
     ln_extra = None

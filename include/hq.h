@@ -217,6 +217,16 @@ hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, i
                            hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                            int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, void* stream);
 
+/* The fused convolution layer with that prologue: GroupNorm + SiLU -> transform -> quantize -> integer convolution ->
+ * rescale.  Arguments as hq_gn_silu_quant and hq_qconv. */
+hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                           const float* gamma, const float* beta, float eps, const hq_weight_desc* desc,
+                           const void* w_dev, int R, int S, int stride, int pad, const float* scale_w,
+                           const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale, void* y,
+                           hq_dtype ydt, void* workspace, size_t ws_bytes, void* scratch, size_t scratch_bytes,
+                           int32_t* dev_status, void* stream);
+
+
 /* ---- Fused linear layer that allocates nothing and takes no workspace (the paper has no counterpart: this is a
  * packaging of hq_qlinear for a particular kind of caller, not another operation). ---------------------------------
  * Who it is for: code that must not, or cannot, obtain device memory at the moment it runs a layer -- an inference

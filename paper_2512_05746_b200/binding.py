@@ -25,7 +25,7 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
-           "hq_ln_quant", "hq_ln_qlinear"]
+           "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -76,12 +76,14 @@ def _load():
     L.hq_ln_quant.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, i32, i32, i32, p, p, i32, i64, p, p]
     L.hq_ln_qlinear.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, C.POINTER(WeightDesc), p, p, p, i32, p, i32, i64,
                                 p, C.c_size_t, p, p]
+    L.hq_gn_silu_qconv.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, C.POINTER(WeightDesc), p, i32, i32, i32,
+                                   i32, p, p, i32, i32, p, p, i32, p, C.c_size_t, p, C.c_size_t, p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
                  "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
-                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear"):
+                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -255,6 +257,19 @@ def hq_gn_silu_quant(x, groups: int, gamma, beta, eps: float, had_block: int, bi
                                 bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
                                 _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)),
            "hq_gn_silu_quant")
+
+
+def hq_gn_silu_qconv(x, groups: int, gamma, beta, eps: float, pw: PreparedWeight, R: int, S: int, stride: int, pad: int,
+                     bias, a_bits: int, y, workspace, scratch, static_scale=None, dev_status=None, stream=None) -> None:
+    """The fused convolution layer with GroupNorm + SiLU in front (x NHWC)."""
+    Nb, H, W, Cin = x.shape
+    mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    _check(lib.hq_gn_silu_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), eps,
+                                C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride, pad, _dptr(pw.s_w_dev), _dptr(bias),
+                                a_bits, mode, _dptr(static_scale), _dptr(y), _dtype_code(y), _dptr(workspace),
+                                workspace.numel() * workspace.element_size(), _dptr(scratch),
+                                scratch.numel() * scratch.element_size(), _dptr(dev_status), _stream(stream)),
+           "hq_gn_silu_qconv")
 
 
 def hq_ln_quant(x, weight, bias, rows_per_group: int, eps: float, had_block: int, bits: int, codes, container: int,

@@ -158,3 +158,40 @@ def test_ln_qlinear_layer(env, oracle, M, K, N, n, rpg, container):
     xn = oracle.layernorm_affine(x, lw, lb, rows_per_group=rpg, eps=1e-6)
     ref = oracle.qlinear(xn.astype(np.float32), w, b, a_bits=4, w_bits=4, had_block=n, weight_mode="folded")
     assert rms_rel(y_gpu, ref["y"]) <= 1e-2
+
+
+@pytest.mark.parametrize("container,static", [(1, True), (0, False)])
+def test_gn_silu_qconv_layer(env, oracle, container, static):
+    """GroupNorm(32) + SiLU -> transform -> quantize -> integer 3x3 convolution -> rescale in one call, with one static
+    scale or per-pixel scales: the output equals the oracle's rescale of the integer convolution of the codes and scales
+    the call left in its workspace, and the whole layer follows the oracle chain to the layers' end-to-end bound."""
+    torch, hq = env
+    rng = np.random.default_rng(7)
+    Nb, H, W, C, Cout, G = 2, 16, 16, 256, 128, 32
+    x = inputs.activations((Nb, H, W, C), outlier_count=3, outlier_scale=8.0, seed=11) + np.float32(0.5)
+    gamma = (1.0 + 0.2 * rng.standard_normal(C)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(C)).astype(np.float32)
+    w, b = inputs.weights((Cout, 3, 3, C), seed=5), inputs.bias(Cout, seed=5)
+    pw = hq.hq_weight_prepare(w, 4, 256, hq.HQ_W_FOLDED, container).to_device()
+    y = torch.zeros((Nb, H, W, Cout), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(Nb * H * W, C, container),), dtype=torch.uint8, device="cuda")
+    scratch = torch.zeros((Nb * G * 24,), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    xn = oracle.groupnorm_silu(x, G, gamma, beta, 1e-5).astype(np.float32)
+    s0 = float(np.float32(np.abs(oracle.transform(xn.reshape(-1, C), 256)).max() / 7.0)) if static else None
+    ss = torch.tensor([s0], dtype=torch.float32, device="cuda") if static else None
+    hq.hq_gn_silu_qconv(torch.from_numpy(x).cuda(), G, torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), 1e-5, pw,
+                        3, 3, 1, 1, torch.from_numpy(b).cuda(), 4, y, ws, scratch, static_scale=ss, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, Nb * H * W, C, container)
+    B = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    qg = q_gpu.reshape(Nb, H, W, C)
+    if static:
+        y_own = oracle.dequant(oracle.conv2d_int(qg, B, 1, 1), np.array([s0], np.float32), pw.s_w, b, pw.alpha)
+    else:
+        y_own = oracle.conv2d_dequant_perpixel(qg, s_gpu, B, 1, 1, pw.s_w, b, pw.alpha)
+    y_gpu = y.float().cpu().numpy()
+    assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
+    ref = oracle.qconv(xn, w, b, a_bits=4, w_bits=4, had_block=256, stride=1, pad=1, weight_mode="folded", static_scale=s0)
+    assert rms_rel(y_gpu, ref["y"]) <= 1e-2
