@@ -145,9 +145,8 @@ hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bits, int64_t
  * Codes and scales live in `workspace` (device, hq_workspace_size bytes); the code container is desc->container.
  * alpha is derived from the descriptor.  y pitch ldy elements.
  * The product kernel is launched so that it may begin (set-up, first weight tile) while the transform kernel is still
- * running; it waits for the transform before it touches codes or activation scales.  The weight blob, scale_w and bias
- * must therefore be complete in device memory when the call is made, not the output of work still in flight on the
- * stream (x may be: the transform kernel is ordered after earlier work in the usual way). */
+ * running; it waits for the transform before it touches codes or activation scales.  Work enqueued on the stream before
+ * the call has completed before either kernel starts, as usual. */
 hq_status hq_workspace_size(int64_t rows, int64_t cols, hq_container cont, size_t* bytes);
 hq_status hq_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx, const hq_weight_desc* desc,
                      const void* w_dev, const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
