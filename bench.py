@@ -48,6 +48,13 @@ def code_pitch(cols):
 
 def codes_name():
     return "nibble" if CODES[0] == 0 else "int8"
+
+
+def ws_views(torch, ws, rows, cols):
+    """Codes [rows, pitch] and scales [rows] inside the workspace of a fused layer call (the documented layout)."""
+    pitch = (code_pitch(cols) + 15) // 16 * 16
+    off = (rows * pitch + 255) // 256 * 256
+    return ws[: rows * pitch].view(rows, pitch), ws[off: off + rows * 4].view(torch.float32)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch at the full size of the default step, from the one-pass ncu
 # capture of this command (a summary is kept under profiles/; taken with these kernel versions: set an entry to
 # None when its kernel changes).  Outputs partly stay in L2 past the end of a launch, so these are below the
@@ -395,7 +402,7 @@ def main_layer_list(args, which):
             cin, rows = L["C"], L["Nb"] * L["H"] * L["W"]
             g = dict(gamma=torch.ones((cin,), device=dev), beta=torch.zeros((cin,), device=dev),
                      scratch=torch.empty((L["Nb"] * 32 * 24,), dtype=torch.uint8, device=dev))
-            codes, sc = hq.workspace_views(r["ws"], rows, cin, CODES[0])
+            codes, sc = ws_views(torch, r["ws"], rows, cin)
             hq.hq_gn_silu_quant(r["x"], 32, g["gamma"], g["beta"], 1e-5, L["had_block"], A_BITS, codes, CODES[0], g["scratch"],
                                 scales=sc)
             g["static"] = sc.max().reshape(1).contiguous()          # one static scale, calibrated on the normalised input
@@ -465,7 +472,7 @@ def main_layer_list(args, which):
         # the prologue alone against the plain transform on the block input (8192 x 1152 bf16)
         Lq = next(L for L in layers if L["name"].endswith(".qkv"))
         rq = Lq["res"]
-        cq, sq = hq.workspace_views(rq["ws"], Lq["M"], Lq["K"], CODES[0])
+        cq, sq = ws_views(torch, rq["ws"], Lq["M"], Lq["K"])
 
         def t_of(fn):
             for _ in range(5):

@@ -205,17 +205,6 @@ def hq_workspace_size(rows: int, cols: int, container: int) -> int:
     return int(out.value)
 
 
-def workspace_views(workspace, rows: int, cols: int, container: int):
-    """The codes [rows, pitch] (uint8) and scales [rows] (fp32) a fused call left in its workspace (pure slicing)."""
-    import torch
-    row_bytes = cols // 2 if container == HQ_CODES_NIBBLE else cols
-    pitch = (row_bytes + 15) // 16 * 16
-    off = (rows * pitch + 255) // 256 * 256
-    codes = workspace[: rows * pitch].view(rows, pitch)
-    scales = workspace[off: off + rows * 4].view(torch.float32)
-    return codes, scales
-
-
 def hq_qlinear(x, pw: PreparedWeight, bias, a_bits: int, y, workspace, static_scale=None, dev_status=None,
                stream=None) -> None:
     M, K = x.shape
@@ -312,25 +301,3 @@ def hq_qconv_width(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int,
 
 def hq_mma_i8_probe(ctas: int, iters: int, dev_status=None, stream=None) -> None:
     _check(lib.hq_mma_i8_probe(ctas, iters, _dptr(dev_status), _stream(stream)), "hq_mma_i8_probe")
-
-
-def decode_blob(pw: PreparedWeight) -> np.ndarray:
-    """Host-side inverse of the blob layout: returns the weight integers B as int32 [N, RS, C].
-    (A test and debugging aid: pure byte shuffling, no arithmetic beyond 256*hi + lo.)"""
-    d = pw.desc
-    Kp = d.RS * d.C_pad
-    rows = pw.blob[: d.N_pad * d.limbs * Kp].reshape(-1, Kp).astype(np.int32)
-    o = np.arange(d.N)
-    if d.limbs == 1:
-        full = rows[o]
-    else:
-        hi = rows[(o // 128) * 256 + (o % 128)]
-        lo = rows[(o // 128) * 256 + 128 + (o % 128)]
-        full = 256 * hi + lo
-    full = full.reshape(d.N, d.RS, d.C_pad)[:, :, : d.C]
-    if d.container == HQ_CODES_NIBBLE:
-        c = np.arange(d.C)
-        r = c & 7
-        slot = np.where(r & 1, 4 + (r >> 1), r >> 1)
-        full = full[:, :, (c & ~7) + slot]
-    return np.ascontiguousarray(full)

@@ -1,17 +1,18 @@
-// Fused online Hadamard transform + symmetric quantization (Eq. 10 with Eq. 5-7, then Eq. 3).
+// Fused online Hadamard transform + symmetric quantization (Eq. 10 with Eq. 5-7, then Eq. 3), and its variants.
 //
-// HBM-bound: every input element is read once (128-bit loads) and 0.5 or 1 byte is written.
-// Fast path (block size n = 2^k, k = 8..12): a block of n channels is owned by n/32 threads, each
-// holding 32 values in registers.
-//   phase A  thread t holds elements {4t + c + (n/8) i : c < 4, i < 8}: fully coalesced 16-byte loads;
-//            a 32-point in-register transform covers index bits {0, 1, k-3, k-2, k-1};
-//   exchange one trip through shared memory (XOR-swizzled, conflict-free both ways);
-//   phase B  thread t holds the 32 contiguous elements 32t .. 32t+31: in-register stages for bits {2,3,4},
-//            warp-shuffle stages for bits 5 .. k-4 (none for k = 8);
-//   then     |max| over the row (shuffles, plus a shared-memory max when a row spans several blocks or
-//            warps), scale, round-half-even by a magic-number add, clamp, pack, one 16-byte store per thread.
+// HBM-bound: every input element is read once (16-byte loads) and 0.5 or 1 byte is written.
+//   fwht_quant_fast     Hadamard blocks of n = 2^k channels, k = 5..12: a block is owned by n/E threads that hold E = 32
+//                       (64 for k >= 10) values each as two-wide fp32 registers; two in-register butterfly phases around
+//                       one trip through a padded shared-memory buffer cover all k stages (k = 12: one lane exchange
+//                       more); then the row maximum (shuffles, plus a shared-memory maximum when a row spans several
+//                       blocks or warps), the scale, round-half-even by a magic-number add, packing, 16-byte stores.
+//                       Optional prologues applied as the values are loaded: GroupNorm (+ SiLU) with given statistics,
+//                       or LayerNorm over the row with a per-sample affine.
+//   fwht_quant_generic  every other block size, including the identity: one row per CTA in shared memory.
+//   width_quant_kernel  the transform along the width axis of an NHWC tensor (Eq. 13-14 as stated), static scale,
+//                       followed by the integer factor q * H_raw.
+//   gn_stats_kernel / gn_finalize_kernel   per-(sample, group) statistics for the GroupNorm prologue.
 // The butterflies run unnormalised (H_raw); 2^(-k/2) is folded into the scale (Eq. 7).
-// A generic shared-memory kernel covers every other block size, including the identity (no transform).
 #include "hq_common.cuh"
 
 namespace hq {
@@ -63,48 +64,6 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
     f.z = __uint_as_float(raw.y << 16);
     f.w = __uint_as_float(raw.y & 0xFFFF0000u);
     return f;
-}
-
-template <int LO, int HI>
-__device__ __forceinline__ void butterflies(float (&v)[32]) {
-#pragma unroll
-    for (int h = LO; h <= HI; h <<= 1) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            if (!(i & h)) {
-                const float a = v[i], b = v[i | h];
-                v[i] = a + b;
-                v[i | h] = a - b;
-            }
-        }
-    }
-}
-
-// Round (ties to even), clamp and pack 32 values held by one thread; returns words through `out`.
-template <bool INT8_OUT>
-__device__ __forceinline__ void quantize_pack(const float (&v)[32], float inv, int bits, uint32_t* out) {
-    const float bias = INT8_OUT ? 128.0f : 8.0f;
-    const float mb = kMagic + bias;
-    const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
-    constexpr int PER_WORD = INT8_OUT ? 4 : 8;
-    constexpr int SHIFT = INT8_OUT ? 8 : 4;
-    // Each rounded value is kMagicBits + (code + bias); summing the shifted words and removing the shifted
-    // constants leaves the biased fields, which one XOR turns into two's complement.
-    uint32_t cst = 0;
-#pragma unroll
-    for (int e = 0; e < PER_WORD; ++e) cst += kMagicBits << (SHIFT * e);
-    constexpr uint32_t UNBIAS = INT8_OUT ? 0x80808080u : 0x88888888u;
-#pragma unroll
-    for (int w = 0; w < 32 / PER_WORD; ++w) {
-        uint32_t acc = 0;
-#pragma unroll
-        for (int e = 0; e < PER_WORD; ++e) {
-            float f = fmaf(v[w * PER_WORD + e], inv, mb);
-            f = fminf(fmaxf(f, lo), hi);
-            acc += __float_as_uint(f) << (SHIFT * e);
-        }
-        out[w] = (acc - cst) ^ UNBIAS;
-    }
 }
 
 // ---- two-wide fp32 arithmetic (one instruction for a pair of values held in a 64-bit register) -----------------

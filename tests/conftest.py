@@ -17,3 +17,19 @@ def oracle():
     import oracle as _o
     _o.lib()
     return _o
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """With HQ_PARITY_STATS=<file>, the measured mismatch fractions and tie distances of the code comparisons are
+    written there as JSON lines (the figures the tolerances of the normalisation prologues are set from)."""
+    path = os.environ.get("HQ_PARITY_STATS")
+    if not path:
+        return
+    import json
+    try:
+        from hq_testutil import PARITY_STATS
+    except ImportError:
+        return
+    with open(path, "w") as f:
+        for rec in PARITY_STATS:
+            f.write(json.dumps(rec) + "\n")

@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
+from hq_testutil import decode_blob
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -95,7 +96,7 @@ def test_weight_prepare_matches_oracle(hq, oracle, mode, container, shape, had_b
     pw = hq.hq_weight_prepare(w, w_bits, had_block, hq.WEIGHT_MODES[mode], container)
     B_ref, s_ref = oracle.prepare_weights(w.reshape(shape[0], -1, shape[-1]), w_bits, had_block, mode)
     assert np.array_equal(pw.s_w, s_ref)
-    assert np.array_equal(hq.decode_blob(pw), B_ref)
+    assert np.array_equal(decode_blob(pw), B_ref)
     d = pw.desc
     assert d.bytes == hq.hq_weight_blob_bytes(shape[0], d.RS, shape[-1], w_bits, had_block, hq.WEIGHT_MODES[mode])
     assert d.max_abs_b == np.abs(B_ref).max()
@@ -110,7 +111,7 @@ def test_weight_prepare_double_close_to_oracle(hq, oracle):
     pw = hq.hq_weight_prepare(w, 4, 512, hq.HQ_W_DOUBLE, hq.HQ_CODES_INT8)
     B_ref, s_ref = oracle.prepare_weights(w.reshape(64, 1, 512), 4, 512, "double")
     assert np.allclose(pw.s_w, s_ref, rtol=1e-6)
-    diff = hq.decode_blob(pw) != B_ref          # butterfly vs dense summation order: only exact ties may differ
+    diff = decode_blob(pw) != B_ref          # butterfly vs dense summation order: only exact ties may differ
     assert diff.mean() <= 1e-4
     assert pw.desc.limbs == 1 and pw.alpha == 1.0
 

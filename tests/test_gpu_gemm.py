@@ -4,7 +4,8 @@ import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
-from hq_testutil import Y_BF16_RTOL, Y_F32_RTOL, pack_nibbles_np, rel_err
+import hq_testutil as hqt
+from hq_testutil import Y_BF16_RTOL, Y_F32_RTOL, pack_nibbles_np, rel_err, weight_integers
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +31,7 @@ def gemm_case(torch, hq, oracle, M, K, N, a_bits, w_bits, had_block, mode, conta
     q = inputs.codes((M, K), a_bits, seed=seed)
     w = inputs.weights((N, K), seed=seed)
     pw = hq.hq_weight_prepare(w, w_bits, had_block, hq.WEIGHT_MODES[mode], container).to_device()
-    B_ref = hq.decode_blob(pw).reshape(N, K)
+    B_ref = weight_integers(oracle, pw, w, w_bits, had_block, mode)
     s_a = inputs.positive_scales(M, seed=seed)
     b = inputs.bias(N, seed=seed) if with_bias else None
     a_dev = to_container(torch, hq, q, container)
@@ -111,7 +112,7 @@ def test_qgemm_extreme_magnitudes(env, oracle):
     w[0, :] = -1.0                                                  # W_int = -7 everywhere -> B[0][0] = -7*1024
     for container in (0, 1):
         pw = hq.hq_weight_prepare(w, 4, 1024, hq.HQ_W_FOLDED, container).to_device()
-        B = hq.decode_blob(pw).reshape(N, K)
+        B = weight_integers(oracle, pw, w, 4, 1024, "folded")
         assert np.abs(B).max() >= 7 * 1024
         q = np.where(B[1] > 0, -8, 7).astype(np.int8)[None, :].repeat(M, axis=0)    # |acc| of channel 1 = sum |q||B|
         q[1::2] = -8
@@ -145,7 +146,7 @@ def test_qgemm_scalar_scale_and_determinism(env, oracle):
         hq.hq_qgemm(a, hq.HQ_CODES_NIBBLE, 4, K, pw, scale_a=s, alpha=pw.alpha, y=y)
         outs.append(y.cpu().numpy())
     assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
-    y_ref = oracle.dequant(oracle.gemm_int(q, hq.decode_blob(pw).reshape(N, K)), np.array([0.037], np.float32), pw.s_w,
+    y_ref = oracle.dequant(oracle.gemm_int(q, weight_integers(oracle, pw, w, 4, 512, "folded")), np.array([0.037], np.float32), pw.s_w,
                            None, pw.alpha)
     assert rel_err(outs[0], y_ref) <= Y_F32_RTOL
 
@@ -172,7 +173,7 @@ def test_qconv2d_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, a_bits, 
     q = inputs.codes((Nb, H, W, C), a_bits, seed=H + W + C)
     w = inputs.weights((Cout, R, R, C), seed=C + Cout)
     pw = hq.hq_weight_prepare(w, 4, hb, hq.WEIGHT_MODES[mode], container).to_device()
-    B_ref = hq.decode_blob(pw).reshape(Cout, R, R, C)
+    B_ref = weight_integers(oracle, pw, w, 4, hb, mode).reshape(Cout, R, R, C)
     b = inputs.bias(Cout, seed=1)
     Ho, Wo = H + 2 * pad - R + 1, W + 2 * pad - R + 1
     acc = torch.full((Nb, Ho, Wo, Cout), 777, dtype=torch.int32, device="cuda")
@@ -211,7 +212,7 @@ def test_qconv2d_stride2_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, pad, 
     q = inputs.codes((Nb, H, W, C), 4, seed=H + C)
     w = inputs.weights((Cout, R, R, C), seed=Cout)
     pw = hq.hq_weight_prepare(w, 4, 128, hq.WEIGHT_MODES[mode], container).to_device()
-    B_ref = hq.decode_blob(pw).reshape(Cout, R, R, C)
+    B_ref = weight_integers(oracle, pw, w, 4, 128, mode).reshape(Cout, R, R, C)
     Ho, Wo = (H + 2 * pad - R) // 2 + 1, (W + 2 * pad - R) // 2 + 1
     acc = torch.full((Nb, Ho, Wo, Cout), 777, dtype=torch.int32, device="cuda")
     y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.float32, device="cuda")
@@ -246,7 +247,7 @@ def test_qconv2d_per_pixel_scales(env, oracle, Nb, H, W, C, Cout, stride, a_bits
     q = inputs.codes((Nb, H, W, C), a_bits, seed=H + W + C + a_bits)
     w = inputs.weights((Cout, 3, 3, C), seed=Cout)
     pw = hq.hq_weight_prepare(w, 4, 128, hq.WEIGHT_MODES[mode], container).to_device()
-    B_ref = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    B_ref = weight_integers(oracle, pw, w, 4, 128, mode).reshape(Cout, 3, 3, C)
     b = inputs.bias(Cout, seed=3)
     s_a = inputs.positive_scales(Nb * H * W, seed=7)
     Ho, Wo = (H + 2 - 3) // stride + 1, (W + 2 - 3) // stride + 1
@@ -269,3 +270,33 @@ def test_int8_tensor_pipe_probe_runs(env):
     hq.hq_mma_i8_probe(4, 64, dev_status=status)
     torch.cuda.synchronize()
     hq.hq_check_status(status)
+
+
+def test_qgemm_sweep_corner_sampled(env, oracle):
+    """The largest point of the shape sweep, 65536 x 4096 x 4096 with the folded two-limb weights of a 4096-point
+    block: int32 accumulators of sampled rows and output channels (first and last of each axis included) against the
+    oracle's integer product.  The codes are drawn on the device (seeded); the sampled rows are copied back."""
+    torch, hq = env
+    M, K, N = 65536, 4096, 4096
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(7)
+    a = torch.randint(-8, 8, (M, K), generator=gen, device="cuda", dtype=torch.int8)
+    w = inputs.weights((N, K), seed=4096)
+    pw = hq.hq_weight_prepare(w, 4, K, hq.HQ_W_FOLDED, hq.HQ_CODES_INT8).to_device()
+    assert pw.desc.limbs == 2
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qgemm(a.view(torch.uint8), hq.HQ_CODES_INT8, 4, K, pw, acc_out=acc, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    rng = np.random.default_rng(3)
+    rows = np.sort(np.concatenate(([0, 127, 128, M - 1], rng.choice(M, size=60, replace=False))))
+    cols = np.sort(np.concatenate(([0, 127, 128, N - 1], rng.choice(N, size=60, replace=False))))
+    w_int, _ = oracle.weight_quantize(w[cols], 4)
+    B = oracle.weight_fold(w_int, K)                                  # exact integers, only the sampled channels
+    assert np.array_equal(B, hqt.decode_blob(pw).reshape(N, K)[cols])
+    ridx = torch.from_numpy(rows).cuda()
+    q = a[ridx].cpu().numpy()
+    ref = oracle.gemm_int(q, B)
+    got = acc[ridx][:, torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.int64)
+    assert np.array_equal(got, ref)

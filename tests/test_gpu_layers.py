@@ -9,7 +9,8 @@ import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
-from hq_testutil import SCALE_RTOL, Y_BF16_RTOL, check_codes, rel_err, unpack_nibbles_np
+from hq_testutil import (SCALE_RTOL, Y_BF16_RTOL, check_codes, rel_err, unpack_nibbles_np, weight_integers,
+                         workspace_views)
 
 pytestmark = pytest.mark.gpu
 
@@ -29,7 +30,7 @@ def env():
 
 
 def _codes_from_ws(hq, ws, rows, cols, container):
-    codes, scales = hq.workspace_views(ws, rows, cols, container)
+    codes, scales = workspace_views(ws, rows, cols, container)
     c = codes.cpu().numpy()
     q = unpack_nibbles_np(c[:, : cols // 2]) if container == hq.HQ_CODES_NIBBLE else c[:, :cols].view(np.int8)
     return q, scales.cpu().numpy()
@@ -51,8 +52,7 @@ def run_linear(torch, hq, oracle, x, w, b, a_bits, had_block, mode, container, r
     ref = oracle.qlinear(x[idx], w, b, a_bits=a_bits, w_bits=4, had_block=had_block, weight_mode=mode)
     assert np.allclose(s_gpu[idx], ref["s_a"], rtol=SCALE_RTOL, atol=0)
     check_codes(q_gpu[idx], ref["q"], ref["v"], "fused linear")
-    B = hq.decode_blob(pw).reshape(N, K)
-    assert np.array_equal(B, ref["B"].reshape(N, K))
+    B = weight_integers(oracle, pw, w, 4, had_block, mode)
     y_own = oracle.dequant(oracle.gemm_int(q_gpu[idx], B), s_gpu[idx], pw.s_w, b, pw.alpha)
     y_gpu = y.float().cpu().numpy()[idx]
     assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
@@ -120,7 +120,7 @@ def test_qconv_small_configuration(env, oracle, a_bits, static):
     else:
         assert np.allclose(s_gpu, ref["s_a"], rtol=SCALE_RTOL, atol=0)
     check_codes(q_gpu, ref["q"].reshape(-1, C), v, "fused conv")
-    B = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    B = weight_integers(oracle, pw, w, 4, 256, "folded").reshape(Cout, 3, 3, C)
     qg = q_gpu.reshape(Nb, H, W, C)
     if static:
         y_own = oracle.dequant(oracle.conv2d_int(qg, B, 1, 1), np.array([s0], np.float32), pw.s_w, b, pw.alpha)
@@ -151,7 +151,7 @@ def test_ln_qlinear_layer(env, oracle, M, K, N, n, rpg, container):
     torch.cuda.synchronize()
     hq.hq_check_status(status)
     q_gpu, s_gpu = _codes_from_ws(hq, ws, M, K, container)
-    B = hq.decode_blob(pw).reshape(N, K)
+    B = weight_integers(oracle, pw, w, 4, n, "folded")
     y_own = oracle.dequant(oracle.gemm_int(q_gpu, B), s_gpu, pw.s_w, b, pw.alpha)
     y_gpu = y.float().cpu().numpy()
     assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
@@ -185,7 +185,7 @@ def test_gn_silu_qconv_layer(env, oracle, container, static):
     torch.cuda.synchronize()
     hq.hq_check_status(status)
     q_gpu, s_gpu = _codes_from_ws(hq, ws, Nb * H * W, C, container)
-    B = hq.decode_blob(pw).reshape(Cout, 3, 3, C)
+    B = weight_integers(oracle, pw, w, 4, 256, "folded").reshape(Cout, 3, 3, C)
     qg = q_gpu.reshape(Nb, H, W, C)
     if static:
         y_own = oracle.dequant(oracle.conv2d_int(qg, B, 1, 1), np.array([s0], np.float32), pw.s_w, b, pw.alpha)
@@ -195,3 +195,71 @@ def test_gn_silu_qconv_layer(env, oracle, container, static):
     assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
     ref = oracle.qconv(xn, w, b, a_bits=4, w_bits=4, had_block=256, stride=1, pad=1, weight_mode="folded", static_scale=s0)
     assert rms_rel(y_gpu, ref["y"]) <= 1e-2
+
+
+def test_qconv_benchmark_configuration_sampled_images(env, oracle):
+    """The 3x3 convolution as the benchmark step runs it: batch 32 (32768 pixels), one code per byte, one static
+    activation scale calibrated as the largest per-pixel scale, bf16 output.  Three sampled images (a convolution
+    with zero padding never looks across images) go through the whole oracle layer."""
+    torch, hq = env
+    cfg = inputs.config_conv_small(0, batch=32)
+    x, w, b = cfg["x"], cfg["w"], cfg["bias"]
+    Nb, H, W, C = x.shape
+    Cout = w.shape[0]
+    cont = hq.HQ_CODES_INT8
+    pw = hq.hq_weight_prepare(w, 4, 256, hq.HQ_W_FOLDED, cont).to_device()
+    xd = torch.from_numpy(x).cuda()
+    codes = torch.empty((Nb * H * W, C), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((Nb * H * W,), dtype=torch.float32, device="cuda")
+    hq.hq_hadamard_quant(xd.view(-1, C), 256, 4, codes, cont, scales=sc)
+    static = sc.max().reshape(1).contiguous()
+    s0 = float(static.cpu()[0])
+    y = torch.zeros((Nb, H, W, Cout), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(Nb * H * W, C, cont),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qconv(xd, pw, 3, 3, 1, 1, torch.from_numpy(b).cuda(), 4, y, ws, static_scale=static, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    q_all, s_gpu = _codes_from_ws(hq, ws, Nb * H * W, C, cont)
+    assert s_gpu[0] == np.float32(s0)
+    q_all = q_all.reshape(Nb, H, W, C)
+    imgs = [0, 13, Nb - 1]
+    ref = oracle.qconv(x[imgs], w, b, a_bits=4, w_bits=4, had_block=256, stride=1, pad=1, weight_mode="folded",
+                       static_scale=s0)
+    # the calibrated scale equals the largest per-pixel scale of the oracle's dynamic quantizer on the whole tensor
+    s_dyn = oracle.quantize(oracle.transform(x.reshape(-1, C), 256), 4)[1]
+    assert np.isclose(s0, s_dyn.max(), rtol=SCALE_RTOL, atol=0)
+    check_codes(q_all[imgs].reshape(-1, C), ref["q"].reshape(-1, C), ref["v"].reshape(-1, C), "bench conv, static scale")
+    B = weight_integers(oracle, pw, w, 4, 256, "folded").reshape(Cout, 3, 3, C)
+    y_own = oracle.dequant(oracle.conv2d_int(q_all[imgs], B, 1, 1), np.array([s0], np.float32), pw.s_w, b, pw.alpha)
+    y_gpu = y.float().cpu().numpy()[imgs]
+    assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
+    assert rms_rel(y_gpu, ref["y"]) <= Y_BF16_RTOL
+
+
+@pytest.mark.parametrize("M,K,N,n", [(1000, 512, 384, 512), (300, 1024, 200, 256)])
+def test_qlinear_w8a8(env, oracle, M, K, N, n):
+    """The fused layer at W8A8: 8-bit codes in the one-byte container, 8-bit Double-Hadamard weights Q(H^T W)
+    (one limb), online transform in front."""
+    torch, hq = env
+    x = inputs.activations((M, K), outlier_count=max(1, K // 100), outlier_scale=20.0, seed=M + K)
+    w, b = inputs.weights((N, K), seed=N), inputs.bias(N, seed=N)
+    cont = hq.HQ_CODES_INT8
+    pw = hq.hq_weight_prepare(w, 8, n, hq.HQ_W_DOUBLE, cont).to_device()
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(M, K, cont),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qlinear(torch.from_numpy(x).cuda(), pw, torch.from_numpy(b).cuda(), 8, y, ws, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, M, K, cont)
+    ref = oracle.qlinear(x, w, b, a_bits=8, w_bits=8, had_block=n, weight_mode="double")
+    assert np.allclose(s_gpu, ref["s_a"], rtol=SCALE_RTOL, atol=0)
+    check_codes(q_gpu, ref["q"], ref["v"], "fused linear W8A8")
+    B = weight_integers(oracle, pw, w, 8, n, "double")
+    y_own = oracle.dequant(oracle.gemm_int(q_gpu, B), s_gpu, pw.s_w, b, pw.alpha)
+    y_gpu = y.float().cpu().numpy()
+    assert rel_err(y_gpu, y_own) <= Y_BF16_RTOL
+    # with 8 bits on both sides the Double-Hadamard layer is close to the float product
+    xw = x.astype(np.float64) @ w.astype(np.float64).T + b
+    assert rms_rel(y_gpu, xw) <= 2e-2

@@ -1,18 +1,20 @@
 """GPU parity of GroupNorm + SiLU fused in front of the transform + quantization (hq_gn_silu_quant) against the CPU
-oracle.  The prologue runs in fp32 with the hardware's fast exponential and division, so the values that get
-quantized carry a relative error of a few 1e-6; codes may therefore differ from the oracle's by one where the oracle's
-pre-rounding value lies within GN_TIE_REL of the row's full scale from a rounding boundary."""
+oracle.  The prologue runs in fp32 with the hardware's fast exponential and division; the transform that follows sums
+a whole block of such values, over which their independent errors average out, so the codes are held to the same rule
+as the plain kernel's (one step of difference only within 1e-6 of the row's full scale from a rounding boundary, for at
+most 1e-4 of the codes) and the scales to the same 1e-6.  Measured on these cases: no differing code in 1.0 M codes
+(GroupNorm) and 2.9e-6 of the codes at a tie distance of 1.5e-8 (LayerNorm); scales within 2.4e-7."""
 import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
-from hq_testutil import unpack_nibbles_np
+from hq_testutil import CODE_MISMATCH_FRAC, CODE_TIE_REL, PARITY_STATS, check_codes, unpack_nibbles_np
 
 pytestmark = pytest.mark.gpu
 
-GN_TIE_REL = 2e-5          # 20x the plain kernel's window: fp32 normalisation + fast exp / divide in front of it
-GN_MISMATCH_FRAC = 2e-3
-GN_SCALE_RTOL = 2e-5
+GN_TIE_REL = CODE_TIE_REL
+GN_MISMATCH_FRAC = CODE_MISMATCH_FRAC
+GN_SCALE_RTOL = 1e-6
 
 
 @pytest.fixture(scope="module")
@@ -59,23 +61,19 @@ def test_gn_silu_quant_matches_oracle(env, oracle, Nb, H, W, C, G, n, bits, dt, 
         assert float(scales.cpu()[0]) == np.float32(s0)
         v = np.clip(v, oracle.qmin(bits) - 0.25, oracle.qmax(bits) + 0.25)
     else:
-        assert np.allclose(scales.cpu().numpy(), s_ref, rtol=GN_SCALE_RTOL, atol=0)
-    bad = q != q_ref
-    if bad.any():
-        assert np.abs(q.astype(np.int32) - q_ref)[bad].max() == 1
-        assert bad.mean() <= GN_MISMATCH_FRAC
-        full = np.maximum(np.abs(v).max(axis=1, keepdims=True), 1.0)
-        dist = np.abs(v - (np.floor(v) + 0.5))
-        assert np.all(dist[bad] <= (GN_TIE_REL * np.broadcast_to(full, v.shape))[bad])
+        dev = float(np.abs(scales.cpu().numpy() / s_ref - 1.0).max())
+        PARITY_STATS.append(dict(what=f"groupnorm prologue scales {Nb}x{H}x{W}x{C} {dt}", max_scale_rel=dev))
+        assert dev <= GN_SCALE_RTOL
+    check_codes(q, q_ref, v, f"groupnorm prologue {Nb}x{H}x{W}x{C} {dt}", tie_rel=GN_TIE_REL, mismatch_frac=GN_MISMATCH_FRAC)
     # the dequantized values are the normalised, activated, transformed input within half a step (Eq. 3)
     s_gpu = scales.cpu().numpy()[:, None] if not static else np.float32(s0)
     inside = np.abs(v) < oracle.qmax(bits)
     assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)
 
 
-LN_TIE_REL = 1e-5          # fp32 row statistics (sums of up to 4608 values) and rsqrt in front of the plain kernel's window
-LN_MISMATCH_FRAC = 1e-3
-LN_SCALE_RTOL = 1e-5
+LN_TIE_REL = CODE_TIE_REL
+LN_MISMATCH_FRAC = CODE_MISMATCH_FRAC
+LN_SCALE_RTOL = 1e-6
 
 
 @pytest.mark.parametrize("rows,cols,n,rpg,bits,dt,cont,static,affine", [
@@ -115,14 +113,10 @@ def test_ln_quant_matches_oracle(env, oracle, rows, cols, n, rpg, bits, dt, cont
         assert float(scales.cpu()[0]) == np.float32(s0)
         v = np.clip(v, oracle.qmin(bits) - 0.25, oracle.qmax(bits) + 0.25)
     else:
-        assert np.allclose(scales.cpu().numpy(), s_ref, rtol=LN_SCALE_RTOL, atol=0)
-    bad = q != q_ref
-    if bad.any():
-        assert np.abs(q.astype(np.int32) - q_ref)[bad].max() == 1
-        assert bad.mean() <= LN_MISMATCH_FRAC
-        full = np.maximum(np.abs(v).max(axis=1, keepdims=True), 1.0)
-        dist = np.abs(v - (np.floor(v) + 0.5))
-        assert np.all(dist[bad] <= (LN_TIE_REL * np.broadcast_to(full, v.shape))[bad])
+        dev = float(np.abs(scales.cpu().numpy() / s_ref - 1.0).max())
+        PARITY_STATS.append(dict(what=f"layernorm prologue scales {rows}x{cols} {dt}", max_scale_rel=dev))
+        assert dev <= LN_SCALE_RTOL
+    check_codes(q, q_ref, v, f"layernorm prologue {rows}x{cols} {dt}", tie_rel=LN_TIE_REL, mismatch_frac=LN_MISMATCH_FRAC)
     s_gpu = scales.cpu().numpy()[:, None] if not static else np.float32(s0)
     inside = np.abs(v) < oracle.qmax(bits)
     assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)

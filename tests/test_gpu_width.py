@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
-from hq_testutil import CODE_MISMATCH_FRAC, CODE_TIE_REL, Y_BF16_RTOL, Y_F32_RTOL, rel_err
+from hq_testutil import CODE_MISMATCH_FRAC, CODE_TIE_REL, PARITY_STATS, Y_BF16_RTOL, Y_F32_RTOL, decode_blob, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -66,11 +66,16 @@ def test_width_quant_matches_oracle(env, oracle, Nb, H, W, C, n, bits, dt):
     z_gpu = z.cpu().numpy()
     q_gpu = codes_from_z(z_gpu, n, closed_form_H(n)) if n > 1 else z_gpu.astype(np.int64)
     bad = q_gpu != q_ref
-    if bad.any():                                             # only rounding ties may differ, by one
+    # Only rounding ties may differ, by one.  One static scale serves the whole tensor and the largest values are
+    # clamped, so the full scale the fp32 error of a pre-rounding value is proportional to is the UNCLAMPED maximum
+    # of |v| (2.5 x qmax here), not the clamp range.
+    full = max(float(np.abs(v).max()), 1.0)
+    dist = np.abs(v - (np.floor(v) + 0.5))
+    PARITY_STATS.append(dict(what=f"width-axis {Nb}x{H}x{W}x{C} n={n} b={bits} {dt}", codes=int(q_ref.size),
+                             mismatch_frac=float(bad.mean()), max_tie_rel=float((dist[bad] / full).max()) if bad.any() else 0.0))
+    if bad.any():
         assert np.abs(q_gpu - q_ref)[bad].max() == 1 and bad.mean() <= CODE_MISMATCH_FRAC
-        vc = np.clip(v, oracle.qmin(bits) - 0.25, oracle.qmax(bits) + 0.25)
-        full = max(float(np.abs(vc).max()), 1.0)
-        assert np.all(np.abs(vc - (np.floor(vc) + 0.5))[bad] <= CODE_TIE_REL * full * 8)
+        assert np.all(dist[bad] <= CODE_TIE_REL * full)
     assert np.array_equal(z_gpu.astype(np.int64), oracle.codes_inverse_width(q_gpu.astype(np.int8), n).astype(np.int64))
     assert q_gpu.min() == oracle.qmin(bits) and q_gpu.max() == oracle.qmax(bits)
     assert np.isclose(float(so.cpu()[0]), np.float32(S) * 2.0 ** (-0.5 * np.log2(n)), rtol=1e-6)
@@ -102,8 +107,8 @@ def test_qconv_width_layer_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, str
     # the device's own integer activations (they may differ from the oracle's at rounding ties) -> oracle conv + rescale
     z_gpu = ws[: Nb * H * W * C].view(torch.int8).cpu().numpy().reshape(Nb, H, W, C)
     assert (z_gpu.astype(np.int64) != ref["z"]).mean() <= 16 * CODE_MISMATCH_FRAC
-    B = hq.decode_blob(pw).reshape(Cout, R, R, C)
-    assert np.array_equal(B, ref["B"]) and np.array_equal(pw.s_w, ref["s_w"])
+    B = ref["B"]
+    assert np.array_equal(decode_blob(pw).reshape(Cout, R, R, C), B) and np.array_equal(pw.s_w, ref["s_w"])
     y_own = oracle.dequant(oracle.conv2d_int_z(z_gpu.astype(np.int32), B, stride, pad), ref["s_a"], pw.s_w, b, ref["alpha"])
     assert rel_err(y.float().cpu().numpy(), y_own) <= (Y_BF16_RTOL if odt == "bf16" else Y_F32_RTOL)
     rms = np.sqrt(np.mean((y.float().cpu().numpy() - ref["y"]) ** 2)) / np.sqrt(np.mean(ref["y"] ** 2))

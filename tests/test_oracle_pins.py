@@ -515,3 +515,30 @@ def test_layernorm_affine_against_library_routine(oracle):
     assert np.allclose(moved, oracle.layernorm_affine(x, 1.0 + scale, shift, rows_per_group=rpg, eps=1e-12), atol=1e-9)
     with pytest.raises(ValueError):
         oracle.layernorm_affine(x, scale[:2], shift, rows_per_group=rpg)          # 12 rows in groups of 4 need 3 vectors
+
+
+# ------------------------------------------------------------------ Single vs Double Hadamard on the weight side
+
+def test_double_hadamard_raises_error_of_low_outlier_weights_and_lowers_it_for_outlier_weights(oracle):
+    """Direction of the "Single Hadamard Transformation" paragraph and of Table 6 on synthetic weights: transforming
+    weights that have few outliers (bounded, or a flat component: Eq. 16) adds outliers and raises their 4-bit
+    quantization error, and with it the layer error of the Double scheme; weights that do have outlier input channels
+    gain from the transform; iid Gaussian weights are indifferent.  A transform applied along the wrong weight axis,
+    or a Double scheme that reuses the scales of W, changes these directions."""
+    from oracle import weight_error_study as st
+    rows = {r["family"]: r for r in st.study(w_bits=4, a_bits=4, had_block=256)}
+    g, u, o, x = rows["gaussian"], rows["uniform"], rows["offset"], rows["outlier-in"]
+    assert 0.9 < g["werr_double"] / g["werr_single"] < 1.1
+    assert abs(g["layer_double"] - g["layer_single"]) < 0.05 * g["layer_single"]
+    for r in (u, o):
+        assert r["werr_double"] > 2.0 * r["werr_single"]
+        assert r["layer_double"] > 1.2 * r["layer_single"]
+        assert r["after"]["kurtosis"] > r["before"]["kurtosis"]
+        assert r["after"]["max_over_sigma"] > 1.5 * r["before"]["max_over_sigma"]
+    assert u["before"]["beyond_3sigma"] == 0.0 and u["after"]["beyond_3sigma"] > 1e-3
+    assert x["werr_double"] < 0.2 * x["werr_single"]
+    assert x["layer_double"] < 0.5 * x["layer_single"]
+    # Eq. 16 on the weight side: the flat component c * 1 of a channel lands in one coefficient, c * 2^(k/2)
+    w = st.make_weights("offset")
+    hw = oracle.transform(w.astype(np.float64), 256)
+    assert np.allclose(hw[:, 0], 16.0 * w.astype(np.float64).mean(axis=1), rtol=1e-12, atol=1e-12)

@@ -39,6 +39,9 @@ def _both_ways(torch, hq, M, K, N, had_block, container, ydtype, seed, static=No
     hq.hq_qlinear_noalloc(x, pw, b, 4, y, static_scale=ss, dev_status=status)
     torch.cuda.synchronize()
     hq.hq_check_status(status)
+    # the two entry points run the same kernels on the same inputs: beyond the tolerances below, the outputs must
+    # be the same bits (left-over bytes of an earlier call that leaked into this one would show here first)
+    assert torch.equal(y, y_ref), "hq_qlinear_noalloc and hq_qlinear differ"
     return y.float().cpu().numpy(), y_ref.float().cpu().numpy().astype(np.float64)
 
 
@@ -54,6 +57,35 @@ def test_noalloc_matches_workspace_version_twice_in_a_row(env):
     # and the first shape again, so stale bytes of a smaller call sit under a larger one
     y, y_ref = _both_ways(torch, hq, 4096, 2048, 384, 2048, hq.HQ_CODES_NIBBLE, torch.bfloat16, seed=3)
     assert rel_err(y, y_ref) <= Y_BF16_RTOL
+
+
+def test_noalloc_layer_that_fills_the_array_to_its_last_bytes(env):
+    """8160 rows of 1024 one-byte codes plus their 8160 scales need 8388480 of the 8388608 bytes: the scales sit at the
+    very end of the array, and one more row would not fit."""
+    torch, hq = env
+    M, K, N = 8160, 1024, 136
+    assert hq.HQ_NOALLOC_SCRATCH_BYTES - 128 == hq.hq_workspace_size(M, K, hq.HQ_CODES_INT8)
+    assert hq.hq_workspace_size(M + 1, K, hq.HQ_CODES_INT8) > hq.HQ_NOALLOC_SCRATCH_BYTES
+    y, y_ref = _both_ways(torch, hq, M, K, N, 1024, hq.HQ_CODES_INT8, torch.bfloat16, seed=4)
+    assert rel_err(y, y_ref) <= Y_BF16_RTOL
+
+
+def test_noalloc_call_takes_no_device_memory(env):
+    """What the entry point is for: once the library is loaded and the first call on the device has been made, a
+    call leaves the amount of free device memory where it was."""
+    torch, hq = env
+    M, K, N = 2048, 512, 256
+    x = torch.from_numpy(inputs.activations((M, K), outlier_count=2, outlier_scale=20.0, seed=5)).cuda()
+    pw = hq.hq_weight_prepare(inputs.weights((N, K), seed=5), 4, 512, hq.HQ_W_FOLDED, hq.HQ_CODES_INT8).to_device()
+    y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    hq.hq_qlinear_noalloc(x, pw, None, 4, y)                    # first call on the device: resolves the array's address
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        hq.hq_qlinear_noalloc(x, pw, None, 4, y)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after >= free_before, f"free device memory fell by {free_before - free_after} bytes"
 
 
 def test_noalloc_refuses_layers_beyond_its_array(env):
