@@ -25,3 +25,25 @@ def test_reference_arm_prints_one_contract_line():
     e2e = d["e2e"]
     assert e2e["value"] == d["value"] and e2e["unit"] == d["unit"]
     assert e2e["h2d_bytes_per_step"] == 0 and e2e["d2h_bytes_per_step"] == 0
+
+
+def test_gpus_flag_forms_a_one_rank_per_gpu_launch():
+    """`bench.py --gpus N` started by hand re-launches itself with one rank per GPU on the loopback address."""
+    sys.path.insert(0, ROOT)
+    import importlib
+    bench = importlib.import_module("bench")
+    cmd = bench.launch_command(4, ["--gpus", "4", "--steps", "3", "--warmup", "3"], port=29511)
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nnodes=1" in cmd and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29511"
+    i = cmd.index(os.path.join(ROOT, "bench.py"))
+    assert cmd[i + 1:] == ["--gpus", "4", "--steps", "3", "--warmup", "3"]
+    free = bench.launch_command(2, [])
+    assert 1024 < int(free[free.index("--master-port") + 1]) < 65536
+
+
+def test_gpus_flag_fails_loudly_without_enough_devices():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=300, cwd=ROOT,
+                         env={k: v for k, v in os.environ.items() if k != "WORLD_SIZE"})
+    assert out.returncode != 0 and "CUDA device" in (out.stderr + out.stdout)
