@@ -61,6 +61,11 @@ def lib():
             L.hqo_codes_inverse_width.argtypes = [p, i64, i64, i64, i64, C.c_int, p]
             L.hqo_conv2d_int_z.argtypes = [p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int, C.c_int, C.c_int, p]
             L.hqo_conv2d_int_z.restype = i64
+            L.hqo_groupnorm.argtypes = [p, i64, i64, i64, i64, C.c_int, p, p, C.c_double, C.c_int, p]
+            L.hqo_attention.argtypes = [p, i64, i64, i64, C.c_int, p]
+            L.hqo_upsample_nearest2x.argtypes = [p, i64, i64, i64, i64, p]
+            L.hqo_timestep_embedding.argtypes = [p, i64, i64, C.c_double, p]
+            L.hqo_conv2d_float.argtypes = [p, p, p, i64, i64, i64, i64, i64, C.c_int, C.c_int, C.c_int, C.c_int, p]
             _lib = L
     return _lib
 
@@ -267,6 +272,64 @@ def layernorm_affine(x, weight=None, bias=None, rows_per_group: int = 0, eps: fl
     _chk(lib().hqo_layernorm_affine(_ptr(x), rows, cols, _ptr(w) if w is not None else None,
                                     _ptr(b) if b is not None else None, int(rows_per_group), float(eps), _ptr(out)),
          "layernorm_affine")
+    return out
+
+
+def groupnorm(x, groups: int, gamma, beta, eps: float = 1e-5, act: str = "none") -> np.ndarray:
+    """GroupNorm of an NHWC tensor with the activation selectable ("none" or "silu"); fp64."""
+    x = _c(x, np.float64)
+    Nb, H, W, Cc = x.shape
+    gamma, beta = _c(gamma, np.float64), _c(beta, np.float64)
+    out = np.empty_like(x)
+    _chk(lib().hqo_groupnorm(_ptr(x), Nb, H, W, Cc, groups, _ptr(gamma), _ptr(beta), float(eps),
+                             {"none": 0, "silu": 1}[act], _ptr(out)), "groupnorm")
+    return out
+
+
+def silu(x) -> np.ndarray:
+    """x * sigmoid(x), fp64."""
+    x = np.asarray(x, np.float64)
+    return x / (1.0 + np.exp(-x))
+
+
+def attention(qkv, heads: int) -> np.ndarray:
+    """Self-attention core on qkv [Nb, L, 3C] (query | key | value column thirds, heads contiguous inside each):
+    softmax(q k^T / sqrt(dh)) v per sample and head -> [Nb, L, C]; fp64."""
+    qkv = _c(qkv, np.float64)
+    Nb, L, C3 = qkv.shape
+    Cc = C3 // 3
+    assert 3 * Cc == C3
+    out = np.empty((Nb, L, Cc), np.float64)
+    _chk(lib().hqo_attention(_ptr(qkv), Nb, L, Cc, heads, _ptr(out)), "attention")
+    return out
+
+
+def upsample_nearest2x(x) -> np.ndarray:
+    x = _c(x, np.float64)
+    Nb, H, W, Cc = x.shape
+    out = np.empty((Nb, 2 * H, 2 * W, Cc), np.float64)
+    _chk(lib().hqo_upsample_nearest2x(_ptr(x), Nb, H, W, Cc, _ptr(out)), "upsample_nearest2x")
+    return out
+
+
+def timestep_embedding(t, dim: int, max_period: float = 10000.0) -> np.ndarray:
+    """[cos(t f_i) | sin(t f_i)], f_i = max_period^(-i / (dim/2)); t [Nb] -> [Nb, dim]; fp64."""
+    t = _c(t, np.float64).reshape(-1)
+    out = np.empty((t.size, dim), np.float64)
+    _chk(lib().hqo_timestep_embedding(_ptr(t), t.size, dim, float(max_period), _ptr(out)), "timestep_embedding")
+    return out
+
+
+def conv2d_float(x, w, bias, stride: int, pad: int) -> np.ndarray:
+    """Floating-point convolution, x NHWC, w [Cout][R][S][C], zero padding; fp64."""
+    x, w = _c(x, np.float64), _c(w, np.float64)
+    Nb, H, W, Cc = x.shape
+    Cout, R, S, _ = w.shape
+    b = None if bias is None else _c(bias, np.float64)
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    out = np.empty((Nb, Ho, Wo, Cout), np.float64)
+    _chk(lib().hqo_conv2d_float(_ptr(x), _ptr(w), _ptr(b), Nb, H, W, Cc, Cout, R, S, stride, pad, _ptr(out)),
+         "conv2d_float")
     return out
 
 

@@ -16,8 +16,10 @@
  * Pins (tests/test_oracle_pins.py): H_raw*H_raw^T = n*I and the closed form
  * (-1)^popcount(i&j); the worked vectors of Eq. 15-16; |u - s*q| <= s/2; involution and
  * Parseval; brute-force integer products; conv == im2col GEMM; exact recovery of X*W_hat
- * when activations are not rounded.  Parity unpinned: nothing in this file (trained scales,
- * LoRA values and image-quality metrics are outside it).
+ * when activations are not rounded; the network's unquantized operations (GroupNorm, SiLU,
+ * attention core, nearest up-sampling, step embedding, float convolution) against torch's CPU
+ * routines in fp64 and closed forms (tests/test_oracle_network_pins.py).  Parity unpinned:
+ * nothing in this file (trained scales, LoRA values and image-quality metrics are outside it).
  *
  * Layout conventions: activations [rows][cols] row-major; weights [N][RS][C] (output
  * channel, filter tap, input channel), i.e. the transpose of the paper's W in R^{Ci x Co};
@@ -439,6 +441,126 @@ int hqo_groupnorm_silu(const double* x, i64 Nb, i64 H, i64 W, i64 C, int groups,
                 const i64 ch = g * cg + c, idx = (n * HW + p) * C + ch;
                 const double y = (x[idx] - mean) * rstd * gamma[ch] + beta[ch];
                 out[idx] = y / (1.0 + exp(-y));
+            }
+    }
+    return 0;
+}
+
+/* ==== The operations around the quantized layers of the noise-prediction network =================================
+ * The method replaces every linear and convolution of the network (overview figure of the framework); what sits
+ * between them is the network's own, unquantized arithmetic.  None of it is in the paper's equations: each function
+ * below is the usual definition written out in fp64, pinned against torch's CPU routines and closed forms. */
+
+/* GroupNorm as above with the activation selectable: act = 0 none (the normalisation in front of an attention
+ * block's QKV projection), act = 1 SiLU. */
+int hqo_groupnorm(const double* x, i64 Nb, i64 H, i64 W, i64 C, int groups, const double* gamma, const double* beta,
+                  double eps, int act, double* out) {
+    if (groups <= 0 || C % groups != 0 || (act != 0 && act != 1)) return -1;
+    const i64 cg = C / groups, HW = H * W;
+#pragma omp parallel for schedule(static)
+    for (i64 ng = 0; ng < Nb * groups; ++ng) {
+        const i64 n = ng / groups, g = ng % groups;
+        double sum = 0.0;
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) sum += x[(n * HW + p) * C + g * cg + c];
+        const double mean = sum / (double)(HW * cg);
+        double var = 0.0;
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) { const double d = x[(n * HW + p) * C + g * cg + c] - mean; var += d * d; }
+        var /= (double)(HW * cg);
+        const double rstd = 1.0 / sqrt(var + eps);
+        for (i64 p = 0; p < HW; ++p)
+            for (i64 c = 0; c < cg; ++c) {
+                const i64 ch = g * cg + c, idx = (n * HW + p) * C + ch;
+                const double y = (x[idx] - mean) * rstd * gamma[ch] + beta[ch];
+                out[idx] = act ? y / (1.0 + exp(-y)) : y;
+            }
+    }
+    return 0;
+}
+
+/* Multi-head self-attention core.  qkv [Nb][L][3*C]: for token t the query, key and value vectors of head h are
+ * qkv[t][h*dh .. ], qkv[t][C + h*dh ..], qkv[t][2C + h*dh ..], dh = C / heads.  Per sample and head:
+ * out[i] = sum_j softmax_j(q_i . k_j / sqrt(dh)) v_j,  written to out [Nb][L][C] at columns h*dh .. */
+int hqo_attention(const double* qkv, i64 Nb, i64 L, i64 C, int heads, double* out) {
+    if (heads <= 0 || C % heads != 0 || L <= 0) return -1;
+    const i64 dh = C / heads;
+    const double scale = 1.0 / sqrt((double)dh);
+#pragma omp parallel for schedule(static)
+    for (i64 nh = 0; nh < Nb * heads; ++nh) {
+        const i64 n = nh / heads, h = nh % heads;
+        double* s = (double*)malloc((size_t)L * sizeof(double));
+        for (i64 i = 0; i < L; ++i) {
+            const double* q = qkv + (n * L + i) * 3 * C + h * dh;
+            double mx = -INFINITY;
+            for (i64 j = 0; j < L; ++j) {
+                const double* k = qkv + (n * L + j) * 3 * C + C + h * dh;
+                double dot = 0.0;
+                for (i64 d = 0; d < dh; ++d) dot += q[d] * k[d];
+                s[j] = dot * scale;
+                if (s[j] > mx) mx = s[j];
+            }
+            double den = 0.0;
+            for (i64 j = 0; j < L; ++j) { s[j] = exp(s[j] - mx); den += s[j]; }
+            double* o = out + (n * L + i) * C + h * dh;
+            for (i64 d = 0; d < dh; ++d) {
+                double acc = 0.0;
+                for (i64 j = 0; j < L; ++j) acc += s[j] * qkv[(n * L + j) * 3 * C + 2 * C + h * dh + d];
+                o[d] = acc / den;
+            }
+        }
+        free(s);
+    }
+    return 0;
+}
+
+/* Nearest-neighbour up-sampling by two: out[n][2h+i][2w+j][c] = x[n][h][w][c], i, j in {0, 1}. */
+int hqo_upsample_nearest2x(const double* x, i64 Nb, i64 H, i64 W, i64 C, double* out) {
+    for (i64 n = 0; n < Nb; ++n)
+        for (i64 ho = 0; ho < 2 * H; ++ho)
+            for (i64 wo = 0; wo < 2 * W; ++wo)
+                for (i64 c = 0; c < C; ++c)
+                    out[((n * 2 * H + ho) * 2 * W + wo) * C + c] = x[((n * H + ho / 2) * W + wo / 2) * C + c];
+    return 0;
+}
+
+/* Sinusoidal embedding of the denoising step: for i < dim/2, f_i = exp(-ln(max_period) * i / (dim/2));
+ * out[n][i] = cos(t[n] * f_i), out[n][dim/2 + i] = sin(t[n] * f_i).  dim even. */
+int hqo_timestep_embedding(const double* t, i64 Nb, i64 dim, double max_period, double* out) {
+    if (dim <= 0 || (dim & 1)) return -1;
+    const i64 half = dim / 2;
+    for (i64 n = 0; n < Nb; ++n)
+        for (i64 i = 0; i < half; ++i) {
+            const double f = exp(-log(max_period) * (double)i / (double)half);
+            out[n * dim + i] = cos(t[n] * f);
+            out[n * dim + half + i] = sin(t[n] * f);
+        }
+    return 0;
+}
+
+/* Floating-point convolution (the network's first and last convolution, which the method leaves unquantized):
+ * x NHWC, w [Cout][R][S][C], zero padding; out[n][ho][wo][co] = bias[co] + sum x[n][ho*st+r-p][wo*st+s-p][c] w[co][r][s][c]. */
+int hqo_conv2d_float(const double* x, const double* w, const double* bias, i64 Nb, i64 H, i64 W, i64 C, i64 Cout,
+                     int R, int S, int stride, int pad, double* out) {
+    const i64 Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - S) / stride + 1;
+    if (Ho <= 0 || Wo <= 0) return -1;
+#pragma omp parallel for schedule(static)
+    for (i64 nho = 0; nho < Nb * Ho; ++nho) {
+        const i64 n = nho / Ho, ho = nho % Ho;
+        for (i64 wo = 0; wo < Wo; ++wo)
+            for (i64 co = 0; co < Cout; ++co) {
+                double t = bias ? bias[co] : 0.0;
+                for (int r = 0; r < R; ++r) {
+                    const i64 hi = ho * stride + r - pad;
+                    if (hi < 0 || hi >= H) continue;
+                    for (int s = 0; s < S; ++s) {
+                        const i64 wi = wo * stride + s - pad;
+                        if (wi < 0 || wi >= W) continue;
+                        for (i64 c = 0; c < C; ++c)
+                            t += x[((n * H + hi) * W + wi) * C + c] * w[((co * R + r) * S + s) * C + c];
+                    }
+                }
+                out[((n * Ho + ho) * Wo + wo) * Cout + co] = t;
             }
     }
     return 0;
