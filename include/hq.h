@@ -230,6 +230,60 @@ hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, i
                            int32_t* dev_status, void* stream);
 
 
+/* ---- Fused linear layer with GroupNorm (optionally + SiLU) in front, on the pixels of an NHWC tensor: the QKV
+ * projection of an attention block (no counterpart in the paper's equations; the paper quantizes the projection, the
+ * normalisation in front of it is the network's own).  Rows = Nb * rows_per_sample; statistics per (sample, group) over
+ * rows_per_sample * (C / groups) values; one activation scale per row.  Other arguments as hq_gn_silu_qconv / hq_qlinear. */
+hq_status hq_gn_qlinear(const void* x, hq_dtype xdt, int64_t Nb, int64_t rows_per_sample, int64_t C, int groups,
+                        const float* gamma, const float* beta, float eps, int silu, const hq_weight_desc* desc,
+                        const void* w_dev, const float* scale_w, const float* bias, int a_bits, void* y, hq_dtype ydt,
+                        int64_t ldy, void* workspace, size_t ws_bytes, void* scratch, size_t scratch_bytes,
+                        int32_t* dev_status, void* stream);
+
+/* ==== The unquantized operations between the quantized layers of the noise-prediction network ======================
+ * The method replaces every linear and convolution of the network (overview figure of the framework; Experiments: the
+ * first and last convolution stay in floating point); what follows is the arithmetic left between them.  None of it is
+ * one of the paper's equations.  All tensors are device bf16 unless stated, channel axis contiguous, 16-byte aligned,
+ * channel counts multiples of 8; every call is asynchronous on `stream` and returns an hq_status as above. */
+
+/* out[i] = x[i] * sigmoid(x[i]); count elements (multiple of 8).  out may alias x. */
+hq_status hq_silu(const void* x, int64_t count, void* out, void* stream);
+/* out[i] = a[i] + b[i] (residual connections); out may alias a or b. */
+hq_status hq_add(const void* a, const void* b, int64_t count, void* out, void* stream);
+/* h[n][r][c] += e[n][c] in place: h [Nb][rows_per_sample][C], e [Nb][C] (the step/class embedding added to every pixel
+ * of a sample inside a residual block). */
+hq_status hq_add_rows_bcast(void* h, const void* e, int64_t Nb, int64_t rows_per_sample, int64_t C, void* stream);
+/* emb[n][:] += table[labels[n]][:]: emb [Nb][dim], table [classes][dim], labels device int32 [Nb] (clamped to the table). */
+hq_status hq_class_embed_add(void* emb, const void* table, const int32_t* labels, int64_t Nb, int64_t dim,
+                             int64_t classes, void* stream);
+/* Sinusoidal embedding of the denoising step: t device fp32 [Nb]; out [Nb][dim], dim even;
+ * out[n][i] = cos(t[n] f_i), out[n][dim/2 + i] = sin(t[n] f_i), f_i = max_period^(-i / (dim/2)). */
+hq_status hq_timestep_embedding(const float* t, int64_t Nb, int64_t dim, float max_period, void* out, void* stream);
+/* Nearest-neighbour up-sampling by two: x NHWC [Nb][H][W][C] -> out [Nb][2H][2W][C]. */
+hq_status hq_upsample_nearest2x(const void* x, int64_t Nb, int64_t H, int64_t W, int64_t C, void* out, void* stream);
+/* Channel concatenation (skip connections): out[r] = a[r] | b[r], a [rows][Ca], b [rows][Cb], out [rows][Ca + Cb]. */
+hq_status hq_concat_channels(const void* a, int64_t Ca, const void* b, int64_t Cb, int64_t rows, void* out,
+                             void* stream);
+/* GroupNorm as a pass of its own, with SiLU when silu != 0 (the normalisation in front of the unquantized last
+ * convolution): x, out NHWC; gamma, beta device fp32 [C]; scratch as for hq_gn_silu_quant (Nb * groups * 24 bytes). */
+hq_status hq_groupnorm_act(const void* x, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups, const float* gamma,
+                           const float* beta, float eps, int silu, void* out, void* scratch, size_t scratch_bytes,
+                           void* stream);
+/* Floating-point convolution for the network's first and last layer (fp32 weights [Cout][R][R][C] and bias on the
+ * device, fp32 accumulation, zero padding, R in {1,3}, stride in {1,2}).  Two shapes are covered: few input channels
+ * (C <= 16, Cout a multiple of 8, bf16 output, fp32 or bf16 input) and few output channels (Cout <= 4, C a multiple of
+ * 8, bf16 input, fp32 output); anything else returns HQ_ERR_UNSUPPORTED. */
+hq_status hq_conv2d_direct(const void* x, hq_dtype xdt, const float* w, const float* bias, int64_t Nb, int64_t H,
+                           int64_t W, int64_t C, int64_t Cout, int R, int stride, int pad, void* y, hq_dtype ydt,
+                           void* stream);
+/* Self-attention core: qkv [Nb][L][3C] holds, per token, the queries of all heads, then the keys, then the values
+ * (head h at columns h*dh .. of each third, dh = C / heads in {32, 48, 64, 96, 128});
+ * out[n][i][h*dh ..] = sum_j softmax_j(q_i . k_j / sqrt(dh)) v_j, out [Nb][L][C].  bf16 operands on the tensor cores,
+ * fp32 accumulation and softmax; the softmax weights are rounded to bf16 before they multiply the values.
+ * dev_status as for the integer product (bounded waits). */
+hq_status hq_attention(const void* qkv, int64_t Nb, int64_t L, int64_t C, int heads, void* out, int32_t* dev_status,
+                       void* stream);
+
 /* ---- Fused linear layer that allocates nothing and takes no workspace (the paper has no counterpart: this is a
  * packaging of hq_qlinear for a particular kind of caller, not another operation). ---------------------------------
  * Who it is for: code that must not, or cannot, obtain device memory at the moment it runs a layer -- an inference

@@ -25,7 +25,9 @@ WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBL
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
-           "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv"]
+           "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv", "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast",
+           "hq_class_embed_add", "hq_timestep_embedding", "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act",
+           "hq_conv2d_direct", "hq_attention"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -78,12 +80,26 @@ def _load():
                                 p, C.c_size_t, p, p]
     L.hq_gn_silu_qconv.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, C.POINTER(WeightDesc), p, i32, i32, i32,
                                    i32, p, p, i32, i32, p, p, i32, p, C.c_size_t, p, C.c_size_t, p, p]
+    L.hq_gn_qlinear.argtypes = [p, i32, i64, i64, i64, i32, p, p, C.c_float, i32, C.POINTER(WeightDesc), p, p, p, i32, p, i32,
+                                i64, p, C.c_size_t, p, C.c_size_t, p, p]
+    L.hq_silu.argtypes = [p, i64, p, p]
+    L.hq_add.argtypes = [p, p, i64, p, p]
+    L.hq_add_rows_bcast.argtypes = [p, p, i64, i64, i64, p]
+    L.hq_class_embed_add.argtypes = [p, p, p, i64, i64, i64, p]
+    L.hq_timestep_embedding.argtypes = [p, i64, i64, C.c_float, p, p]
+    L.hq_upsample_nearest2x.argtypes = [p, i64, i64, i64, i64, p, p]
+    L.hq_concat_channels.argtypes = [p, i64, p, i64, i64, p, p]
+    L.hq_groupnorm_act.argtypes = [p, i64, i64, i64, i64, i32, p, p, C.c_float, i32, p, p, C.c_size_t, p]
+    L.hq_conv2d_direct.argtypes = [p, i32, p, p, i64, i64, i64, i64, i64, i32, i32, i32, p, i32, p]
+    L.hq_attention.argtypes = [p, i64, i64, i64, i32, p, p, p]
     L.hq_alpha_for.restype = C.c_float
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
                  "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
-                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv"):
+                 "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv",
+                 "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast", "hq_class_embed_add", "hq_timestep_embedding",
+                 "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act", "hq_conv2d_direct", "hq_attention"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -301,3 +317,70 @@ def hq_qconv_width(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int,
 
 def hq_mma_i8_probe(ctas: int, iters: int, dev_status=None, stream=None) -> None:
     _check(lib.hq_mma_i8_probe(ctas, iters, _dptr(dev_status), _stream(stream)), "hq_mma_i8_probe")
+
+
+def hq_gn_qlinear(x, Nb: int, groups: int, gamma, beta, eps: float, silu: bool, pw: PreparedWeight, bias, a_bits: int, y,
+                  workspace, scratch, dev_status=None, stream=None) -> None:
+    """The fused linear layer on the pixels of x [Nb * rows_per_sample, C] with GroupNorm (+ SiLU) in front."""
+    M, Cin = x.shape
+    _check(lib.hq_gn_qlinear(_dptr(x), _dtype_code(x), Nb, M // Nb, Cin, groups, _dptr(gamma), _dptr(beta), eps, int(silu),
+                             C.byref(pw.desc), _dptr(pw.blob_dev), _dptr(pw.s_w_dev), _dptr(bias), a_bits, _dptr(y),
+                             _dtype_code(y), y.stride(0), _dptr(workspace), workspace.numel() * workspace.element_size(),
+                             _dptr(scratch), scratch.numel() * scratch.element_size(), _dptr(dev_status), _stream(stream)),
+           "hq_gn_qlinear")
+
+
+def hq_silu(x, out, stream=None) -> None:
+    _check(lib.hq_silu(_dptr(x), x.numel(), _dptr(out), _stream(stream)), "hq_silu")
+
+
+def hq_add(a, b, out, stream=None) -> None:
+    _check(lib.hq_add(_dptr(a), _dptr(b), a.numel(), _dptr(out), _stream(stream)), "hq_add")
+
+
+def hq_add_rows_bcast(h, e, stream=None) -> None:
+    """h [Nb, ..., C] += e [Nb, C] in place."""
+    Nb, Cc = e.shape
+    _check(lib.hq_add_rows_bcast(_dptr(h), _dptr(e), Nb, h.numel() // (Nb * Cc), Cc, _stream(stream)), "hq_add_rows_bcast")
+
+
+def hq_class_embed_add(emb, table, labels, stream=None) -> None:
+    Nb, dim = emb.shape
+    _check(lib.hq_class_embed_add(_dptr(emb), _dptr(table), _dptr(labels), Nb, dim, table.shape[0], _stream(stream)),
+           "hq_class_embed_add")
+
+
+def hq_timestep_embedding(t, out, max_period: float = 10000.0, stream=None) -> None:
+    Nb, dim = out.shape
+    _check(lib.hq_timestep_embedding(_dptr(t), Nb, dim, max_period, _dptr(out), _stream(stream)), "hq_timestep_embedding")
+
+
+def hq_upsample_nearest2x(x, out, stream=None) -> None:
+    Nb, H, W, Cc = x.shape
+    _check(lib.hq_upsample_nearest2x(_dptr(x), Nb, H, W, Cc, _dptr(out), _stream(stream)), "hq_upsample_nearest2x")
+
+
+def hq_concat_channels(a, b, out, stream=None) -> None:
+    Ca, Cb = a.shape[-1], b.shape[-1]
+    _check(lib.hq_concat_channels(_dptr(a), Ca, _dptr(b), Cb, a.numel() // Ca, _dptr(out), _stream(stream)),
+           "hq_concat_channels")
+
+
+def hq_groupnorm_act(x, groups: int, gamma, beta, eps: float, silu: bool, out, scratch, stream=None) -> None:
+    Nb, H, W, Cc = x.shape
+    _check(lib.hq_groupnorm_act(_dptr(x), Nb, H, W, Cc, groups, _dptr(gamma), _dptr(beta), eps, int(silu), _dptr(out),
+                                _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)), "hq_groupnorm_act")
+
+
+def hq_conv2d_direct(x, w, bias, R: int, stride: int, pad: int, y, stream=None) -> None:
+    """Floating-point convolution: x NHWC, w device fp32 [Cout, R, R, C], y NHWC."""
+    Nb, H, W, Cc = x.shape
+    _check(lib.hq_conv2d_direct(_dptr(x), _dtype_code(x), _dptr(w), _dptr(bias), Nb, H, W, Cc, w.shape[0], R, stride, pad,
+                                _dptr(y), _dtype_code(y), _stream(stream)), "hq_conv2d_direct")
+
+
+def hq_attention(qkv, Nb: int, heads: int, out, dev_status=None, stream=None) -> None:
+    """qkv [Nb * L, 3C] -> out [Nb * L, C]."""
+    M, C3 = qkv.shape
+    _check(lib.hq_attention(_dptr(qkv), Nb, M // Nb, C3 // 3, heads, _dptr(out), _dptr(dev_status), _stream(stream)),
+           "hq_attention")

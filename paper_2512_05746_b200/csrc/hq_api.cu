@@ -25,7 +25,8 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
 hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
                                const float* gamma, const float* beta, float eps, int had_block, int bits,
                                hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
-                               int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st);
+                               int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                               int silu);
 hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
                           const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
                           hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
@@ -144,10 +145,38 @@ extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, i
     unsigned char* codes = static_cast<unsigned char*>(workspace);
     float* scales = reinterpret_cast<float*>(codes + scales_offset(rows, C, cont));
     s = launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, desc->had_block, a_bits, mode, static_scale, codes,
-                             cont, ldc, scales, scratch, scratch_bytes, st);
+                             cont, ldc, scales, scratch, scratch_bytes, st, 1);
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st, true);
+}
+
+// The fused linear layer on the pixels of an NHWC tensor with GroupNorm (optionally + SiLU) in front: the QKV
+// projection of an attention block, whose input is the normalised feature map.  Rows = Nb * rows_per_sample pixels.
+extern "C" hq_status hq_gn_qlinear(const void* x, hq_dtype xdt, int64_t Nb, int64_t rows_per_sample, int64_t C, int groups,
+                                   const float* gamma, const float* beta, float eps, int silu, const hq_weight_desc* desc,
+                                   const void* w_dev, const float* scale_w, const float* bias, int a_bits, void* y,
+                                   hq_dtype ydt, int64_t ldy, void* workspace, size_t ws_bytes, void* scratch,
+                                   size_t scratch_bytes, int32_t* dev_status, void* stream) {
+    using namespace hq;
+    if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+    if (Nb <= 0 || rows_per_sample <= 0) return HQ_ERR_SHAPE;
+    const hq_container cont = hq_container(desc->container);
+    const int64_t M = Nb * rows_per_sample;
+    size_t need = 0;
+    hq_status s = hq_workspace_size(M, C, cont, &need);
+    if (s != HQ_OK) return s;
+    if (ws_bytes < need) return HQ_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* codes = static_cast<unsigned char*>(workspace);
+    float* scales = reinterpret_cast<float*>(codes + scales_offset(M, C, cont));
+    const int64_t ldc = code_pitch(C, cont);
+    s = launch_gn_silu_quant(x, xdt, Nb, rows_per_sample, 1, C, groups, gamma, beta, eps, desc->had_block, a_bits,
+                             HQ_SCALE_PER_ROW, nullptr, codes, cont, ldc, scales, scratch, scratch_bytes, st, silu != 0);
+    if (s != HQ_OK) return s;
+    return launch_qgemm(codes, cont, a_bits, M, C, ldc, desc, w_dev, scales, 0, scale_w, bias, hq_alpha_for(desc), nullptr,
+                        y, ydt, ldy, dev_status, st, true);
 }
 
 extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,

@@ -1,0 +1,392 @@
+// The unquantized operations that sit between the quantized layers of the noise-prediction network (the method replaces
+// every linear and convolution; this is what is left): SiLU, residual and broadcast additions, the sinusoidal step
+// embedding with the class-embedding lookup, nearest-neighbour up-sampling, channel concatenation, GroupNorm with an
+// optional SiLU as a stand-alone pass, and the network's first and last convolution, which stay in floating point.
+// All activations are bf16, row-major with the channel axis contiguous (NHWC); arithmetic is fp32.
+// Every kernel is HBM-bound element-wise work: 16-byte loads and stores, one element group per thread.
+#include "hq_common.cuh"
+
+namespace hq {
+
+// GroupNorm statistics of an NHWC tensor into `scratch` (defined in hq_quant.cu): [samples][groups][2] fp64 sums,
+// followed by [samples][groups][2] floats (mean, 1/sqrt(var + eps)).
+hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
+                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st);
+
+namespace {
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float silu_f(float y) { return y / (1.0f + __expf(-y)); }
+
+struct F8 { float v[8]; };
+__device__ __forceinline__ F8 unpack8(const uint4 w) {
+    F8 r;
+    r.v[0] = bf16_lo(w.x); r.v[1] = bf16_hi(w.x); r.v[2] = bf16_lo(w.y); r.v[3] = bf16_hi(w.y);
+    r.v[4] = bf16_lo(w.z); r.v[5] = bf16_hi(w.z); r.v[6] = bf16_lo(w.w); r.v[7] = bf16_hi(w.w);
+    return r;
+}
+__device__ __forceinline__ uint4 pack8(const F8& f) {
+    return make_uint4(pack2(f.v[0], f.v[1]), pack2(f.v[2], f.v[3]), pack2(f.v[4], f.v[5]), pack2(f.v[6], f.v[7]));
+}
+
+// out = silu(x), n8 groups of 8 values
+__global__ void __launch_bounds__(256) silu_kernel(const uint4* x, uint4* out, int64_t n8) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    F8 f = unpack8(__ldg(x + i));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) f.v[e] = silu_f(f.v[e]);
+    out[i] = pack8(f);
+}
+
+// out = a + b
+__global__ void __launch_bounds__(256) add_kernel(const uint4* a, const uint4* b, uint4* out, int64_t n8) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    F8 fa = unpack8(__ldcs(a + i));
+    const F8 fb = unpack8(__ldcs(b + i));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) fa.v[e] += fb.v[e];
+    out[i] = pack8(fa);
+}
+
+// h[n][r][c] += e[n][c]   (c8 = C / 8 vectors per row)
+__global__ void __launch_bounds__(256) add_rows_bcast_kernel(uint4* h, const uint4* e, int64_t n8, int c8,
+                                                             int64_t vec_per_sample) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const int64_t n = i / vec_per_sample;
+    const int c = int(i % c8);
+    F8 fh = unpack8(h[i]);
+    const F8 fe = unpack8(__ldg(e + n * c8 + c));
+#pragma unroll
+    for (int k = 0; k < 8; ++k) fh.v[k] += fe.v[k];
+    h[i] = pack8(fh);
+}
+
+// emb[n][:] += table[labels[n]][:]
+__global__ void __launch_bounds__(256) class_embed_add_kernel(__nv_bfloat16* emb, const __nv_bfloat16* table,
+                                                              const int32_t* labels, int Nb, int dim, int classes) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Nb * dim) return;
+    const int n = i / dim, d = i - n * dim;
+    int lab = labels[n];
+    lab = lab < 0 ? 0 : (lab >= classes ? classes - 1 : lab);
+    emb[i] = __float2bfloat16_rn(__bfloat162float(emb[i]) + __bfloat162float(table[int64_t(lab) * dim + d]));
+}
+
+// out[n][i] = cos(t[n] f_i), out[n][half + i] = sin(t[n] f_i), f_i = exp(-ln(max_period) i / half)
+__global__ void __launch_bounds__(256) timestep_embedding_kernel(const float* t, int Nb, int dim, float max_period,
+                                                                 __nv_bfloat16* out) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const int half = dim / 2;
+    if (idx >= Nb * half) return;
+    const int n = idx / half, i = idx - n * half;
+    const float f = expf(-logf(max_period) * float(i) / float(half));
+    const float a = t[n] * f;
+    out[int64_t(n) * dim + i] = __float2bfloat16_rn(cosf(a));
+    out[int64_t(n) * dim + half + i] = __float2bfloat16_rn(sinf(a));
+}
+
+// out[n][2h+i][2w+j][:] = x[n][h][w][:]; one thread per input vector, four stores
+__global__ void __launch_bounds__(256) upsample2x_kernel(const uint4* x, uint4* out, int64_t n8, int c8, int W, int H) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const int c = int(i % c8);
+    const int64_t pix = i / c8;
+    const int w = int(pix % W);
+    const int64_t nh = pix / W;                       // n * H + h
+    const uint4 v = __ldcs(x + i);
+    const int64_t o = ((2 * nh) * (2 * int64_t(W)) + 2 * w) * c8 + c;     // (n, 2h, 2w)
+    out[o] = v;
+    out[o + c8] = v;
+    out[o + 2 * int64_t(W) * c8] = v;
+    out[o + 2 * int64_t(W) * c8 + c8] = v;
+}
+
+// out[r][0..Ca) = a[r][:], out[r][Ca..Ca+Cb) = b[r][:]
+__global__ void __launch_bounds__(256) concat_kernel(const uint4* a, int ca8, const uint4* b, int cb8, uint4* out,
+                                                     int64_t n8) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const int c8 = ca8 + cb8;
+    const int64_t r = i / c8;
+    const int c = int(i - r * c8);
+    out[i] = c < ca8 ? __ldcs(a + r * ca8 + c) : __ldcs(b + r * cb8 + (c - ca8));
+}
+
+// y = act((x - mean) rstd gamma + beta) with the statistics of the element's (sample, group)
+__global__ void __launch_bounds__(256) gn_apply_kernel(const uint4* x, uint4* out, int64_t n8, int c8,
+                                                       int64_t vec_per_sample, const float* stats, const float* gamma,
+                                                       const float* beta, int groups, int cg, int act) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const int64_t n = i / vec_per_sample;
+    const int c0 = int(i % c8) * 8;
+    F8 f = unpack8(__ldcs(x + i));
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const int c = c0 + e;
+        const float2 st = *reinterpret_cast<const float2*>(stats + (n * groups + c / cg) * 2);
+        const float a = st.y * __ldg(gamma + c);
+        const float y = fmaf(f.v[e], a, fmaf(-st.x, a, __ldg(beta + c)));
+        f.v[e] = act ? silu_f(y) : y;
+    }
+    out[i] = pack8(f);
+}
+
+// Convolution with few input channels (the network's first convolution): a warp takes one output pixel, each lane
+// eight consecutive output channels per round; the weights sit in shared memory as [tap * C + c][Cout].
+template <typename InT>
+__global__ void __launch_bounds__(256) conv_small_cin_kernel(const InT* x, const float* w, const float* bias,
+                                                             __nv_bfloat16* out, int Nb, int H, int W, int C, int Cout,
+                                                             int R, int stride, int pad, int Ho, int Wo) {
+    extern __shared__ float sw[];                      // [R*R*C][Cout]
+    const int taps = R * R * C;
+    for (int i = threadIdx.x; i < taps * Cout; i += blockDim.x) {
+        const int co = i / taps, k = i - co * taps;   // global layout [Cout][R][R][C]
+        sw[k * Cout + co] = w[i];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t pixels = int64_t(Nb) * Ho * Wo;
+    for (int64_t p = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); p < pixels;
+         p += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo = int(p % Wo);
+        const int ho = int((p / Wo) % Ho);
+        const int n = int(p / (int64_t(Wo) * Ho));
+        for (int co0 = lane * 8; co0 < Cout; co0 += 256) {
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = bias != nullptr ? __ldg(bias + co0 + e) : 0.f;
+            for (int r = 0; r < R; ++r) {
+                const int hi = ho * stride + r - pad;
+                if (hi < 0 || hi >= H) continue;
+                for (int s = 0; s < R; ++s) {
+                    const int wi = wo * stride + s - pad;
+                    if (wi < 0 || wi >= W) continue;
+                    const InT* px = x + ((int64_t(n) * H + hi) * W + wi) * C;
+                    for (int c = 0; c < C; ++c) {
+                        float xv;
+                        if (sizeof(InT) == 4) xv = __ldg(reinterpret_cast<const float*>(px) + c);
+                        else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(px)[c]);
+                        const float4* wr = reinterpret_cast<const float4*>(sw + ((r * R + s) * C + c) * Cout + co0);
+                        const float4 w0 = wr[0], w1 = wr[1];
+                        acc[0] = fmaf(xv, w0.x, acc[0]); acc[1] = fmaf(xv, w0.y, acc[1]);
+                        acc[2] = fmaf(xv, w0.z, acc[2]); acc[3] = fmaf(xv, w0.w, acc[3]);
+                        acc[4] = fmaf(xv, w1.x, acc[4]); acc[5] = fmaf(xv, w1.y, acc[5]);
+                        acc[6] = fmaf(xv, w1.z, acc[6]); acc[7] = fmaf(xv, w1.w, acc[7]);
+                    }
+                }
+            }
+            F8 f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f.v[e] = acc[e];
+            *reinterpret_cast<uint4*>(out + p * Cout + co0) = pack8(f);
+        }
+    }
+}
+
+// Convolution with few output channels (the network's last convolution): a warp takes one output pixel, each lane eight
+// input channels per round of 256 for every filter tap (coalesced 512-byte reads), the weights [Cout][R][R][C] sit in
+// shared memory as they are, and the partial sums of the warp are added up by shuffles.  Output fp32.
+template <int COUT>
+__global__ void __launch_bounds__(256) conv_small_cout_kernel(const __nv_bfloat16* x, const float* w, const float* bias,
+                                                              float* out, int Nb, int H, int W, int C, int R, int stride,
+                                                              int pad, int Ho, int Wo) {
+    extern __shared__ float sw[];                      // [COUT][R*R][C]
+    const int wsize = COUT * R * R * C;
+    for (int i = threadIdx.x; i < wsize; i += blockDim.x) sw[i] = w[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t pixels = int64_t(Nb) * Ho * Wo;
+    for (int64_t p = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); p < pixels;
+         p += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo = int(p % Wo);
+        const int ho = int((p / Wo) % Ho);
+        const int n = int(p / (int64_t(Wo) * Ho));
+        float acc[COUT];
+#pragma unroll
+        for (int o = 0; o < COUT; ++o) acc[o] = 0.f;
+        for (int r = 0; r < R; ++r) {
+            const int hi = ho * stride + r - pad;
+            if (hi < 0 || hi >= H) continue;
+            for (int s = 0; s < R; ++s) {
+                const int wi = wo * stride + s - pad;
+                if (wi < 0 || wi >= W) continue;
+                const __nv_bfloat16* px = x + ((int64_t(n) * H + hi) * W + wi) * C;
+                for (int c0 = lane * 8; c0 < C; c0 += 256) {
+                    const F8 f = unpack8(__ldg(reinterpret_cast<const uint4*>(px + c0)));
+#pragma unroll
+                    for (int o = 0; o < COUT; ++o) {
+                        const float4* wr = reinterpret_cast<const float4*>(sw + (o * R * R + r * R + s) * C + c0);
+                        const float4 w0 = wr[0], w1 = wr[1];
+                        acc[o] = fmaf(f.v[0], w0.x, fmaf(f.v[1], w0.y, fmaf(f.v[2], w0.z, fmaf(f.v[3], w0.w, acc[o]))));
+                        acc[o] = fmaf(f.v[4], w1.x, fmaf(f.v[5], w1.y, fmaf(f.v[6], w1.z, fmaf(f.v[7], w1.w, acc[o]))));
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 0; o < COUT; ++o) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc[o] += __shfl_xor_sync(0xffffffffu, acc[o], off);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int o = 0; o < COUT; ++o) out[p * COUT + o] = acc[o] + (bias != nullptr ? __ldg(bias + o) : 0.f);
+        }
+    }
+}
+
+inline int blocks_for(int64_t n, int threads) { return int((n + threads - 1) / threads); }
+
+}  // namespace
+}  // namespace hq
+
+using namespace hq;
+
+extern "C" hq_status hq_silu(const void* x, int64_t count, void* out, void* stream) {
+    if (count < 0) return HQ_ERR_SHAPE;
+    if (count == 0) return HQ_OK;
+    if (x == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(out) || count % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const int64_t n8 = count / 8;
+    silu_kernel<<<blocks_for(n8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(x), static_cast<uint4*>(out), n8);
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_add(const void* a, const void* b, int64_t count, void* out, void* stream) {
+    if (count < 0) return HQ_ERR_SHAPE;
+    if (count == 0) return HQ_OK;
+    if (a == nullptr || b == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out) || count % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const int64_t n8 = count / 8;
+    add_kernel<<<blocks_for(n8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(a), static_cast<const uint4*>(b), static_cast<uint4*>(out), n8);
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_add_rows_bcast(void* h, const void* e, int64_t Nb, int64_t rows_per_sample, int64_t C,
+                                       void* stream) {
+    if (Nb < 0 || rows_per_sample < 0 || C <= 0) return HQ_ERR_SHAPE;
+    if (Nb == 0 || rows_per_sample == 0) return HQ_OK;
+    if (h == nullptr || e == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(h) || !aligned16(e) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const int64_t n8 = Nb * rows_per_sample * (C / 8);
+    add_rows_bcast_kernel<<<blocks_for(n8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<uint4*>(h), static_cast<const uint4*>(e), n8, int(C / 8), rows_per_sample * (C / 8));
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_class_embed_add(void* emb, const void* table, const int32_t* labels, int64_t Nb, int64_t dim,
+                                        int64_t classes, void* stream) {
+    if (Nb < 0 || dim <= 0 || classes <= 0 || Nb * dim > 0x7FFFFFFF) return HQ_ERR_SHAPE;
+    if (Nb == 0) return HQ_OK;
+    if (emb == nullptr || table == nullptr || labels == nullptr) return HQ_ERR_INVALID_ARG;
+    class_embed_add_kernel<<<blocks_for(Nb * dim, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<__nv_bfloat16*>(emb), static_cast<const __nv_bfloat16*>(table), labels, int(Nb), int(dim), int(classes));
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_timestep_embedding(const float* t, int64_t Nb, int64_t dim, float max_period, void* out,
+                                           void* stream) {
+    if (Nb < 0 || dim <= 0 || (dim & 1) || !(max_period > 1.0f) || Nb * dim > 0x7FFFFFFF) return HQ_ERR_SHAPE;
+    if (Nb == 0) return HQ_OK;
+    if (t == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
+    timestep_embedding_kernel<<<blocks_for(Nb * (dim / 2), 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        t, int(Nb), int(dim), max_period, static_cast<__nv_bfloat16*>(out));
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_upsample_nearest2x(const void* x, int64_t Nb, int64_t H, int64_t W, int64_t C, void* out,
+                                           void* stream) {
+    if (Nb < 0 || H <= 0 || W <= 0 || C <= 0 || H > 0x3FFFFFFF || W > 0x3FFFFFFF) return HQ_ERR_SHAPE;
+    if (Nb == 0) return HQ_OK;
+    if (x == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(out) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const int64_t n8 = Nb * H * W * (C / 8);
+    upsample2x_kernel<<<blocks_for(n8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(x), static_cast<uint4*>(out), n8, int(C / 8), int(W), int(H));
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_concat_channels(const void* a, int64_t Ca, const void* b, int64_t Cb, int64_t rows, void* out,
+                                        void* stream) {
+    if (rows < 0 || Ca <= 0 || Cb <= 0) return HQ_ERR_SHAPE;
+    if (rows == 0) return HQ_OK;
+    if (a == nullptr || b == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out) || Ca % 8 != 0 || Cb % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const int64_t n8 = rows * ((Ca + Cb) / 8);
+    concat_kernel<<<blocks_for(n8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(a), int(Ca / 8), static_cast<const uint4*>(b), int(Cb / 8), static_cast<uint4*>(out), n8);
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_groupnorm_act(const void* x, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                                      const float* gamma, const float* beta, float eps, int silu, void* out,
+                                      void* scratch, size_t scratch_bytes, void* stream) {
+    if (x == nullptr || out == nullptr || gamma == nullptr || beta == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
+    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0 || groups <= 0 || C % groups != 0) return HQ_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(out) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float* stats = nullptr;
+    hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st);
+    if (s != HQ_OK) return s;
+    const int64_t n8 = Nb * H * W * (C / 8);
+    gn_apply_kernel<<<blocks_for(n8, 256), 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(out), n8,
+                                                         int(C / 8), H * W * (C / 8), stats, gamma, beta, groups,
+                                                         int(C / groups), silu != 0);
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+extern "C" hq_status hq_conv2d_direct(const void* x, hq_dtype xdt, const float* w, const float* bias, int64_t Nb,
+                                      int64_t H, int64_t W, int64_t C, int64_t Cout, int R, int stride, int pad, void* y,
+                                      hq_dtype ydt, void* stream) {
+    if (x == nullptr || w == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if ((xdt != HQ_F32 && xdt != HQ_BF16) || (ydt != HQ_F32 && ydt != HQ_BF16)) return HQ_ERR_INVALID_ARG;
+    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0) return HQ_ERR_SHAPE;
+    if ((R != 1 && R != 3) || (stride != 1 && stride != 2) || pad < 0 || pad > 1) return HQ_ERR_UNSUPPORTED;
+    const int64_t Ho = (H + 2 * pad - R) / stride + 1, Wo = (W + 2 * pad - R) / stride + 1;
+    if (Ho <= 0 || Wo <= 0) return HQ_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem = size_t(R) * R * C * Cout * sizeof(float);
+    if (smem > 160 * 1024) return HQ_ERR_UNSUPPORTED;
+    const int64_t pixels = Nb * Ho * Wo;
+    const int grid = int(pixels / 8 < 148 * 16 ? (pixels + 7) / 8 : 148 * 16);
+    if (ydt == HQ_BF16 && C <= 16 && Cout % 8 == 0) {                          // few input channels
+        if (!aligned16(y)) return HQ_ERR_ALIGNMENT;
+        if (xdt == HQ_F32) {
+            HQ_CUDA_OK(cudaFuncSetAttribute(conv_small_cin_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+            conv_small_cin_kernel<float><<<grid, 256, smem, st>>>(static_cast<const float*>(x), w, bias,
+                static_cast<__nv_bfloat16*>(y), int(Nb), int(H), int(W), int(C), int(Cout), R, stride, pad, int(Ho), int(Wo));
+        } else {
+            HQ_CUDA_OK(cudaFuncSetAttribute(conv_small_cin_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+            conv_small_cin_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(x), w, bias,
+                static_cast<__nv_bfloat16*>(y), int(Nb), int(H), int(W), int(C), int(Cout), R, stride, pad, int(Ho), int(Wo));
+        }
+        return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+    }
+    if (ydt == HQ_F32 && xdt == HQ_BF16 && Cout <= 4 && C % 8 == 0) {          // few output channels
+        if (!aligned16(x)) return HQ_ERR_ALIGNMENT;
+#define HQ_COUT_CASE(N)                                                                                             \
+        case N:                                                                                                     \
+            HQ_CUDA_OK(cudaFuncSetAttribute(conv_small_cout_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
+            conv_small_cout_kernel<N><<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(x), w, bias,       \
+                static_cast<float*>(y), int(Nb), int(H), int(W), int(C), R, stride, pad, int(Ho), int(Wo));         \
+            break;
+        switch (int(Cout)) {
+            HQ_COUT_CASE(1) HQ_COUT_CASE(2) HQ_COUT_CASE(3) HQ_COUT_CASE(4)
+            default: return HQ_ERR_UNSUPPORTED;
+        }
+#undef HQ_COUT_CASE
+        return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+    }
+    return HQ_ERR_UNSUPPORTED;
+}

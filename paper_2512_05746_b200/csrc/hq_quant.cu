@@ -38,6 +38,7 @@ struct QuantParams {
     const float* gn_gamma;   // [cols]
     const float* gn_beta;    // [cols]
     int gn_groups;
+    int gn_silu;             // 1: SiLU after the normalisation, 0: none
     int64_t gn_rows_per_sample;
     // optional LayerNorm over each row with a per-sample affine, applied before the transform (ln_on != 0)
     int ln_on;
@@ -146,10 +147,12 @@ __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, i
 //            KLOG = 12 needs one more stage than fits and takes it with a lane exchange.
 // Dynamic scales never need the clamp (|t| * qmax / max|t| rounds to at most qmax); static scales do.
 // PRO: prologue applied to the values before the transform: 0 none, 1 GroupNorm + SiLU (statistics given), 2 LayerNorm
-// over the row (statistics taken here: the row is in the registers of its threads) with a per-sample affine.
+// over the row (statistics taken here: the row is in the registers of its threads) with a per-sample affine, 3 GroupNorm
+// alone (the normalisation in front of an attention block's QKV projection).
 template <int KLOG, int E, typename InT, bool INT8_OUT, bool STATIC, int PRO>
 __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
-    constexpr bool GN = PRO == 1;
+    constexpr bool GN = PRO == 1 || PRO == 3;          // 3: GroupNorm without the SiLU
+    constexpr bool GN_SILU = PRO == 1;
     constexpr bool LN = PRO == 2;
     griddep_launch();      // a GEMM launched as a programmatic dependent may start its prologue as this grid drains
     constexpr int N = 1 << KLOG;
@@ -212,8 +215,9 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
                 const int ch = blk * N + 4 * (tb + TB * i);
                 const float4 a4 = *reinterpret_cast<const float4*>(gn_a + ch);
                 const float4 b4 = *reinterpret_cast<const float4*>(gn_b + ch);
-                f.x = silu(fmaf(f.x, a4.x, b4.x)); f.y = silu(fmaf(f.y, a4.y, b4.y));
-                f.z = silu(fmaf(f.z, a4.z, b4.z)); f.w = silu(fmaf(f.w, a4.w, b4.w));
+                f.x = fmaf(f.x, a4.x, b4.x); f.y = fmaf(f.y, a4.y, b4.y);
+                f.z = fmaf(f.z, a4.z, b4.z); f.w = fmaf(f.w, a4.w, b4.w);
+                if (GN_SILU) { f.x = silu(f.x); f.y = silu(f.y); f.z = silu(f.z); f.w = silu(f.w); }
             }
             if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
             v[2 * i] = pk2(f.x, f.y);
@@ -599,9 +603,13 @@ cudaError_t launch_fast(const QuantParams& p, bool int8_out, int grid, int threa
         kern<<<grid, threads, smem, st>>>(p);
         return cudaGetLastError();
     };
-    if (p.gn_stats != nullptr) {
+    if (p.gn_stats != nullptr && p.gn_silu) {
         if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 1>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 1>);
         return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, 1>) : go(fwht_quant_fast<KLOG, E, InT, false, false, 1>);
+    }
+    if (p.gn_stats != nullptr) {
+        if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 3>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 3>);
+        return stat ? go(fwht_quant_fast<KLOG, E, InT, false, true, 3>) : go(fwht_quant_fast<KLOG, E, InT, false, false, 3>);
     }
     if (p.ln_on) {
         if (int8_out) return stat ? go(fwht_quant_fast<KLOG, E, InT, true, true, 2>) : go(fwht_quant_fast<KLOG, E, InT, true, false, 2>);
@@ -633,7 +641,7 @@ cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int gri
 }  // namespace
 
 // Launches the transform+quantize kernel; shared by the public entry point and the fused layer calls.
-struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; };
+struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; int silu; };
 struct LnArgs { const float* w; const float* b; int64_t rows_per_group; float eps; };
 
 static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
@@ -667,7 +675,7 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
     p.scales = scales;
     if (gn != nullptr) {
         p.gn_stats = gn->stats; p.gn_gamma = gn->gamma; p.gn_beta = gn->beta; p.gn_groups = gn->groups;
-        p.gn_rows_per_sample = gn->rows_per_sample;
+        p.gn_rows_per_sample = gn->rows_per_sample; p.gn_silu = gn->silu;
     }
     if (ln != nullptr) {
         p.ln_on = 1; p.ln_w = ln->w; p.ln_b = ln->b; p.ln_rows_per_group = ln->rows_per_group; p.ln_eps = ln->eps;
@@ -730,16 +738,13 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
                              nullptr, st);
 }
 
-// GroupNorm + SiLU of an NHWC tensor fused into the transform+quantize kernel: statistics per (sample, group) first
-// (fp64 sums in `scratch`, which is cleared here), then the quantize kernel applies x * a[c] + b[c] and SiLU as it
-// loads.  scratch: Nb * groups * (2 doubles + 2 floats).
-hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
-                               const float* gamma, const float* beta, float eps, int had_block, int bits,
-                               hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
-                               int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st) {
-    if (x == nullptr || gamma == nullptr || beta == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
+// GroupNorm statistics of an NHWC tensor (hw pixels per sample): fp64 sums per (sample, group) in `scratch` (cleared
+// here), then mean and 1/sqrt(var + eps) as floats behind them.  scratch: Nb * groups * (2 doubles + 2 floats).
+hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
+                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st) {
+    if (x == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
-    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0 || groups <= 0) return HQ_ERR_SHAPE;
+    if (Nb <= 0 || hw <= 0 || C <= 0 || groups <= 0) return HQ_ERR_SHAPE;
     if (C % groups != 0 || (C / groups) % 4 != 0) return HQ_ERR_SHAPE;      // whole channel quads per group
     if (groups > 1024) return HQ_ERR_UNSUPPORTED;
     const size_t need = size_t(Nb) * groups * (2 * sizeof(double) + 2 * sizeof(float));
@@ -749,7 +754,6 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
     if (reinterpret_cast<uintptr_t>(x) % (4 * elt) != 0) return HQ_ERR_ALIGNMENT;
     double* sums = static_cast<double*>(scratch);
     float* stats = reinterpret_cast<float*>(sums + size_t(Nb) * groups * 2);
-    const int64_t hw = H * W;
     HQ_CUDA_OK(cudaMemsetAsync(sums, 0, size_t(Nb) * groups * 2 * sizeof(double), st));
     // enough CTAs that a thread walks about 16 pixels per channel quad (short dependent chains, many loads in flight)
     const int64_t ppl = C / 4 < 256 ? 256 / (C / 4) : 1;
@@ -768,7 +772,24 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
     const int total = int(Nb * groups);
     gn_finalize_kernel<<<(total + 127) / 128, 128, 0, st>>>(sums, hw * (C / groups), double(eps), total, stats);
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
-    const GnArgs gn{stats, gamma, beta, groups, hw};
+    *stats_out = stats;
+    return HQ_OK;
+}
+
+// GroupNorm (+ SiLU when `silu`) of an NHWC tensor fused into the transform+quantize kernel: statistics per (sample,
+// group) first, then the quantize kernel applies x * a[c] + b[c] and the activation as it loads.
+hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                               const float* gamma, const float* beta, float eps, int had_block, int bits,
+                               hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                               int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
+                               int silu) {
+    if (gamma == nullptr || beta == nullptr) return HQ_ERR_INVALID_ARG;
+    if (H <= 0 || W <= 0) return HQ_ERR_SHAPE;
+    const int64_t hw = H * W;
+    const float* stats = nullptr;
+    hq_status s = launch_gn_stats(x, xdt, Nb, hw, C, groups, eps, scratch, scratch_bytes, &stats, st);
+    if (s != HQ_OK) return s;
+    const GnArgs gn{stats, gamma, beta, groups, hw, silu};
     return launch_quant_impl(x, xdt, Nb * hw, C, C, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales, &gn,
                              st);
 }
@@ -840,7 +861,7 @@ extern "C" hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, i
                                       hq_container cont, int64_t ld_codes, float* scales, void* scratch,
                                       size_t scratch_bytes, void* stream) {
     return hq::launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, had_block, bits, mode, static_scale, codes,
-                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream));
+                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream), 1);
 }
 
 extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,

@@ -114,3 +114,101 @@ def config_sweep_point(M: int, K: int, N: int, seed: int = 0) -> dict:
                 x=activations((M, K), outlier_count=max(1, round(0.01 * K)), outlier_scale=20.0,
                               seed=seed, stream=50),
                 w=weights((N, K), seed=seed, stream=51), bias=bias(N, seed=seed, stream=52))
+
+
+# ---------------------------------------------------------------------------------------------
+# A latent-diffusion UNet: configuration and seeded random parameters (names and shapes only).
+# ---------------------------------------------------------------------------------------------
+
+def unet_config(batch: int = 64, latent: int = 64, in_ch: int = 3, base: int = 256, mults=(1, 2, 3, 4),
+                res_blocks: int = 2, attn_resolutions=(32, 16, 8), heads: int = 8, groups: int = 32,
+                classes: int = 1000, had_block: int = 256) -> dict:
+    """The noise-prediction network the workload names: residual blocks of GroupNorm + SiLU + 3x3 convolution, a step
+    + class embedding fed into every residual block, self-attention at the listed resolutions, stride-2 convolutions
+    down, nearest up-sampling + convolution up, skip connections by channel concatenation."""
+    return dict(batch=batch, latent=latent, in_ch=in_ch, base=base, mults=tuple(mults), res_blocks=res_blocks,
+                attn_resolutions=tuple(attn_resolutions), heads=heads, groups=groups, classes=classes, had_block=had_block)
+
+
+def unet_params(cfg: dict, seed: int = 0) -> dict:
+    """name -> fp32 array for every parameter of the network, drawn from the seeded stream in a fixed order.
+    Convolution weights are [Cout, R, R, Cin], linear weights [N, K], both ~N(0, 1/fan_in) so that activations keep
+    their scale through the network; biases ~N(0, 0.01); norm gains 1 + 0.1 N(0,1), offsets 0.1 N(0,1); the class
+    table ~N(0, 0.3)."""
+    P = {}
+    counter = [0]
+
+    def draw(shape, std):
+        counter[0] += 1
+        return np.ascontiguousarray(_rng(seed, 2000 + counter[0]).standard_normal(size=shape, dtype=np.float32) * np.float32(std))
+
+    def conv(name, cin, cout, R):
+        P[name + ".w"] = draw((cout, R, R, cin), 1.0 / np.sqrt(R * R * cin))
+        P[name + ".b"] = draw((cout,), 0.01)
+
+    def linear(name, K, N):
+        P[name + ".w"] = draw((N, K), 1.0 / np.sqrt(K))
+        P[name + ".b"] = draw((N,), 0.01)
+
+    def norm(name, ch):
+        P[name + ".gamma"] = np.ascontiguousarray(1.0 + draw((ch,), 0.1), dtype=np.float32)
+        P[name + ".beta"] = draw((ch,), 0.1)
+
+    def resblock(name, cin, cout):
+        norm(name + ".norm1", cin)
+        conv(name + ".conv1", cin, cout, 3)
+        linear(name + ".emb", temb, cout)
+        norm(name + ".norm2", cout)
+        conv(name + ".conv2", cout, cout, 3)
+        if cin != cout:
+            conv(name + ".skip", cin, cout, 1)
+
+    def attention(name, ch):
+        norm(name + ".norm", ch)
+        linear(name + ".qkv", ch, 3 * ch)
+        linear(name + ".proj", ch, ch)
+
+    base, mults, nres = cfg["base"], cfg["mults"], cfg["res_blocks"]
+    temb = 4 * base
+    linear("time_embed.0", base, temb)
+    linear("time_embed.2", temb, temb)
+    P["label_emb"] = draw((cfg["classes"], temb), 0.3)
+    conv("in_conv", cfg["in_ch"], base, 3)
+    ch, res = base, cfg["latent"]
+    skips = [ch]
+    for lvl, m in enumerate(mults):
+        for b in range(nres):
+            resblock(f"down{lvl}.res{b}", ch, m * base)
+            ch = m * base
+            if res in cfg["attn_resolutions"]:
+                attention(f"down{lvl}.attn{b}", ch)
+            skips.append(ch)
+        if lvl + 1 < len(mults):
+            conv(f"down{lvl}.downsample", ch, ch, 3)
+            res //= 2
+            skips.append(ch)
+    resblock("mid.res0", ch, ch)
+    attention("mid.attn", ch)
+    resblock("mid.res1", ch, ch)
+    for lvl in reversed(range(len(mults))):
+        m = mults[lvl]
+        for b in range(nres + 1):
+            resblock(f"up{lvl}.res{b}", ch + skips.pop(), m * base)
+            ch = m * base
+            if res in cfg["attn_resolutions"]:
+                attention(f"up{lvl}.attn{b}", ch)
+        if lvl > 0:
+            res *= 2
+            conv(f"up{lvl}.upsample", ch, ch, 3)
+    norm("out_norm", ch)
+    conv("out_conv", ch, cfg["in_ch"], 3)
+    return P
+
+
+def unet_inputs(cfg: dict, seed: int = 0) -> dict:
+    """Latent x NHWC ~N(0,1), denoising steps t in [0, 1000), class labels."""
+    r = _rng(seed, 1999)
+    Nb, S = cfg["batch"], cfg["latent"]
+    return dict(x=np.ascontiguousarray(r.standard_normal(size=(Nb, S, S, cfg["in_ch"]), dtype=np.float32)),
+                t=r.integers(0, 1000, size=(Nb,)).astype(np.float32),
+                y=r.integers(0, cfg["classes"], size=(Nb,)).astype(np.int32))
