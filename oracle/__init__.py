@@ -292,6 +292,16 @@ def silu(x) -> np.ndarray:
     return x / (1.0 + np.exp(-x))
 
 
+def round_bf16(x) -> np.ndarray:
+    """The value a bf16 store keeps: fp64 -> fp32 -> the nearest number with 8 significant bits (ties to even), back
+    as fp64.  Used where a tensor is defined to be held in bf16 between two layers."""
+    f = np.ascontiguousarray(np.asarray(x, np.float64).astype(np.float32))
+    u = f.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    out = r.astype(np.uint32).view(np.float32).astype(np.float64)
+    return np.where(np.isfinite(f), out, f.astype(np.float64))
+
+
 def attention(qkv, heads: int) -> np.ndarray:
     """Self-attention core on qkv [Nb, L, 3C] (query | key | value column thirds, heads contiguous inside each):
     softmax(q k^T / sqrt(dh)) v per sample and head -> [Nb, L, C]; fp64."""

@@ -276,7 +276,8 @@ class UNet:
 
         h = self._new((Nb, S, S, base))
         w_in, b_in = self.f32["in_conv.w"], self.f32["in_conv.b"]
-        self._glue("in_conv", "conv_float", lambda: hq.hq_conv2d_direct(self.x_in, w_in, b_in, 3, 1, 1, h), x=self.x_in, out=h)
+        self._glue("in_conv", "conv_float", (lambda o=h: hq.hq_conv2d_direct(self.x_in, w_in, b_in, 3, 1, 1, o)), x=self.x_in,
+                   out=h)
         ch, res = base, S
         skips = [h]
         for lvl, m in enumerate(mults):

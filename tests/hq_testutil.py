@@ -113,3 +113,15 @@ def weight_integers(oracle, pw, w, w_bits: int, had_block: int, mode: str) -> np
     diff = B_blob != B_orc
     assert diff.mean() <= 1e-4 and (not diff.any() or np.abs(B_blob - B_orc)[diff].max() == 1)
     return B_blob
+
+
+def attention_bound(oracle, qr, Nb, L, C, heads, want):
+    """Element-wise error bound of the attention core from its arithmetic.  A bf16 rounding moves a value by at most
+    2^-8 of itself (8 significant bits).  The softmax weights p_j are rounded to bf16 before they multiply the values,
+    so an output sum_j p_j v_j / sum_j p_j may move by up to 2^-8 * sum_j p_j |v_j| through the numerator and by 2^-8 of
+    itself through the denominator; the result is rounded to bf16 once more (2^-8 of itself); the fp32 accumulation
+    and the approximate exp2 are far below that.  sum_j p_j |v_j| is the oracle's own attention applied to |v|."""
+    qa = qr.reshape(Nb, L, 3 * C).copy()
+    qa[:, :, 2 * C:] = np.abs(qa[:, :, 2 * C:])
+    A = oracle.attention(qa, heads).reshape(Nb * L, C)
+    return 2.0 ** -8 * A + 2.0 ** -7 * np.abs(want) + 1e-6 * A

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 from paper_2512_05746_b200 import inputs
-from hq_testutil import PARITY_STATS, Y_BF16_RTOL, Y_F32_RTOL, rel_err
+from hq_testutil import PARITY_STATS, Y_BF16_RTOL, Y_F32_RTOL, attention_bound, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -128,18 +128,6 @@ ATTN_CASES = [
     (1, 200, 128, 2),       # ragged: 200 = 128 + 72 queries and keys
     (1, 16, 64, 2),         # a 4x4 map
 ]
-
-
-def attention_bound(oracle, qr, Nb, L, C, heads, want):
-    """Element-wise error bound of the attention core from its arithmetic.  A bf16 rounding moves a value by at most
-    2^-8 of itself (8 significant bits).  The softmax weights p_j are rounded to bf16 before they multiply the values,
-    so an output sum_j p_j v_j / sum_j p_j may move by up to 2^-8 * sum_j p_j |v_j| through the numerator and by 2^-8 of
-    itself through the denominator; the result is rounded to bf16 once more (2^-8 of itself); the fp32 accumulation
-    and the approximate exp2 are far below that.  sum_j p_j |v_j| is the oracle's own attention applied to |v|."""
-    qa = qr.reshape(Nb, L, 3 * C).copy()
-    qa[:, :, 2 * C:] = np.abs(qa[:, :, 2 * C:])
-    A = oracle.attention(qa, heads).reshape(Nb * L, C)
-    return 2.0 ** -8 * A + 2.0 ** -7 * np.abs(want) + 1e-6 * A
 
 
 @pytest.mark.parametrize("Nb,L,C,heads", ATTN_CASES)

@@ -102,3 +102,13 @@ def test_conv2d_float_equals_torch(oracle, R, stride, pad, C, Cout):
     xi = np.random.default_rng(1).integers(-8, 8, size=(1, 5, 5, C)).astype(np.int8)
     wi = np.random.default_rng(2).integers(-8, 8, size=(Cout, R, R, C)).astype(np.int32)
     assert np.array_equal(oracle.conv2d_float(xi, wi, None, stride, pad), oracle.conv2d_int(xi, wi, stride, pad))
+
+
+def test_round_bf16_equals_torch_conversion(oracle):
+    """Ties go to even, the sign is kept, values already representable come back unchanged."""
+    x = np.concatenate([rnd((4000,), 5) * 10.0 ** rnd((4000,), 6), [0.0, -0.0, 1.0, 1.00390625, 1.01171875, -3.0e38, 1e-40]])
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
+    got = oracle.round_bf16(x)
+    assert np.array_equal(got, want)
+    assert oracle.round_bf16(1.00390625) == 1.0 and oracle.round_bf16(1.01171875) == 1.015625      # ties: to even
+    assert np.array_equal(oracle.round_bf16(got), got)
