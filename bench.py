@@ -400,24 +400,17 @@ def main_reference(args):
 
 
 def main_layer_list(args, which):
-    """All quantized layers of a network-shaped workload, one after the other on one stream, bf16 activations,
-    W4A4 with folded two-limb weights.  3x3 convolutions use one static activation scale, 1x1 convolutions and linears
-    per-row scales.  The bf16 glue between the layers is not part of this path.
-    unet: 121 layers of the UNet-shaped workload (batch 64, 64x64 latent); dit: 143 linears of a width-1152,
-    depth-28 diffusion transformer (batch 32, 256 tokens)."""
+    """The quantized linears of the DiT-shaped workload, one after the other on one stream, bf16 activations, W4A4 with
+    folded two-limb weights, per-row scales: 143 linears of a width-1152, depth-28 diffusion transformer (batch 32,
+    256 tokens).  The attention core and the other glue between them are not part of this workload."""
     import torch
     from paper_2512_05746_b200 import binding as hq
-    from paper_2512_05746_b200 import dit, unet
+    from paper_2512_05746_b200 import dit
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    if which == "unet":
-        layers = unet.quantized_layers()
-        label = "the 121 quantized layers of the UNet-shaped workload (batch 64, 64x64 latent)"
-        wl = "configs[3] quantized layers only: 121 layers, 47 distinct shapes"
-    else:
-        layers = dit.quantized_layers()
-        label = "the 143 quantized linears of the DiT-XL/2-shaped workload (batch 32, 256 tokens, width 1152 = 9 x 128)"
-        wl = "DiT-XL/2-shaped quantized linears: 28 blocks x (adaLN, QKV, proj, FC1, FC2) + embedding MLP"
+    layers = dit.quantized_layers()
+    label = "the 143 quantized linears of the DiT-XL/2-shaped workload (batch 32, 256 tokens, width 1152 = 9 x 128)"
+    wl = "DiT-XL/2-shaped quantized linears: 28 blocks x (adaLN, QKV, proj, FC1, FC2) + embedding MLP"
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
     cache = {}
@@ -502,54 +495,6 @@ def main_layer_list(args, which):
     for d in per_shape.values():
         d["ms_each"] = d["ms"] / d["count"]
         d["tops"] = 2.0 * d["macs"] * d["limbs"] / (d["ms_each"] * 1e-3) / 1e12
-    # The UNet's residual-block convolutions take SiLU(GroupNorm32(h)) as input: the same forward with that prologue
-    # fused into the transform kernel of those layers (statistics pass + normalise-on-load), reported beside the main figure.
-    gn_extra = None
-    if which == "unet":
-        gn_layers = [L for L in layers if L["kind"] == "conv" and L["R"] == 3 and L["stride"] == 1 and
-                     (".conv1" in L["name"] or ".conv2" in L["name"])]
-        for L in gn_layers:
-            r = L["res"]
-            if "gn" in r:
-                continue
-            cin, rows = L["C"], L["Nb"] * L["H"] * L["W"]
-            g = dict(gamma=torch.ones((cin,), device=dev), beta=torch.zeros((cin,), device=dev),
-                     scratch=torch.empty((L["Nb"] * 32 * 24,), dtype=torch.uint8, device=dev))
-            codes, sc = ws_views(torch, r["ws"], rows, cin)
-            hq.hq_gn_silu_quant(r["x"], 32, g["gamma"], g["beta"], 1e-5, L["had_block"], A_BITS, codes, CODES[0], g["scratch"],
-                                scales=sc)
-            g["static"] = sc.max().reshape(1).contiguous()          # one static scale, calibrated on the normalised input
-            r["gn"] = g
-        torch.cuda.synchronize()
-        gn_names = {L["name"] for L in gn_layers}
-
-        def forward_gn():
-            for L in layers:
-                r = L["res"]
-                if L["name"] in gn_names:
-                    g = r["gn"]
-                    hq.hq_gn_silu_qconv(r["x"], 32, g["gamma"], g["beta"], 1e-5, r["pw"], L["R"], L["R"], L["stride"], L["pad"],
-                                        r["bias"], A_BITS, r["y"], r["ws"], g["scratch"], static_scale=g["static"],
-                                        dev_status=status)
-                elif L["kind"] == "conv":
-                    hq.hq_qconv(r["x"], r["pw"], L["R"], L["R"], L["stride"], L["pad"], r["bias"], A_BITS, r["y"], r["ws"],
-                                static_scale=r["static"], dev_status=status)
-                else:
-                    hq.hq_qlinear(r["x"], r["pw"], r["bias"], A_BITS, r["y"], r["ws"], dev_status=status)
-
-        for _ in range(3):
-            forward_gn()
-        torch.cuda.synchronize()
-        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g0.record()
-        for _ in range(steps):
-            forward_gn()
-        g1.record()
-        torch.cuda.synchronize()
-        hq.hq_check_status(status)
-        gn_extra = dict(ms_per_step=g0.elapsed_time(g1) / steps, layers_with_prologue=len(gn_layers),
-                        note="GroupNorm(32) + SiLU fused in front of the residual-block 3x3 convolutions "
-                             "(hq_gn_silu_qconv)")
     # The transformer's QKV and FC1 linears take modulate(LayerNorm(x), shift, scale) as input: the same forward with that
     # prologue fused into the transform kernel of those layers (row statistics from the registers that hold the row).
     ln_extra = None
@@ -616,11 +561,82 @@ def main_layer_list(args, which):
                                       tops_1limb_equiv=2.0 * macs / ms / 1e9,
                                       l2="activations of the large layers exceed L2"),
                           clocks=clocks, gpu_launches=2 * len(layers) * steps, per_shape=per_shape,
-                          with_groupnorm_prologue=gn_extra, with_layernorm_prologue=ln_extra)))
+                          with_layernorm_prologue=ln_extra)))
 
 
 def main_unet(args):
-    return main_layer_list(args, "unet")
+    """One denoising step of the UNet-shaped network (batch 64, 64x64x3 latent, base 256, multipliers (1,2,3,4), two
+    residual blocks per level, 8-head self-attention at 32/16/8, step + class embedding): every convolution but the first
+    and last and every linear is a Hadamard-quantized W4A4 layer (3x3 convolutions with a calibrated static scale and
+    GroupNorm + SiLU fused into their transform kernel), data flows from layer to layer, and the bf16 operations between
+    them (attention core, additions, concatenation, up-sampling, embeddings, first / last convolution) run in the
+    library's own kernels.  Reports the full forward, and the quantized layers and the glue timed on their own over the
+    buffers of a complete forward."""
+    import torch
+    from paper_2512_05746_b200 import binding as hq
+    from paper_2512_05746_b200.unet import UNet, quantized_layers
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    batch = 64 if args.rows == 32768 else max(1, int(args.rows))          # --rows N: a reduced batch for profiler captures
+    cfg = inputs.unet_config(batch=batch)
+    t_setup = time.time()
+    P = inputs.unet_params(cfg, seed=0)
+    I = inputs.unet_inputs(cfg, seed=0)
+    net = UNet(cfg, P, hq, dev, container=CODES[0], a_bits=A_BITS).build(batch)
+    del P
+    x, t, y = torch.from_numpy(I["x"]), torch.from_numpy(I["t"]), torch.from_numpy(I["y"])
+    net.calibrate(x, t, y)
+    t_setup = time.time() - t_setup
+    stream = torch.cuda.current_stream()
+    for _ in range(max(3, min(args.warmup, 5))):
+        net.run()
+    t_one = timed_region(torch, net.run, 2, stream) / 2
+    steps = max(args.steps, int(600.0 / max(t_one, 1e-3)) + 1)          # at least 0.6 s in the timed region
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms_full = timed_region(torch, net.run, steps, stream) / steps
+    clocks = sampler.stop()
+    clocks["window"] = "the timed region (full forwards)"
+    reps = max(5, steps // 3)
+    ms_q = timed_region(torch, lambda: net.run(tags=("q",)), reps, stream) / reps
+    ms_g = timed_region(torch, lambda: net.run(tags=("g",)), reps, stream) / reps
+    hq.hq_check_status(net.status)
+    # one forward with an event after every call: time per kind of operation
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(net.tape) + 1)]
+    evs[0].record(stream)
+    for i, (_, _, call) in enumerate(net.tape):
+        call()
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    by_kind = {}
+    for i, (tag, name, _) in enumerate(net.tape):
+        if tag == "q":
+            kind = "quantized " + ("conv3x3" if (".conv" in name or "sample" in name) else "conv1x1" if name.endswith(".skip") else "linear")
+        else:
+            kind = ("attention core" if name.endswith(".core") else "residual / embedding add" if ("residual" in name or "emb_add" in name)
+                    else "concat" if name.endswith(".concat") else "upsample" if name.endswith(".nearest")
+                    else "first / last conv" if name in ("in_conv", "out_conv") else "final groupnorm" if name == "out_norm"
+                    else "embedding path")
+        d = by_kind.setdefault(kind, dict(calls=0, ms=0.0))
+        d["calls"] += 1
+        d["ms"] += evs[i].elapsed_time(evs[i + 1])
+    layers = quantized_layers(batch=batch)
+    macs = sum(L["macs"] for L in layers)
+    nq = sum(1 for tag, _, _ in net.tape if tag == "q")
+    attn_flops = net.attn_flops
+    print(json.dumps(dict(metric="UNet forwards/s: one denoising step of the UNet-shaped network, batch 64 per forward",
+                          value=1e3 / ms_full, unit="forwards/s", n_gpus=1, steps=steps, warmup=max(3, min(args.warmup, 5)),
+                          ms_per_step=ms_full, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="int8",
+                          data="synthetic",
+                          config=dict(workload=f"configs[3] UNet forward: batch {batch}, 64x64x3 latent, base 256, mult (1,2,3,4), attention at "
+                                               f"32/16/8 with 8 heads, 1000 classes; W4A{A_BITS}, folded weights, {codes_name()} codes, bf16 activations",
+                                      quantized_layers=nq, library_calls=len(net.tape), samples_per_s=batch * 1e3 / ms_full,
+                                      l2="activations of the large layers exceed L2", setup_s=t_setup),
+                          full_forward_ms=ms_full, quantized_only_ms=ms_q, glue_ms=ms_g,
+                          quantized_tops=2.0 * macs / (ms_q * 1e-3) / 1e12,
+                          attention_tflops=attn_flops / (by_kind.get("attention core", dict(ms=1e30))["ms"] * 1e-3) / 1e12,
+                          by_kind={k: dict(calls=v["calls"], ms=round(v["ms"], 4)) for k, v in sorted(by_kind.items())},
+                          clocks=clocks, gpu_launches=len(net.tape) * steps)))
 
 
 def main_sweep(args):

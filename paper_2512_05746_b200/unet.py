@@ -241,6 +241,7 @@ class UNet:
         qkv = self._linear(name + ".qkv", x2, norm=name + ".norm", Nb=Nb)
         a = self._new((Nb * H * W, ch))
         heads = self.cfg["heads"]
+        self.attn_flops += 4.0 * Nb * float(H * W) ** 2 * ch
         self._glue(name + ".core", "attention", lambda: hq.hq_attention(qkv, Nb, heads, a, dev_status=self.status),
                    qkv=qkv, out=a, Nb=Nb, heads=heads)
         pr = self._linear(name + ".proj", a)
@@ -256,6 +257,7 @@ class UNet:
         temb = 4 * base
         self.tape = []
         self.Nb = Nb
+        self.attn_flops = 0.0          # 4 L^2 C per sample and attention block (QK^T and PV)
         self._ws_need = 256
         self.scratch = t.empty((Nb * cfg["groups"] * 24,), dtype=t.uint8, device=self.dev)
         self.x_in = t.empty((Nb, S, S, cfg["in_ch"]), dtype=t.bfloat16, device=self.dev)
