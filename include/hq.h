@@ -64,8 +64,13 @@ typedef enum { HQ_SCALE_PER_ROW = 0, HQ_SCALE_STATIC = 1 } hq_scale_mode;
  *  PLAIN : B = Q(W)                       (Eq. 3 per output channel)
  *  FOLDED: B = H_raw * Q(W)               (the inner product of Eq. 12 / Eq. 14, exact integers; the
  *                                          paper's Single-Hadamard semantics; needs w_bits + log2(had_block) bits)
- *  DOUBLE: B = Q(H^T W), H orthonormal    (the Double-Hadamard scheme the paper compares against) */
-typedef enum { HQ_W_PLAIN = 0, HQ_W_FOLDED = 1, HQ_W_DOUBLE = 2 } hq_weight_mode;
+ *  DOUBLE: B = Q(H^T W), H orthonormal    (the Double-Hadamard scheme the paper compares against)
+ *  PLAIN_A2: B = Q(W) laid out for activations that arrive as TWO int8 limbs per channel, [hi(C) | lo(C)] per pixel
+ *            (the width-axis convolution with blocks wider than 16 positions, whose integer activations q * H_raw need
+ *            more than 8 bits): the blob describes 2C input channels per tap and two weight limbs, "hi" rows
+ *            [Q(W) | 0] and "lo" rows [0 | Q(W)], so that the two-limb product 256 * acc_hi + acc_lo of the kernel is
+ *            sum (256 * a_hi + a_lo) * Q(W). */
+typedef enum { HQ_W_PLAIN = 0, HQ_W_FOLDED = 1, HQ_W_DOUBLE = 2, HQ_W_PLAIN_A2 = 3 } hq_weight_mode;
 
 /* Host-side description of a prepared weight blob (filled by hq_weight_prepare). */
 typedef struct {
@@ -170,12 +175,19 @@ hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W
  *   had_block_w = 2^k divides W (0/1: no transform); static_scale = S (device, 1 float); bits in {3,4,8}.
  *   The integer factor must fit a signed byte: had_block_w * 2^(bits-1) <= 128 (16 positions at 4 bits, 32 at 3 bits),
  *   otherwise HQ_ERR_OVERFLOW_RISK.
+ * hq_hadamard_quant_width2: the same for wider blocks (up to 64 positions, so the full width of a 32- or 64-wide feature
+ *   map is one block as in Eq. 13): z is written as two int8 limbs per channel, z = 256 * hi + lo with lo in [-128, 127],
+ *   z_limbs device NHWC [Nb][H][W][2C] = [hi(C) | lo(C)] per pixel.  C % 2 == 0.
  * hq_qconv_width: the whole layer.  desc / w_dev: PLAIN one-limb weights prepared for the INT8 container
  *   (had_block of the descriptor is ignored); workspace as for hq_qconv with the INT8 container;
- *   y = 2^(-k/2) * S * S_w[o] * Conv(z, W_int) + bias[o]. */
+ *   y = 2^(-k/2) * S * S_w[o] * Conv(z, W_int) + bias[o].  With a PLAIN_A2 descriptor (desc->C == 2 C) the layer runs
+ *   through hq_hadamard_quant_width2 and the two-limb product; workspace hq_workspace_size(Nb*H*W, 2C, INT8). */
 hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                   int had_block_w, int bits, const float* static_scale, void* z_codes,
                                   float* scale_out, void* stream);
+hq_status hq_hadamard_quant_width2(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                   int had_block_w, int bits, const float* static_scale, void* z_limbs,
+                                   float* scale_out, void* stream);
 hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                          const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
                          const float* scale_w, const float* bias, int a_bits, int had_block_w,

@@ -19,15 +19,15 @@ HQ_OK = 0
 HQ_F32, HQ_BF16 = 0, 1
 HQ_CODES_NIBBLE, HQ_CODES_INT8 = 0, 1
 HQ_SCALE_PER_ROW, HQ_SCALE_STATIC = 0, 1
-HQ_W_PLAIN, HQ_W_FOLDED, HQ_W_DOUBLE = 0, 1, 2
-WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBLE}
+HQ_W_PLAIN, HQ_W_FOLDED, HQ_W_DOUBLE, HQ_W_PLAIN_A2 = 0, 1, 2, 3
+WEIGHT_MODES = {"plain": HQ_W_PLAIN, "folded": HQ_W_FOLDED, "double": HQ_W_DOUBLE, "plain_a2": HQ_W_PLAIN_A2}
 
 EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_quant", "hq_weight_blob_bytes",
            "hq_weight_prepare", "hq_qgemm", "hq_qconv2d", "hq_workspace_size", "hq_qlinear", "hq_qconv",
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
            "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv", "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast",
            "hq_class_embed_add", "hq_timestep_embedding", "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act",
-           "hq_conv2d_direct", "hq_attention"]
+           "hq_conv2d_direct", "hq_attention", "hq_hadamard_quant_width2"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -71,6 +71,8 @@ def _load():
     L.hq_qlinear_noalloc.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i32, i64,
                                      p, p]
     L.hq_hadamard_quant_width.argtypes = [p, i32, i64, i64, i64, i64, i32, i32, p, p, p, p]
+    L.hq_hadamard_quant_width2.argtypes = [p, i32, i64, i64, i64, i64, i32, i32, p, p, p, p]
+    L.hq_hadamard_quant_width2.restype = C.c_int
     L.hq_qconv_width.argtypes = [p, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32, i32,
                                  p, p, i32, p, C.c_size_t, p, p]
     L.hq_gn_silu_quant.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, i32, i32, i32, p, p, i32, i64, p, p,
@@ -303,6 +305,13 @@ def hq_hadamard_quant_width(x, had_block_w: int, bits: int, static_scale, z, sca
     Nb, H, W, Cin = x.shape
     _check(lib.hq_hadamard_quant_width(_dptr(x), _dtype_code(x), Nb, H, W, Cin, had_block_w, bits, _dptr(static_scale),
                                        _dptr(z), _dptr(scale_out), _stream(stream)), "hq_hadamard_quant_width")
+
+
+def hq_hadamard_quant_width2(x, had_block_w: int, bits: int, static_scale, z_limbs, scale_out=None, stream=None) -> None:
+    """As hq_hadamard_quant_width for blocks of up to 64 positions: z_limbs int8 NHWC [Nb, H, W, 2C] = [hi | lo]."""
+    Nb, H, W, Cin = x.shape
+    _check(lib.hq_hadamard_quant_width2(_dptr(x), _dtype_code(x), Nb, H, W, Cin, had_block_w, bits, _dptr(static_scale),
+                                        _dptr(z_limbs), _dptr(scale_out), _stream(stream)), "hq_hadamard_quant_width2")
 
 
 def hq_qconv_width(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias, a_bits: int, had_block_w: int,

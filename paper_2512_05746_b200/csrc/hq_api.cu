@@ -34,6 +34,9 @@ hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t col
 hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
                                       int had_block_w, int bits, const float* static_scale, void* z, float* scale_out,
                                       cudaStream_t st);
+hq_status launch_hadamard_quant_width2(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                       int had_block_w, int bits, const float* static_scale, void* z_limbs,
+                                       float* scale_out, cudaStream_t st);
 
 namespace {
 int64_t code_pitch(int64_t cols, hq_container cont) {
@@ -214,6 +217,25 @@ extern "C" hq_status hq_qconv_width(const void* x, hq_dtype xdt, int64_t Nb, int
                                     int32_t* dev_status, void* stream) {
     using namespace hq;
     if (desc == nullptr || workspace == nullptr || y == nullptr) return HQ_ERR_INVALID_ARG;
+    if (desc->mode == HQ_W_PLAIN_A2) {
+        // blocks wider than a signed byte allows: z travels as two int8 limbs per channel, [hi(C) | lo(C)] per pixel,
+        // and meets weights whose "hi" rows are [Q(W) | 0] and "lo" rows [0 | Q(W)] in the two-limb product
+        if (desc->limbs != 2 || desc->container != HQ_CODES_INT8 || desc->C != 2 * C) return HQ_ERR_SHAPE;
+        if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
+        const int64_t rows2 = Nb * H * W;
+        size_t need2 = 0;
+        hq_status s2 = hq_workspace_size(rows2, 2 * C, HQ_CODES_INT8, &need2);
+        if (s2 != HQ_OK) return s2;
+        if (ws_bytes < need2) return HQ_ERR_WORKSPACE;
+        if ((2 * C) % 16 != 0) return HQ_ERR_ALIGNMENT;
+        cudaStream_t st2 = static_cast<cudaStream_t>(stream);
+        unsigned char* z2 = static_cast<unsigned char*>(workspace);
+        float* scale2 = reinterpret_cast<float*>(z2 + scales_offset(rows2, 2 * C, HQ_CODES_INT8));
+        s2 = launch_hadamard_quant_width2(x, xdt, Nb, H, W, C, had_block_w, a_bits, static_scale, z2, scale2, st2);
+        if (s2 != HQ_OK) return s2;
+        return launch_qconv2d(z2, HQ_CODES_INT8, 8, Nb, H, W, 2 * C, desc, w_dev, R, S, stride, pad, scale2, 1, scale_w, bias,
+                              1.0f, nullptr, y, ydt, dev_status, st2, true);
+    }
     if (desc->mode != HQ_W_PLAIN || desc->limbs != 1 || desc->container != HQ_CODES_INT8) return HQ_ERR_SHAPE;
     if (!aligned16(workspace)) return HQ_ERR_ALIGNMENT;
     const int64_t rows = Nb * H * W;

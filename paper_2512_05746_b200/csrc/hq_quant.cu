@@ -532,6 +532,72 @@ __global__ void __launch_bounds__(256) width_quant_kernel(const WidthParams p) {
     }
 }
 
+// The same for blocks of 32 or 64 positions, where z = q * H_raw needs more than a signed byte: a thread owns 2 consecutive
+// channels of one block of NB positions, and z leaves as two int8 limbs, z = 256 * hi + lo with lo in [-128, 127], laid
+// out per pixel as [hi(C) | lo(C)] (the operand of a convolution whose weights were prepared for two activation limbs).
+struct Width2Params {
+    const void* x;
+    int64_t items;        // Nb * H * (W / NB) * (C / 2)
+    int64_t C;
+    int c2;               // C / 2
+    int wblocks;          // W / NB
+    int bits;
+    float norm;           // 2^(-k/2)
+    const float* static_scale;
+    int8_t* z;            // [pixels][2 C]
+    float* scale_out;
+};
+
+template <int NB, typename InT>
+__global__ void __launch_bounds__(128) width_quant2_kernel(const Width2Params p) {
+    griddep_launch();
+    const int64_t item = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const float S = __ldg(p.static_scale);
+    if (item == 0 && p.scale_out != nullptr) p.scale_out[0] = S * p.norm;
+    if (item >= p.items) return;
+    const int c2 = int(item % p.c2);
+    const int64_t rest = item / p.c2;
+    const int b = int(rest % p.wblocks);
+    const int64_t nh = rest / p.wblocks;
+    const int64_t pix0 = (nh * p.wblocks + b) * NB;                 // first pixel of the block
+    const InT* src = reinterpret_cast<const InT*>(p.x) + pix0 * p.C + 2 * c2;
+
+    f32x2 v[NB];                                                    // [position along w], one channel pair
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        if (sizeof(InT) == 4) {
+            const float2 f = __ldcs(reinterpret_cast<const float2*>(src + int64_t(i) * p.C));
+            v[i] = pk2(f.x, f.y);
+        } else {
+            const uint32_t raw = __ldcs(reinterpret_cast<const uint32_t*>(src + int64_t(i) * p.C));
+            v[i] = pk2(__uint_as_float(raw << 16), __uint_as_float(raw & 0xFFFF0000u));
+        }
+    }
+    butterflies_pairs<NB, 1, NB / 2>(v);
+    const float inv = p.norm / S;
+    const float lo = kMagic + float(-(1 << (p.bits - 1))), hi = kMagic + float((1 << (p.bits - 1)) - 1);
+    const f32x2 inv2 = pk2(inv, inv), mg2 = pk2(kMagic, kMagic);
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        float a, bb;
+        upk2(fma2(v[i], inv2, mg2), a, bb);
+        v[i] = pk2(fminf(fmaxf(a, lo), hi) - kMagic, fminf(fmaxf(bb, lo), hi) - kMagic);
+    }
+    butterflies_pairs<NB, 1, NB / 2>(v);                            // z = q * H_raw: small integers, exact in fp32
+    int8_t* dst = p.z + pix0 * 2 * p.C + 2 * c2;
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        float a, bb;
+        upk2(v[i], a, bb);
+        const int z0 = __float2int_rn(a), z1 = __float2int_rn(bb);
+        const int l0 = ((z0 + 128) & 255) - 128, l1 = ((z1 + 128) & 255) - 128;
+        const int h0 = (z0 - l0) >> 8, h1 = (z1 - l1) >> 8;
+        int8_t* px = dst + int64_t(i) * 2 * p.C;
+        *reinterpret_cast<uint16_t*>(px) = uint16_t((h0 & 255) | ((h1 & 255) << 8));
+        *reinterpret_cast<uint16_t*>(px + p.C) = uint16_t((l0 & 255) | ((l1 & 255) << 8));
+    }
+}
+
 // ---- GroupNorm statistics: sums and sums of squares per (sample, group), then mean and 1/sqrt(var + eps) --------
 // x NHWC; grid (chunks, samples); a thread owns channel quads (coalesced over channels) and walks the pixels of its
 // chunk, accumulating in fp64; per-CTA shared-memory reduction per group, one fp64 atomic pair per group and CTA.
@@ -845,6 +911,44 @@ hq_status launch_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, i
     return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
+// Width-axis transform + quantization + integer factor for blocks of up to 64 positions: z as two int8 limbs per channel.
+hq_status launch_hadamard_quant_width2(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                       int had_block_w, int bits, const float* static_scale, void* z_limbs,
+                                       float* scale_out, cudaStream_t st) {
+    if (x == nullptr || z_limbs == nullptr || static_scale == nullptr) return HQ_ERR_INVALID_ARG;
+    if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4 && bits != 8) return HQ_ERR_INVALID_ARG;
+    if (Nb <= 0 || H <= 0 || W <= 0 || C <= 0) return HQ_ERR_SHAPE;
+    const int nb = had_block_w > 1 ? had_block_w : 1;
+    if (!is_pow2(nb) || W % nb != 0) return HQ_ERR_SHAPE;
+    if (nb > 64) return HQ_ERR_UNSUPPORTED;                       // 64 two-wide registers per thread is the limit here
+    if ((int64_t(nb) << (bits - 1)) > 32768) return HQ_ERR_OVERFLOW_RISK;     // z must fit two limbs
+    if (C % 2 != 0) return HQ_ERR_UNSUPPORTED;
+    const int elt = xdt == HQ_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(x) % (2 * elt) != 0 || reinterpret_cast<uintptr_t>(z_limbs) % 2 != 0) return HQ_ERR_ALIGNMENT;
+
+    Width2Params p{};
+    p.x = x; p.C = C; p.c2 = int(C / 2); p.wblocks = int(W / nb); p.bits = bits;
+    p.items = Nb * H * (W / nb) * (C / 2);
+    p.norm = float(exp2(-0.5 * double(ilog2(nb))));
+    p.static_scale = static_scale; p.z = static_cast<int8_t*>(z_limbs); p.scale_out = scale_out;
+    const int threads = 128;
+    const int64_t grid64 = (p.items + threads - 1) / threads;
+    if (grid64 > 0x7FFFFFFF) return HQ_ERR_UNSUPPORTED;
+    const int grid = int(grid64);
+#define HQ_WIDTH2_CASE(NBV)                                                                             \
+    case NBV:                                                                                           \
+        if (xdt == HQ_F32) width_quant2_kernel<NBV, float><<<grid, threads, 0, st>>>(p);                \
+        else width_quant2_kernel<NBV, __nv_bfloat16><<<grid, threads, 0, st>>>(p);                      \
+        break;
+    switch (nb) {
+        HQ_WIDTH2_CASE(2) HQ_WIDTH2_CASE(4) HQ_WIDTH2_CASE(8) HQ_WIDTH2_CASE(16) HQ_WIDTH2_CASE(32) HQ_WIDTH2_CASE(64)
+        default: return HQ_ERR_UNSUPPORTED;
+    }
+#undef HQ_WIDTH2_CASE
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
 }  // namespace hq
 
 extern "C" hq_status hq_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
@@ -869,6 +973,13 @@ extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_
                                              float* scale_out, void* stream) {
     return hq::launch_hadamard_quant_width(x, xdt, Nb, H, W, C, had_block_w, bits, static_scale, z_codes, scale_out,
                                            static_cast<cudaStream_t>(stream));
+}
+
+extern "C" hq_status hq_hadamard_quant_width2(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                                              int had_block_w, int bits, const float* static_scale, void* z_limbs,
+                                              float* scale_out, void* stream) {
+    return hq::launch_hadamard_quant_width2(x, xdt, Nb, H, W, C, had_block_w, bits, static_scale, z_limbs, scale_out,
+                                            static_cast<cudaStream_t>(stream));
 }
 
 extern "C" hq_status hq_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx,

@@ -24,6 +24,7 @@ constexpr int kTileN = 128;
 int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
 int limbs_for(int w_bits, int had_block, hq_weight_mode mode) {
+    if (mode == HQ_W_PLAIN_A2) return 2;
     if (mode != HQ_W_FOLDED || had_block <= 1) return 1;
     return (int64_t(had_block) << (w_bits - 1)) > 128 ? 2 : 1;
 }
@@ -60,7 +61,8 @@ extern "C" int64_t hq_weight_blob_bytes(int64_t N, int32_t RS, int64_t C, int32_
                                         hq_weight_mode mode) {
     if (N <= 0 || RS <= 0 || C <= 0) return 0;
     const int limbs = hq::limbs_for(w_bits, had_block, mode);
-    return hq::round_up(N, hq::kTileN) * limbs * RS * hq::round_up(C, hq::kTileK);
+    const int64_t Ck = mode == HQ_W_PLAIN_A2 ? 2 * C : C;          // channels per tap along K
+    return hq::round_up(N, hq::kTileN) * limbs * RS * hq::round_up(Ck, hq::kTileK);
 }
 
 extern "C" hq_status hq_weight_prepare(const float* w, int64_t N, int32_t RS, int64_t C, int32_t w_bits,
@@ -69,14 +71,17 @@ extern "C" hq_status hq_weight_prepare(const float* w, int64_t N, int32_t RS, in
     using namespace hq;
     if (w == nullptr || blob == nullptr || s_w == nullptr || desc == nullptr) return HQ_ERR_INVALID_ARG;
     if (w_bits != 4 && w_bits != 8) return HQ_ERR_INVALID_ARG;
-    if (mode != HQ_W_PLAIN && mode != HQ_W_FOLDED && mode != HQ_W_DOUBLE) return HQ_ERR_INVALID_ARG;
+    if (mode != HQ_W_PLAIN && mode != HQ_W_FOLDED && mode != HQ_W_DOUBLE && mode != HQ_W_PLAIN_A2) return HQ_ERR_INVALID_ARG;
+    if (mode == HQ_W_PLAIN_A2 && container != HQ_CODES_INT8) return HQ_ERR_SHAPE;
     if (container != HQ_CODES_NIBBLE && container != HQ_CODES_INT8) return HQ_ERR_INVALID_ARG;
     if (N <= 0 || RS <= 0 || C <= 0) return HQ_ERR_SHAPE;
     const int n = had_block > 1 ? had_block : 1;
     if (n > 1 && (!is_pow2(n) || C % n != 0)) return HQ_ERR_SHAPE;
     if (container == HQ_CODES_NIBBLE && C % 8 != 0) return HQ_ERR_SHAPE;
     const int limbs = limbs_for(w_bits, had_block, mode);
-    const int64_t C_pad = round_up(C, kTileK), N_pad = round_up(N, kTileN);
+    const bool a2 = mode == HQ_W_PLAIN_A2;
+    const int64_t Ck = a2 ? 2 * C : C;                              // channels per tap along K
+    const int64_t C_pad = round_up(Ck, kTileK), N_pad = round_up(N, kTileN);
     const int64_t Kp = int64_t(RS) * C_pad;
     const int64_t need = N_pad * limbs * Kp;
     if (blob_bytes < need) return HQ_ERR_WORKSPACE;
@@ -103,8 +108,10 @@ extern "C" hq_status hq_weight_prepare(const float* w, int64_t N, int32_t RS, in
 
         const int64_t grp = o / kTileN, within = o % kTileN;
         for (int t = 0; t < RS; ++t) {
-            for (int64_t c = 0; c < C; ++c) {
-                const int32_t v = B[t * C + c];
+            for (int64_t c = 0; c < Ck; ++c) {
+                // two activation limbs: the channels of a tap are [hi(C) | lo(C)] and B = [256 Q(W) | Q(W)], whose limb
+                // split below gives the "hi" rows [Q(W) | 0] and the "lo" rows [0 | Q(W)]
+                const int32_t v = a2 ? (c < C ? 256 * B[t * C + c] : B[t * C + (c - C)]) : B[t * C + c];
                 max_abs = std::max(max_abs, v < 0 ? -v : v);
                 // position along K inside the tap
                 int64_t pos = c;
@@ -128,7 +135,7 @@ extern "C" hq_status hq_weight_prepare(const float* w, int64_t N, int32_t RS, in
             }
         }
     }
-    desc->N = N; desc->C = C; desc->RS = RS; desc->w_bits = w_bits; desc->had_block = had_block;
+    desc->N = N; desc->C = Ck; desc->RS = RS; desc->w_bits = w_bits; desc->had_block = had_block;
     desc->mode = int32_t(mode); desc->limbs = limbs; desc->container = int32_t(container);
     desc->C_pad = C_pad; desc->N_pad = N_pad; desc->bytes = need; desc->max_abs_b = max_abs; desc->reserved = 0;
     return HQ_OK;

@@ -113,3 +113,80 @@ def test_qconv_width_layer_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, str
     assert rel_err(y.float().cpu().numpy(), y_own) <= (Y_BF16_RTOL if odt == "bf16" else Y_F32_RTOL)
     rms = np.sqrt(np.mean((y.float().cpu().numpy() - ref["y"]) ** 2)) / np.sqrt(np.mean(ref["y"] ** 2))
     assert rms <= Y_BF16_RTOL
+
+
+WIDE_CASES = [
+    # Nb, H, W, C, had_block_w, bits, dtype
+    (2, 6, 32, 64, 32, 4, "f32"),       # the full width of a 32-wide map as one block
+    (1, 5, 64, 32, 64, 4, "bf16"),      # ... of a 64-wide map
+    (2, 3, 64, 16, 32, 4, "f32"),       # two 32-blocks
+    (2, 4, 64, 8, 64, 3, "f32"),
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,n,bits,dt", WIDE_CASES)
+def test_width_quant_two_limbs_matches_oracle(env, oracle, Nb, H, W, C, n, bits, dt):
+    """Blocks of 32 and 64 positions: z = q * H_raw leaves as two int8 limbs per channel, [hi | lo] per pixel."""
+    torch, hq = env
+    x = inputs.activations((Nb, H, W, C), outlier_count=max(1, C // 50), outlier_scale=20.0, seed=W + C + n)
+    x[:, :, ::n, 1] = 1000.0         # a spike at the head of every block of channel 1: flat after the transform, so that
+    xt = torch.from_numpy(x).cuda()  # all n codes sit at qmax and z = q * H_raw reaches n * qmax, beyond a signed byte
+    if dt == "bf16":
+        xt = xt.to(torch.bfloat16)
+        x = xt.float().cpu().numpy()
+    u = oracle.transform_width(x, n)
+    S = float(np.float32(np.abs(u).max() / oracle.qmax(bits) / 2.5))
+    zl = torch.full((Nb, H, W, 2 * C), 77, dtype=torch.int8, device="cuda")
+    so = torch.zeros((1,), dtype=torch.float32, device="cuda")
+    hq.hq_hadamard_quant_width2(xt, n, bits, torch.tensor([S], dtype=torch.float32, device="cuda"), zl, so)
+    torch.cuda.synchronize()
+    zz = zl.cpu().numpy().astype(np.int64)
+    hi, lo = zz[..., :C], zz[..., C:]
+    assert lo.min() >= -128 and lo.max() <= 127
+    z_gpu = 256 * hi + lo
+    q_ref, _, v = oracle.quantize(u, bits, static_scale=S, want_v=True)
+    q_gpu = codes_from_z(z_gpu, n, closed_form_H(n))
+    bad = q_gpu != q_ref
+    full = max(float(np.abs(v).max()), 1.0)
+    dist = np.abs(v - (np.floor(v) + 0.5))
+    PARITY_STATS.append(dict(what=f"width-axis two limbs {Nb}x{H}x{W}x{C} n={n} b={bits} {dt}", codes=int(q_ref.size),
+                             mismatch_frac=float(bad.mean()), max_tie_rel=float((dist[bad] / full).max()) if bad.any() else 0.0))
+    if bad.any():
+        assert np.abs(q_gpu - q_ref)[bad].max() == 1 and bad.mean() <= CODE_MISMATCH_FRAC
+        assert np.all(dist[bad] <= CODE_TIE_REL * full)
+    assert np.array_equal(z_gpu, oracle.codes_inverse_width(q_gpu.astype(np.int8), n).astype(np.int64))
+    assert np.abs(z_gpu).max() > 127                           # the case needs the second limb
+    assert np.isclose(float(so.cpu()[0]), np.float32(S) * 2.0 ** (-0.5 * np.log2(n)), rtol=1e-6)
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,R,stride,n,odt", [
+    (2, 32, 32, 128, 128, 3, 1, 32, "bf16"),     # the full-width transform of Eq. 13 on a 32-wide map
+    (1, 16, 64, 64, 200, 3, 1, 64, "f32"),       # ... on a 64-wide map, ragged Cout
+    (2, 32, 32, 64, 64, 3, 2, 32, "f32"),        # stride 2
+])
+def test_qconv_width_two_limbs_layer_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, stride, n, odt):
+    torch, hq = env
+    x = inputs.activations((Nb, H, W, C), outlier_count=max(1, C // 100), outlier_scale=20.0, seed=H + C)
+    w = inputs.weights((Cout, R, R, C), seed=Cout + R)
+    b = inputs.bias(Cout, seed=2)
+    pad = R // 2
+    S = float(np.float32(np.abs(oracle.transform_width(x, n)).max() / 7 / 2.0))
+    pw = hq.hq_weight_prepare(w, 4, 1, hq.HQ_W_PLAIN_A2, hq.HQ_CODES_INT8).to_device()
+    assert pw.desc.C == 2 * C and pw.desc.limbs == 2
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
+    y = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16 if odt == "bf16" else torch.float32, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(Nb * H * W, 2 * C, hq.HQ_CODES_INT8),), dtype=torch.uint8, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_qconv_width(torch.from_numpy(x).cuda(), pw, R, R, stride, pad, torch.from_numpy(b).cuda(), 4, n,
+                      torch.tensor([S], dtype=torch.float32, device="cuda"), y, ws, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    ref = oracle.qconv_width(x, w, b, a_bits=4, w_bits=4, had_block_w=n, stride=stride, pad=pad, static_scale=S)
+    zz = ws[: Nb * H * W * 2 * C].view(torch.int8).cpu().numpy().reshape(Nb, H, W, 2 * C).astype(np.int64)
+    z_gpu = 256 * zz[..., :C] + zz[..., C:]
+    assert (z_gpu != ref["z"]).mean() <= n * CODE_MISMATCH_FRAC          # one code touches the n positions of its block
+    assert np.array_equal(pw.s_w, ref["s_w"])
+    y_own = oracle.dequant(oracle.conv2d_int_z(z_gpu.astype(np.int32), ref["B"], stride, pad), ref["s_a"], pw.s_w, b, ref["alpha"])
+    assert rel_err(y.float().cpu().numpy(), y_own) <= (Y_BF16_RTOL if odt == "bf16" else Y_F32_RTOL)
+    rms = np.sqrt(np.mean((y.float().cpu().numpy() - ref["y"]) ** 2)) / np.sqrt(np.mean(ref["y"] ** 2))
+    assert rms <= Y_BF16_RTOL
