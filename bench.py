@@ -324,6 +324,18 @@ def measure_variants(torch, hq, device, layers, status, stream, rank):
         g.setdefault(L["name"], []).append(b.elapsed_time(c2))
     out["one_limb_gemm_ms"] = {k: float(np.median(v)) for k, v in g.items()}
     del plain
+    # --- transform + quantization fused into the product kernel's operand tile (one kernel, no codes in memory)
+    if layers[0]["cont"] == 1:
+        fused = {}
+        for L in layers:
+            if L["kind"] != "linear" or L["K"] not in (128, 256, 512):
+                continue
+            one = per_pass(lambda: hq.hq_qlinear_fused(L["x"], L["pw"], L["bias"], A_BITS, L["y"], dev_status=status, stream=stream))
+            two = per_pass(lambda: hq.hq_qlinear(L["x"], L["pw"], L["bias"], A_BITS, L["y"], L["ws"], dev_status=status, stream=stream))
+            fused[L["name"]] = dict(one_kernel_ms=one, two_kernels_ms=two)
+        out["fused_operand_load"] = dict(per_layer=fused,
+                                         note="hq_qlinear_fused (activation tile stationary, transform by the epilogue warps) "
+                                              "against hq_qlinear (two kernels, dependent launch), whole layer")
     # --- the same convolution with the width-axis transform (the paper's literal form; one weight limb)
     pw_w = hq.hq_weight_prepare(inputs.config_conv_small(seed=rank, batch=1)["w"], W_BITS, 1, hq.HQ_W_PLAIN,
                                 hq.HQ_CODES_INT8).to_device(device)

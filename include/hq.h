@@ -163,6 +163,16 @@ hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W
                    const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
                    int32_t* dev_status, void* stream);
 
+/* ---- The fused linear layer as ONE kernel: the transform and the quantization run inside the product kernel and write
+ * their codes straight into the shared-memory operand tile the tensor core reads (the "online" transform of the
+ * Single-Hadamard schematic, Eq. 10 -> Eq. 3 -> Eq. 12, without a trip of the codes through memory).  No workspace.
+ * Same arithmetic and results as hq_qlinear.  Covers K in {128, 256, 512} (the whole reduction in one operand tile),
+ * had_block in 32 .. K, weights prepared for the INT8 container, bf16 output with a 16-byte aligned pitch; anything else
+ * returns HQ_ERR_UNSUPPORTED (use hq_qlinear). */
+hq_status hq_qlinear_fused(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64_t ldx, const hq_weight_desc* desc,
+                           const void* w_dev, const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                           const float* static_scale, void* y, int64_t ldy, int32_t* dev_status, void* stream);
+
 /* ---- Eq. 13 + Eq. 14 with the transform on the WIDTH axis, as the paper states the convolution ---------------------
  * The paper reshapes X_c [B][Cin][h][w] to (B*Cin*h) x w and multiplies by the block-diagonal H_c (w x w): every
  * image row of every channel is transformed along w.  The weights are quantized untransformed and the integer core

@@ -49,6 +49,8 @@ __global__ void __launch_bounds__(128, 1) mma_probe_kernel(int iters, int32_t* d
     if (threadIdx.x < 32) tmem_dealloc(tmem_base, 256);
 }
 
+}  // namespace
+
 // ---- host side ------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -117,6 +119,8 @@ int sm_count() {
     }
     return cached[dev];
 }
+
+namespace {
 
 // Ring depth and weight residency for a problem; fills p.stages / p.b_resident and returns the shared-memory size.
 size_t plan_smem(GemmParams& p, bool frag) {

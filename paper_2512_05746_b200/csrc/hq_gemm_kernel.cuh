@@ -987,4 +987,11 @@ cudaError_t launch_nibble_conv(int mode, int grid, size_t smem, cudaStream_t st,
                                const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p);
 
 }  // namespace gemm
+
+// Host helpers defined in hq_gemm.cu: tensor-map encoders (byte matrices with an optional 128-byte swizzle; the bf16
+// output map with 32 x 32 boxes in the 64-byte swizzle) and the SM count of the current device.
+bool encode_2d(CUtensorMap* tm, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
+               uint32_t box_inner, uint32_t box_rows, bool swizzle128);
+bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy);
+int sm_count();
 }  // namespace hq

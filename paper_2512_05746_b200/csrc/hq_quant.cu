@@ -14,12 +14,11 @@
 //   gn_stats_kernel / gn_finalize_kernel   per-(sample, group) statistics for the GroupNorm prologue.
 // The butterflies run unnormalised (H_raw); 2^(-k/2) is folded into the scale (Eq. 7).
 #include "hq_common.cuh"
+#include "hq_fwht.cuh"
 
 namespace hq {
 namespace {
 
-constexpr float kMagic = 12582912.0f;            // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
-constexpr uint32_t kMagicBits = 0x4B400000u;
 
 struct QuantParams {
     const void* x;
@@ -67,73 +66,6 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
     return f;
 }
 
-// ---- two-wide fp32 arithmetic (one instruction for a pair of values held in a 64-bit register) -----------------
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pk2(float lo, float hi) { f32x2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
-__device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { f32x2 r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
-
-// Butterflies over pair-index bits: element distance 2*h for h = LO .. HI (pairs stay pairs).
-template <int P, int LO, int HI>
-__device__ __forceinline__ void butterflies_pairs(f32x2 (&v)[P]) {
-#pragma unroll
-    for (int h = LO; h <= HI; h <<= 1) {
-#pragma unroll
-        for (int i = 0; i < P; ++i) {
-            if (!(i & h)) {
-                const f32x2 a = v[i], b = v[i | h];
-                v[i] = add2(a, b);
-                v[i | h] = sub2(a, b);
-            }
-        }
-    }
-}
-// The stage between the two values of each pair.
-template <int P>
-__device__ __forceinline__ void butterfly_within_pairs(f32x2 (&v)[P]) {
-#pragma unroll
-    for (int i = 0; i < P; ++i) {
-        float a, b;
-        upk2(v[i], a, b);
-        v[i] = pk2(a + b, a - b);
-    }
-}
-
-__host__ __device__ constexpr int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
-
-// Rounds E values held as pairs (ties to even, optional clamp) and packs them in register order into words: 8
-// four-bit codes or 4 bytes per word.  Each rounded value is kMagicBits + (code + bias); summing the shifted bit
-// patterns and removing the shifted constants leaves the biased fields, which one XOR turns into two's complement.
-template <int E, bool INT8_OUT, bool CLAMP>
-__device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, int bits, uint32_t (&out)[INT8_OUT ? E / 4 : E / 8]) {
-    const float bias = INT8_OUT ? 128.0f : 8.0f;
-    const float mb = kMagic + bias;
-    const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
-    const f32x2 inv2 = pk2(inv, inv), mb2 = pk2(mb, mb);
-    constexpr int PER_WORD = INT8_OUT ? 4 : 8;
-    constexpr int SHIFT = INT8_OUT ? 8 : 4;
-    uint32_t cst = 0;
-#pragma unroll
-    for (int e = 0; e < PER_WORD; ++e) cst += kMagicBits << (SHIFT * e);
-    constexpr uint32_t UNBIAS = INT8_OUT ? 0x80808080u : 0x88888888u;
-#pragma unroll
-    for (int w = 0; w < E / PER_WORD; ++w) {
-        uint32_t acc = 0;
-#pragma unroll
-        for (int e = 0; e < PER_WORD; e += 2) {
-            float f0, f1;
-            upk2(fma2(v[(w * PER_WORD + e) / 2], inv2, mb2), f0, f1);
-            if (CLAMP) { f0 = fminf(fmaxf(f0, lo), hi); f1 = fminf(fmaxf(f1, lo), hi); }
-            acc += __float_as_uint(f0) << (SHIFT * e);
-            acc += __float_as_uint(f1) << (SHIFT * (e + 1));
-        }
-        out[w] = (acc - cst) ^ UNBIAS;
-    }
-}
-
 // Fast path.  A Hadamard block of n = 2^KLOG channels is owned by TB = n / E threads that hold E values each, as
 // E/2 two-wide registers (butterflies between pairs are one instruction per two values).
 //   phase A  thread t holds the float4s {t + TB i}: coalesced 16-byte loads; the E-point in-register transform
@@ -161,7 +93,6 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     constexpr int TB = N / E;                          // threads per Hadamard block
     constexpr int R = KLOG - LE;                       // index bits left for phase B
     constexpr bool PAIR = R >= LE - 1;
-    constexpr bool SHUF = R == LE;
     static_assert(R <= LE, "block too large for this thread shape");
     constexpr int J = PAIR ? E / 2 : E / 4;            // float4 slots a phase-B thread (pair) walks
     constexpr int S = ilog2_c(J);
@@ -263,41 +194,9 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
             v[2 * i + 1] = valid ? fma2(mul2(v[2 * i + 1], rstd2), pk2(a4.z, a4.w), pk2(b4.z, b4.w)) : pk2(0.f, 0.f);
         }
     }
-    butterfly_within_pairs<P>(v);                      // index bit 0
-    butterflies_pairs<P, 1, P / 2>(v);                 // index bit 1 and the top LE-2 bits
-
     float4* grp = xch + (tid / TB) * GS;
-    {
-        // slot f = tb + TB i sits at f + f / J; with TB and J dividing one another that is a per-thread base plus a
-        // compile-time offset
-        ulonglong2* wr = reinterpret_cast<ulonglong2*>(grp + tb + (tb >> S));
-#pragma unroll
-        for (int i = 0; i < E / 4; ++i) wr[TB * i + ((TB * i) >> S)] = make_ulonglong2(v[2 * i], v[2 * i + 1]);
-    }
-    if (TB > 32 || shared_max) __syncthreads(); else __syncwarp();
-    if (!PAIR) {
-        const ulonglong2* rd = reinterpret_cast<const ulonglong2*>(grp + (J + 1) * tb);
-#pragma unroll
-        for (int j = 0; j < E / 4; ++j) {
-            const ulonglong2 q = rd[j];
-            v[2 * j] = q.x; v[2 * j + 1] = q.y;
-        }
-        butterflies_pairs<P, 2, (2 << R) / 2>(v);      // index bits 2 .. R+1 are pair-index bits 1 .. R
-    } else {
-        const f32x2* rd = reinterpret_cast<const f32x2*>(grp + (J + 1) * (tb >> 1)) + (tb & 1);
-#pragma unroll
-        for (int j = 0; j < P; ++j) v[j] = rd[2 * j];
-        butterflies_pairs<P, 1, P / 2>(v);             // index bits 2 .. LE are pair-index bits 0 .. LE-2
-        if (SHUF) {                                    // index bit LE+1 lives in lane bit 1
-            const float sgn = (tb & 2) ? -1.0f : 1.0f;
-            const f32x2 sgn2 = pk2(sgn, sgn);
-#pragma unroll
-            for (int e = 0; e < P; ++e) {
-                const f32x2 other = __shfl_xor_sync(0xffffffffu, v[e], 2);
-                v[e] = fma2(sgn2, v[e], other);
-            }
-        }
-    }
+    if (TB > 32 || shared_max) fwht_stages<KLOG, E, true>(v, grp, tb);
+    else fwht_stages<KLOG, E, false>(v, grp, tb);
 
     float inv, scale;
     if (!STATIC) {
@@ -332,26 +231,7 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
 
     constexpr int NW = INT8_OUT ? E / 4 : E / 8;       // packed words per thread
     uint32_t w[NW];
-    round_pack<E, INT8_OUT, STATIC>(v, inv, p.bits, w);
-    if (PAIR) {
-        // w holds the codes of channel pairs {4j, 4j+1} (+2 for the odd thread).  The even thread of a pair emits
-        // the first half of the group's bytes, the odd thread the second half; each needs the other's words of
-        // that half, fetched with one exchange, and interleaves at pair granularity (1 byte or 2 bytes).
-        constexpr int H = NW / 2;
-        const bool odd = tb & 1;
-        uint32_t o[NW];
-#pragma unroll
-        for (int i = 0; i < H; ++i) {
-            const uint32_t send = odd ? w[i] : w[i + H];
-            const uint32_t keep = odd ? w[i + H] : w[i];
-            const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
-            const uint32_t ev = odd ? recv : keep, od = odd ? keep : recv;
-            o[2 * i + 0] = __byte_perm(ev, od, INT8_OUT ? 0x5410 : 0x5140);
-            o[2 * i + 1] = __byte_perm(ev, od, INT8_OUT ? 0x7632 : 0x7362);
-        }
-#pragma unroll
-        for (int i = 0; i < NW; ++i) w[i] = o[i];
-    }
+    pack_codes<KLOG, E, INT8_OUT, STATIC>(v, inv, p.bits, tb, w);
     if (valid) {
         uint8_t* dst = p.codes + row * p.ld_codes + (int64_t(blk) * N + E * tb) / (INT8_OUT ? 1 : 2);
 #pragma unroll

@@ -263,3 +263,64 @@ def test_qlinear_w8a8(env, oracle, M, K, N, n):
     # with 8 bits on both sides the Double-Hadamard layer is close to the float product
     xw = x.astype(np.float64) @ w.astype(np.float64).T + b
     assert rms_rel(y_gpu, xw) <= 2e-2
+
+
+FUSED_CASES = [
+    # M, K, N, had_block, mode, a_bits, dtype, static
+    (256, 256, 256, 256, "folded", 4, "f32", False),      # the small linear configuration
+    (1000, 512, 384, 512, "folded", 4, "f32", False),     # ragged rows, three column tiles
+    (777, 512, 200, 256, "folded", 4, "bf16", False),     # two Hadamard blocks per row, ragged columns
+    (300, 128, 72, 128, "plain", 3, "f32", False),        # one K block, one weight limb
+    (2500, 256, 520, 64, "double", 4, "bf16", False),     # four blocks per row; several row tiles per CTA range
+    (640, 512, 256, 32, "folded", 4, "f32", True),        # static scale, 16 blocks per row (one lane each)
+    (40000, 512, 640, 512, "folded", 4, "f32", False),    # more tiles than CTAs: ranges that start inside a row tile
+]
+
+
+@pytest.mark.parametrize("M,K,N,n,mode,a_bits,dt,static", FUSED_CASES)
+def test_qlinear_fused_single_kernel(env, oracle, M, K, N, n, mode, a_bits, dt, static):
+    """The one-kernel fused layer: its output against the oracle's rescale of the integer product of the ORACLE's codes
+    (the codes never leave the chip), allowing for the few codes on rounding ties; and bit-for-bit against the two-kernel
+    hq_qlinear, which runs the same arithmetic."""
+    torch, hq = env
+    x = inputs.activations((M, K), dist="student_t3", outlier_count=max(1, K // 100), outlier_scale=30.0, seed=M + K)
+    w, b = inputs.weights((N, K), seed=N), inputs.bias(N, seed=N)
+    xt = torch.from_numpy(x).cuda()
+    if dt == "bf16":
+        xt = xt.to(torch.bfloat16)
+        x = xt.float().cpu().numpy()
+    cont = hq.HQ_CODES_INT8
+    pw = hq.hq_weight_prepare(w, 4, n, hq.WEIGHT_MODES[mode], cont).to_device()
+    bd = torch.from_numpy(b).cuda()
+    s0 = None
+    ss = None
+    if static:
+        s0 = float(np.float32(np.abs(oracle.transform(x, n)).max() / oracle.qmax(a_bits) / 3.0))
+        ss = torch.tensor([s0], dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y = torch.full((M, N), 9.0, dtype=torch.bfloat16, device="cuda")
+    hq.hq_qlinear_fused(xt, pw, bd, a_bits, y, static_scale=ss, dev_status=status)
+    y2 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.zeros((hq.hq_workspace_size(M, K, cont),), dtype=torch.uint8, device="cuda")
+    hq.hq_qlinear(xt, pw, bd, a_bits, y2, ws, static_scale=ss, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    assert torch.equal(y, y2), "one-kernel and two-kernel layers differ"
+    idx = np.arange(M) if M <= 3000 else np.sort(np.random.default_rng(5).choice(M, size=192, replace=False))
+    ref = oracle.qlinear(x[idx], w, b, a_bits=a_bits, w_bits=4, had_block=n, weight_mode=mode, static_scale=s0)
+    q_gpu, s_gpu = _codes_from_ws(hq, ws, M, K, cont)            # the two-kernel path's codes: the same arithmetic
+    v = ref["v"] if not static else np.clip(ref["v"], oracle.qmin(a_bits) - 0.25, oracle.qmax(a_bits) + 0.25)
+    check_codes(q_gpu[idx], ref["q"], v, "fused one-kernel linear")
+    B = weight_integers(oracle, pw, w, 4, n, mode)
+    sa = s_gpu[idx] if not static else np.array([s0], np.float32)
+    y_own = oracle.dequant(oracle.gemm_int(q_gpu[idx], B), sa, pw.s_w, b, pw.alpha)
+    assert rel_err(y.float().cpu().numpy()[idx], y_own) <= Y_BF16_RTOL
+
+
+def test_qlinear_fused_refuses_other_shapes(env):
+    torch, hq = env
+    x = torch.zeros((64, 1024), device="cuda")
+    pw = hq.hq_weight_prepare(inputs.weights((128, 1024), seed=0), 4, 1024, hq.HQ_W_FOLDED, hq.HQ_CODES_INT8).to_device()
+    with pytest.raises(hq.HqError) as e:
+        hq.hq_qlinear_fused(x, pw, None, 4, torch.zeros((64, 128), dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == 3
