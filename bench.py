@@ -324,6 +324,29 @@ def measure_variants(torch, hq, device, layers, status, stream, rank):
         g.setdefault(L["name"], []).append(b.elapsed_time(c2))
     out["one_limb_gemm_ms"] = {k: float(np.median(v)) for k, v in g.items()}
     del plain
+    # --- the short-reduction products on pairs of SMs (tcgen05.mma.cta_group::2), GEMM only, codes already in the workspaces
+    if layers[0]["cont"] == 1:
+        def gemm_only_ms(sub):
+            evs2 = []
+            for _ in range(40):
+                run_step_split(torch, hq, sub, status, evs2, gemm_only=True)
+            torch.cuda.synchronize()
+            acc = {}
+            for L, a, b, c2 in evs2[len(sub) * 10:]:
+                acc.setdefault(L["name"], []).append(b.elapsed_time(c2))
+            return {k: float(np.median(v)) for k, v in acc.items()}
+        lin = [L for L in layers if L["kind"] == "linear" and L["K"] <= 512]
+        one_cta = gemm_only_ms(lin)
+        before = hq.hq_set_pair_gemm(True)
+        try:
+            paired = gemm_only_ms(lin)
+        finally:
+            hq.hq_set_pair_gemm(before)
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        pr_ms = per_pass(lambda: hq.hq_mma_i8_probe_pair(sms // 2, 20000, dev_status=status, stream=stream))
+        out["gemm_on_sm_pairs"] = dict(per_layer={k: dict(one_cta_ms=one_cta[k], pair_ms=paired[k]) for k in one_cta},
+                                       paired_mma_probe_tops=(sms // 2) * 20000 * 2.0 * 256 * 256 * 32 / (pr_ms * 1e-3) / 1e12,
+                                       note="hq_set_pair_gemm(1): 2-CTA clusters, each CTA half of the weight tile; GEMM launches only")
     # --- transform + quantization fused into the product kernel's operand tile (one kernel, no codes in memory)
     if layers[0]["cont"] == 1:
         fused = {}

@@ -333,6 +333,11 @@ hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, 
                              int a_bits, hq_scale_mode mode, const float* static_scale, void* y, hq_dtype ydt,
                              int64_t ldy, int32_t* dev_status, void* stream);
 
+/* Tuning switch: whether hq_qgemm and the fused layer calls run short-reduction products (K_pad <= 512, one code per
+ * byte, bf16 output, M >= 256) on pairs of SMs (tcgen05.mma.cta_group::2: each CTA of a 2-CTA cluster holds half of the
+ * weight tile).  Results are identical either way.  Returns the previous setting.  Process-wide, not thread-safe. */
+int hq_set_pair_gemm(int enable);
+
 /* alpha of the rescale for a descriptor: 2^(-k/2) for FOLDED weights (the second normalisation of Eq. 12), else 1. */
 float hq_alpha_for(const hq_weight_desc* desc);
 
@@ -340,6 +345,9 @@ float hq_alpha_for(const hq_weight_desc* desc);
  * Runs `iters` back-to-back 128x256x32 int8 MMAs per SM on resident shared-memory tiles on `ctas` CTAs.
  * The caller times it with events; ops = ctas * iters * 2*128*256*32.  dev_status as above. */
 hq_status hq_mma_i8_probe(int ctas, int iters, int32_t* dev_status, void* stream);
+/* The same for the paired MMA (tcgen05.mma.cta_group::2, 256x256x32 per 2-CTA cluster): `pairs` clusters;
+ * ops = pairs * iters * 2*256*256*32. */
+hq_status hq_mma_i8_probe_pair(int pairs, int iters, int32_t* dev_status, void* stream);
 
 #if defined(__GNUC__)
 #pragma GCC visibility pop

@@ -27,7 +27,7 @@ EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_qua
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
            "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv", "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast",
            "hq_class_embed_add", "hq_timestep_embedding", "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act",
-           "hq_conv2d_direct", "hq_attention", "hq_hadamard_quant_width2", "hq_qlinear_fused"]
+           "hq_conv2d_direct", "hq_attention", "hq_hadamard_quant_width2", "hq_qlinear_fused", "hq_set_pair_gemm", "hq_mma_i8_probe_pair"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -71,6 +71,10 @@ def _load():
     L.hq_qlinear_noalloc.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i32, i64,
                                      p, p]
     L.hq_hadamard_quant_width.argtypes = [p, i32, i64, i64, i64, i64, i32, i32, p, p, p, p]
+    L.hq_mma_i8_probe_pair.argtypes = [i32, i32, p, p]
+    L.hq_mma_i8_probe_pair.restype = C.c_int
+    L.hq_set_pair_gemm.argtypes = [i32]
+    L.hq_set_pair_gemm.restype = C.c_int
     L.hq_qlinear_fused.argtypes = [p, i32, i64, i64, i64, C.POINTER(WeightDesc), p, p, p, i32, i32, p, p, i64, p, p]
     L.hq_qlinear_fused.restype = C.c_int
     L.hq_hadamard_quant_width2.argtypes = [p, i32, i64, i64, i64, i64, i32, i32, p, p, p, p]
@@ -404,3 +408,12 @@ def hq_qlinear_fused(x, pw: PreparedWeight, bias, a_bits: int, y, static_scale=N
     _check(lib.hq_qlinear_fused(_dptr(x), _dtype_code(x), M, K, x.stride(0), C.byref(pw.desc), _dptr(pw.blob_dev),
                                 _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y), y.stride(0),
                                 _dptr(dev_status), _stream(stream)), "hq_qlinear_fused")
+
+
+def hq_set_pair_gemm(enable: bool) -> bool:
+    """Whether short-reduction products run on pairs of SMs (cta_group::2); returns the previous setting."""
+    return bool(lib.hq_set_pair_gemm(int(bool(enable))))
+
+
+def hq_mma_i8_probe_pair(pairs: int, iters: int, dev_status=None, stream=None) -> None:
+    _check(lib.hq_mma_i8_probe_pair(pairs, iters, _dptr(dev_status), _stream(stream)), "hq_mma_i8_probe_pair")

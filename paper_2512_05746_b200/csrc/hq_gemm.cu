@@ -19,6 +19,16 @@
 
 namespace hq {
 using namespace gemm;
+
+// hq_gemm_pair.cu: the same product on pairs of SMs (tcgen05.mma.cta_group::2) for the shapes it covers
+bool pair_kernel_covers(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,
+                        const int32_t* acc_out, bool combine_fast);
+hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
+                            const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
+                            const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
+                            bool after_quant);
+int g_pair_gemm = 0;       // hq_set_pair_gemm
+
 namespace {
 
 // ---- issue-rate probe: back-to-back MMAs on resident tiles ---------------------------------------------
@@ -214,6 +224,10 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
                   dev_status);
 
+    if (g_pair_gemm && pair_kernel_covers(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))
+        return launch_qgemm_pair(a_codes, M, K, lda, desc, w_dev, scale_a, scale_a_is_scalar, scale_w, bias, alpha, y, ldy,
+                                 dev_status, st, after_quant);
+
     CUtensorMap tmA, tmB, tmY{};
     const bool nib = cont == HQ_CODES_NIBBLE;
     if (!encode_2d(&tmA, a_codes, uint64_t(row_bytes), uint64_t(M), uint64_t(lda), nib ? kBK / 2 : kBK, kBM, !nib))
@@ -318,6 +332,12 @@ extern "C" hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bi
     return hq::launch_qconv2d(a_codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale_a,
                               scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, dev_status,
                               static_cast<cudaStream_t>(stream), false);
+}
+
+extern "C" int hq_set_pair_gemm(int enable) {
+    const int before = hq::g_pair_gemm;
+    hq::g_pair_gemm = enable ? 1 : 0;
+    return before;
 }
 
 extern "C" hq_status hq_mma_i8_probe(int ctas, int iters, int32_t* dev_status, void* stream) {

@@ -1,0 +1,495 @@
+// Integer GEMM with the rescale epilogue (Eq. 12) on PAIRS of SMs: tcgen05.mma.cta_group::2.
+//
+// Two CTAs of a cluster share one 256 x 256 x K tile: each holds its own 128 activation rows and HALF of the 256
+// operand-B rows in its shared memory (with two weight limbs: one CTA the "hi" rows, the other the "lo" rows), one lane of
+// the leader CTA issues every MMA for both tensor cores, and each CTA's tensor memory receives the 128 x 256 accumulator of
+// its own rows.  Per SM and MMA the tensor core reads 8 KB of operands from its shared memory instead of 12 KB -- the
+// shared-memory data pipe, not the tensor pipe, is what bounds the one-CTA kernel on short reductions -- and the resident
+// weight tile shrinks to 64 KB, which leaves room for an activation ring of eight stages.
+//
+// Covered: plain GEMM, one code per byte, K_pad <= 512 (weights resident), bf16 output through bulk tensor stores.
+// Every CTA issues its own TMA loads (no multicast); the loads of the second CTA signal the leader's barriers; MMA
+// completion is committed to both CTAs' barriers; the second CTA's epilogue warps release the accumulators with remote
+// barrier arrivals.  Every wait is bounded.
+#include <cuda.h>
+
+#include "hq_gemm_kernel.cuh"
+
+namespace hq {
+namespace {
+using namespace gemm;
+
+constexpr int kPairThreads = 320;              // producer warp, MMA warp, eight epilogue warps
+constexpr int kPairMaxStages = 8;
+constexpr int kPairBBytes = 128 * kBK;         // this CTA's half of a weight K block: 128 rows x 128 bytes
+constexpr int kPairParamBytes = kEpiWarps * 2 * (kBN / 2) * 4;
+
+struct PairParams {
+    int64_t M; int N, limbs, num_kb, tiles_m2, tiles_n, stages;
+    const float* scale_a; int sa_scalar;
+    const float* scale_w; const float* bias; float alpha;
+    int pdl;
+    int32_t* dev_status;
+};
+
+struct PairCtl {
+    uint64_t full[kPairMaxStages];     // leader: both CTAs' activation stages have landed
+    uint64_t empty[kPairMaxStages];    // each CTA: the MMAs that read the stage have completed
+    uint64_t bfull[kResidentKb];       // leader: both halves of a weight K block have landed
+    uint64_t bfree;                    // each CTA: the MMAs on the old weight tile have completed
+    uint64_t tfull[2];                 // each CTA: an accumulator is complete
+    uint64_t tempty[2];                // leader: both CTAs' epilogue warps have read an accumulator
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+struct PairLayout { int b_off, a_off, staging_off, param_off, ctl_off, total; };
+__host__ __device__ inline PairLayout pair_layout(int num_kb, int stages) {
+    PairLayout L;
+    L.b_off = 0;
+    L.a_off = num_kb * kPairBBytes;
+    L.staging_off = L.a_off + stages * kABytes;
+    L.param_off = L.staging_off + kEpiWarps * 2 * kStagingBytes;       // two staging buffers per epilogue warp
+    L.ctl_off = L.param_off + kPairParamBytes;
+    L.total = L.ctl_off + int(sizeof(PairCtl)) + 1024;
+    return L;
+}
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The address of the same shared-memory object in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_u32(p)), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion bytes are credited to the barrier at `bar_cluster_addr` (this CTA's or the leader's).
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on the barrier at the same offset in both CTAs of the pair once all MMAs issued so far have completed.
+__device__ __forceinline__ void mma_commit_pair(uint64_t* bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(mask)
+                 : "memory");
+}
+
+// One poll with a short suspend-time hint: barriers of this kernel are completed from the other CTA (remote arrivals,
+// multicast commits, the peer's TMA bytes), and a thread parked for long on such a barrier is not resumed promptly.
+#ifndef HQ_PAIR_WAIT_NS
+#define HQ_PAIR_WAIT_NS 64
+#endif
+__device__ __forceinline__ bool pair_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(uint32_t(HQ_PAIR_WAIT_NS))
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool wait_pair(uint64_t* bar, uint32_t parity, PairCtl* ctl, int32_t* dev_status, int32_t code) {
+    if (pair_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000000LL) {
+        if (pair_try_wait(bar, parity)) return true;
+        if (ctl->abort_flag) return false;
+    }
+    ctl->abort_flag = 1;
+    if (dev_status) atomicExch(dev_status, code);
+    return false;
+}
+
+// The row-per-lane bulk-store epilogue of the one-CTA kernel (16 columns at a time: two tensor-memory loads, 256 * hi + lo,
+// rescale, bf16 into a staging buffer in the 64-byte swizzle of the output tensor map, one bulk tensor store per 32
+// columns), with the accumulator handed back by an arrival on the LEADER's barrier (a cluster address).
+template <int LIMBS>
+__device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
+                                              const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0, int row0,
+                                              uint32_t tempty_leader) {
+    constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
+    const uint32_t wsw = (lane >> 1) & 3;
+    uint32_t hi[16], lo[16];
+    tmem_ld_32x16(t_row, hi);
+    if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
+#pragma unroll
+    for (int st = 0; st < NSTEPS; ++st) {
+        int32_t w[16];
+        tmem_ld_wait_16(hi);
+        if (LIMBS == 2) {
+            tmem_ld_wait_16(lo);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) w[j] = int32_t(hi[j]) * 256 + int32_t(lo[j]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) w[j] = int32_t(hi[j]);
+        }
+        if (st + 1 < NSTEPS) {
+            tmem_ld_32x16(t_row + uint32_t((st + 1) * 16), hi);
+            if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2 + (st + 1) * 16), lo);
+        } else {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty_leader);
+        }
+        // two staging buffers, used in turn: the copy engine must be done reading the one written two stores ago
+        unsigned char* buf = stg + ((st >> 1) & 1) * kStagingBytes;
+        unsigned char* wr = buf + lane * 64;
+        if ((st & 1) == 0) {
+            if (lane == 0) bulk_wait_read_1();
+            __syncwarp();
+        }
+        const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
+        const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float4 s0 = sw4[2 * j], s1 = sw4[2 * j + 1], c0 = b4[2 * j], c1 = b4[2 * j + 1];
+            uint4 o;
+            o.x = pack_bf16x2(fmaf(float(w[8 * j + 0]) * s0.x, sa_eff, c0.x), fmaf(float(w[8 * j + 1]) * s0.y, sa_eff, c0.y));
+            o.y = pack_bf16x2(fmaf(float(w[8 * j + 2]) * s0.z, sa_eff, c0.z), fmaf(float(w[8 * j + 3]) * s0.w, sa_eff, c0.w));
+            o.z = pack_bf16x2(fmaf(float(w[8 * j + 4]) * s1.x, sa_eff, c1.x), fmaf(float(w[8 * j + 5]) * s1.y, sa_eff, c1.y));
+            o.w = pack_bf16x2(fmaf(float(w[8 * j + 6]) * s1.z, sa_eff, c1.z), fmaf(float(w[8 * j + 7]) * s1.w, sa_eff, c1.w));
+            *reinterpret_cast<uint4*>(wr + (((2 * (st & 1) + j) ^ wsw) << 4)) = o;
+        }
+        if (st & 1) {
+            fence_proxy_async_smem();                  // the lanes' writes become visible to the copy engine
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(tmY, buf, col0 + (st >> 1) * 32, row0);
+                bulk_commit_group();
+            }
+        }
+    }
+}
+
+template <int LIMBS>
+__global__ void __launch_bounds__(kPairThreads, 1)
+qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmY, const PairParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const PairLayout L = pair_layout(p.num_kb, p.stages);
+    unsigned char* sB = smem + L.b_off;
+    unsigned char* sA = smem + L.a_off;
+    unsigned char* sStage = smem + L.staging_off;
+    float* sParam = reinterpret_cast<float*>(smem + L.param_off);
+    PairCtl* ctl = reinterpret_cast<PairCtl*>(smem + L.ctl_off);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();                 // 0: leader (issues the MMAs), 1: its peer
+    const int nstages = p.stages, num_kb = p.num_kb;
+    // the pair's contiguous range of 256-row tiles in column-tile-major order (consecutive tiles share their weights)
+    const int T = p.tiles_m2 * p.tiles_n, G = gridDim.x >> 1, c = blockIdx.x >> 1;
+    const int first = int(int64_t(c) * T / G);
+    const int count = int(int64_t(c + 1) * T / G) - first;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int k = 0; k < kResidentKb; ++k) mbar_init(&ctl->bfull[k], 1);
+        mbar_init(&ctl->bfree, 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 2 * kEpiWarps); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+        tma_prefetch_desc(&tmY);
+    }
+    if (warp == 1) { __syncwarp(); tmem_alloc_pair(&ctl->tmem_base, kTmemCols); tmem_relinquish_pair(); }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers are initialised and both tensor memories allocated
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (one per CTA, its own halves)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            int cur_n = -1, reloads = 0;
+            bool ok = true;
+            for (int i = 0; i < count && ok; ++i) {
+                const int u = first + i;
+                const int n_tile = u / p.tiles_m2, m2 = u - n_tile * p.tiles_m2;
+                if (n_tile != cur_n) {
+                    // the previous weight tile must have been read by its last MMA before it is overwritten
+                    if (reloads > 0 && !wait_pair(&ctl->bfree, uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
+                    for (int kb = 0; kb < num_kb; ++kb) {
+                        if (rank == 0) mbar_expect_tx(&ctl->bfull[kb], 2u * uint32_t(kPairBBytes));
+                        tma_load_2d_pair(sB + kb * kPairBBytes, &tmB, map_to_cta(&ctl->bfull[kb], 0), kb * kBK,
+                                         n_tile * kBN + int(rank) * 128);
+                    }
+                    cur_n = n_tile; ++reloads;
+                }
+                if (i == 0 && p.pdl) griddep_wait();       // the codes come from the kernel before this one
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!wait_pair(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
+                    if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(kABytes));
+                    tma_load_2d_pair(sA + stage * kABytes, &tmA, map_to_cta(&ctl->full[stage], 0), kb * kBK,
+                                     m2 * 256 + int(rank) * 128);
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_i8(256, kBN);
+            int stage = 0; uint32_t phase = 0;
+            int cur_n = -1, reloads = 0;
+            bool ok = true;
+            for (int i = 0; i < count && ok; ++i) {
+                const int u = first + i;
+                const int n_tile = u / p.tiles_m2, m2 = u - n_tile * p.tiles_m2;
+                bool new_b = false;
+                if (n_tile != cur_n) { cur_n = n_tile; ++reloads; new_b = true; }
+                const int as = i & 1;
+                if (!wait_pair(&ctl->tempty[as], (uint32_t(i >> 1) & 1u) ^ 1u, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (new_b && !wait_pair(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                    if (!wait_pair(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sA + stage * kABytes));
+                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sB + kb * kPairBBytes));
+#pragma unroll
+                    for (int k = 0; k < kBK / 32; ++k)
+                        mma_i8_pair(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                    mma_commit_pair(&ctl->empty[stage]);
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                mma_commit_pair(&ctl->tfull[as]);
+                // the next tile of the range starts a new weight tile: tell both producers when the MMAs on the old one are done
+                if (i + 1 < count && m2 + 1 == p.tiles_m2) mma_commit_pair(&ctl->bfree);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2-9 of both CTAs)
+        const int ew = warp - 2;
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int chalf = ew >> 2;                    // which half of the tile's columns this warp takes
+        unsigned char* stg = sStage + ew * 2 * kStagingBytes;
+        float* prm_sw = sParam + ew * 2 * (kBN / 2);
+        float* prm_b = prm_sw + kBN / 2;
+        constexpr int cols_per_tile = LIMBS == 2 ? kBN / 2 : kBN;
+        constexpr int cols_per_warp = cols_per_tile / 2;
+        const int wc0 = chalf * cols_per_warp;
+        const uint32_t tempty_leader[2] = {map_to_cta(&ctl->tempty[0], 0), map_to_cta(&ctl->tempty[1], 0)};
+        int last_n = -1;
+        bool ok = true;
+        float sa_next = 0.f;
+        if (p.pdl) griddep_wait();                    // scale_a comes from the kernel before this one
+        for (int i = 0; i < count && ok; ++i) {
+            const int u = first + i;
+            const int n_tile = u / p.tiles_m2, m2 = u - n_tile * p.tiles_m2;
+            const int as = i & 1;
+            const int col_base = n_tile * cols_per_tile;
+            if (n_tile != last_n) {
+                last_n = n_tile;
+                __syncwarp();
+                for (int cc = lane; cc < cols_per_warp; cc += 32) {
+                    const int col = col_base + wc0 + cc;
+                    prm_sw[cc] = col < p.N ? __ldg(p.scale_w + col) : 0.f;
+                    prm_b[cc] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
+                }
+                __syncwarp();
+            }
+            // the row scale of this tile was requested while the previous tile was processed
+            float sa = sa_next;
+            if (i == 0) {
+                const int64_t my_row = int64_t(m2) * 256 + int(rank) * 128 + q * 32 + lane;
+                sa = p.sa_scalar ? __ldg(p.scale_a) : (my_row < p.M ? __ldg(p.scale_a + my_row) : 0.f);
+            }
+            if (!wait_pair(&ctl->tfull[as], uint32_t(i >> 1) & 1u, ctl, p.dev_status, kStatusAccumWait)) { ok = false; break; }
+            tc_fence_after();
+            sa_next = sa;
+            if (i + 1 < count && !p.sa_scalar) {
+                const int u2 = u + 1;
+                const int n2 = u2 / p.tiles_m2, m2n = u2 - n2 * p.tiles_m2;
+                const int64_t row2 = int64_t(m2n) * 256 + int(rank) * 128 + q * 32 + lane;
+                sa_next = row2 < p.M ? __ldg(p.scale_a + row2) : 0.f;
+            }
+            const float sa_eff = p.alpha * sa;
+            const int row0 = m2 * 256 + int(rank) * 128 + q * 32;
+            const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
+            epilogue_pair<LIMBS>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as]);
+        }
+        if (lane == 0) bulk_wait_read_all();           // shared memory must outlive the copy engine's reads
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // neither CTA leaves while its peer may still signal its barriers or read its operands
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
+// Issue-rate probe of the paired int8 MMA: back-to-back 256 x 256 x 32 MMAs of a 2-CTA cluster on resident tiles.
+__global__ void __launch_bounds__(128, 1) mma_pair_probe_kernel(int iters, int32_t* dev_status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ uint64_t done_bar;
+    __shared__ uint32_t tmem_slot;
+    const uint32_t rank = cluster_rank();
+    for (int i = threadIdx.x; i < (kABytes + kPairBBytes) / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem)[i] = 0x01010101u;
+    if (threadIdx.x == 0) { mbar_init(&done_bar, 1); fence_barrier_init(); }
+    fence_proxy_async_smem();
+    if (threadIdx.x >= 32 && threadIdx.x < 64) { __syncwarp(); tmem_alloc_pair(&tmem_slot, 256); tmem_relinquish_pair(); }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    if (threadIdx.x == 0) {
+        if (rank == 0) {
+            const uint32_t idesc = make_idesc_i8(256, kBN);
+            const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(smem));
+            const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(smem + kABytes));
+            for (int i = 0; i < iters; ++i)
+                mma_i8_pair(tmem_base, a_desc + uint64_t((i & 3) * 2), b_desc + uint64_t((i & 3) * 2), idesc, i != 0 ? 1u : 0u);
+            mma_commit_pair(&done_bar);
+        }
+        mbar_wait(&done_bar, 0, dev_status, kStatusAccumWait);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (threadIdx.x >= 32 && threadIdx.x < 64) tmem_dealloc_pair(tmem_base, 256);
+}
+
+template <int LIMBS>
+cudaError_t launch_pair(int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                        const CUtensorMap& tmY, const PairParams& p) {
+    auto kern = qgemm_pair_kernel<LIMBS>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(grid)); cfg.blockDim = dim3(unsigned(kPairThreads));
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    int na = 1;
+    if (p.pdl) {
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        na = 2;
+    }
+    cfg.attrs = attr; cfg.numAttrs = unsigned(na);
+    return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
+}
+
+// How many 2-CTA clusters of this kernel the device runs at once (the SM count of a GPC need not be even).
+template <int LIMBS>
+int max_pairs(size_t smem) {
+    static int cached[64][2] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return sm_count() / 2;
+    int& slot = cached[dev][LIMBS - 1];
+    if (slot == 0) {
+        auto kern = qgemm_pair_kernel<LIMBS>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(unsigned(sm_count() / 2 * 2)); cfg.blockDim = dim3(unsigned(kPairThreads));
+        cfg.dynamicSmemBytes = smem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0)
+            n = sm_count() / 2 - 2;
+        slot = n < sm_count() / 2 ? n : sm_count() / 2;
+    }
+    return slot;
+}
+
+}  // namespace
+
+// Whether the pair kernel covers a problem (see the top of this file); the caller has validated the arguments.
+bool pair_kernel_covers(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,
+                        const int32_t* acc_out, bool combine_fast) {
+    return cont == HQ_CODES_INT8 && desc->RS == 1 && desc->C_pad <= int64_t(kResidentKb) * kBK && y != nullptr &&
+           acc_out == nullptr && ydt == HQ_BF16 && aligned16(y) && (ldy * 2) % 16 == 0 && combine_fast && M >= 256;
+}
+
+hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
+                            const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
+                            const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
+                            bool after_quant) {
+    PairParams p{};
+    p.M = M; p.N = int(desc->N); p.limbs = desc->limbs;
+    p.num_kb = int(desc->C_pad / kBK);
+    p.tiles_m2 = int((M + 255) / 256);
+    p.tiles_n = int(desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
+    p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
+    p.pdl = after_quant ? 1 : 0; p.dev_status = dev_status;
+    size_t smem = 0;
+    for (int stages = kPairMaxStages; stages >= 2; --stages) {
+        const PairLayout L = pair_layout(p.num_kb, stages);
+        if (L.total <= kSmemLimit) { p.stages = stages; smem = size_t(L.total); break; }
+    }
+    if (smem == 0) return HQ_ERR_UNSUPPORTED;
+    CUtensorMap tmA, tmB, tmY;
+    if (!encode_2d(&tmA, a_codes, uint64_t(K), uint64_t(M), uint64_t(lda), kBK, kBM, true)) return HQ_ERR_CUDA;
+    const uint64_t Kp = uint64_t(desc->C_pad);
+    if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
+    if (!encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
+    const int tiles = p.tiles_m2 * p.tiles_n;
+    const int pairs_max = desc->limbs == 2 ? max_pairs<2>(smem) : max_pairs<1>(smem);
+    const int pairs = tiles < pairs_max ? tiles : pairs_max;
+    cudaError_t e = desc->limbs == 2 ? launch_pair<2>(2 * pairs, smem, st, tmA, tmB, tmY, p)
+                                     : launch_pair<1>(2 * pairs, smem, st, tmA, tmB, tmY, p);
+    return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+}  // namespace hq
+
+extern "C" hq_status hq_mma_i8_probe_pair(int pairs, int iters, int32_t* dev_status, void* stream) {
+    using namespace hq;
+    if (pairs <= 0 || iters <= 0) return HQ_ERR_INVALID_ARG;
+    const size_t smem = 1024 + hq::gemm::kABytes + kPairBBytes;
+    HQ_CUDA_OK(cudaFuncSetAttribute(mma_pair_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(unsigned(2 * pairs)); cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem; cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mma_pair_probe_kernel, iters, dev_status) == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}

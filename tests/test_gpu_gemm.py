@@ -300,3 +300,52 @@ def test_qgemm_sweep_corner_sampled(env, oracle):
     ref = oracle.gemm_int(q, B)
     got = acc[ridx][:, torch.from_numpy(cols).cuda()].cpu().numpy().astype(np.int64)
     assert np.array_equal(got, ref)
+
+
+PAIR_CASES = [
+    # M, K, N, had_block, mode
+    (512, 256, 256, 256, "folded"),
+    (1000, 512, 384, 512, "folded"),      # ragged rows (3.9 pair tiles), three column tiles
+    (777, 512, 328, 512, "plain"),        # one weight limb, ragged columns
+    (300, 128, 72, 128, "folded"),        # one K block
+    (40000, 256, 384, 256, "double"),     # more pair tiles than clusters; the weight tile changes inside a pair's range
+    (256, 384, 136, 128, "folded"),       # three K blocks
+]
+
+
+@pytest.mark.parametrize("M,K,N,n,mode", PAIR_CASES)
+def test_qgemm_on_sm_pairs_matches_oracle(env, oracle, M, K, N, n, mode):
+    """The product on pairs of SMs (tcgen05.mma.cta_group::2, each CTA of a cluster holding half of the weight tile):
+    bf16 output against the oracle's rescale of the oracle's integer product, and bit for bit against the one-CTA
+    kernel."""
+    torch, hq = env
+    q = inputs.codes((M, K), 4, seed=M + N)
+    w = inputs.weights((N, K), seed=N)
+    pw = hq.hq_weight_prepare(w, 4, n, hq.WEIGHT_MODES[mode], hq.HQ_CODES_INT8).to_device()
+    B = weight_integers(oracle, pw, w, 4, n, mode)
+    s_a = inputs.positive_scales(M, seed=M)
+    b = inputs.bias(N, seed=N)
+    a_dev = to_container(torch, hq, q, hq.HQ_CODES_INT8)
+    sa_dev, b_dev = torch.from_numpy(s_a).cuda(), torch.from_numpy(b).cuda()
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y_one = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    y_pair = torch.full((M, N), 3.0, dtype=torch.bfloat16, device="cuda")
+    hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_one, dev_status=status)
+    before = hq.hq_set_pair_gemm(True)
+    try:
+        hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_pair, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        hq.hq_set_pair_gemm(before)
+    hq.hq_check_status(status)
+    y_ref = oracle.dequant(oracle.gemm_int(q, B), s_a, pw.s_w, b, pw.alpha)
+    assert rel_err(y_pair.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+    assert torch.equal(y_pair, y_one)
+
+
+def test_paired_tensor_pipe_probe_runs(env):
+    torch, hq = env
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_mma_i8_probe_pair(2, 64, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
