@@ -4,7 +4,8 @@
 // One CTA of 128 threads takes 128 queries of one (sample, head) and walks the keys in blocks of 128:
 //   S = Q K_j^T      tcgen05.mma kind::f16 (bf16 operands from shared memory, fp32 accumulator in tensor memory)
 //   row softmax      thread t owns query row t = lane t of tensor memory: running maximum and sum (online softmax),
-//                    P = exp2(c (S - m)) rounded to bf16 into shared memory, the output accumulator rescaled in tensor
+//                    P = exp2(c (S - m)) rounded to bf16 into shared memory (the sum runs over the unrounded values: the
+//                    roundings of 128 weights average out), the output accumulator rescaled in tensor
 //                    memory when the running maximum moved
 //   O += P V_j       tcgen05.mma again, V read as an MN-major operand so that it needs no transpose
 // and finally O / sum goes out as bf16.  Operands are staged by plain 16-byte loads into the unswizzled canonical
@@ -81,19 +82,32 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // rows_valid are zero.  Consecutive lanes take consecutive rows of a group, so the shared-memory stores of a warp fall
 // into four 128-byte runs.
 template <int DH>
-__device__ __forceinline__ void stage_tile(unsigned char* dst, const __nv_bfloat16* src, int64_t pitch, int rows_valid,
-                                           int tid) {
+__device__ __forceinline__ void fetch_tile(uint4 (&reg)[DH / 8], const __nv_bfloat16* src, int64_t pitch, int rows_valid, int tid) {
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) {
+        const int f = tid + 128 * i;
+        const int rg = f / DH, within = f - rg * DH;
+        const int row = rg * 8 + (within & 7), v = within >> 3;
+        reg[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (row < rows_valid) reg[i] = __ldg(reinterpret_cast<const uint4*>(src + int64_t(row) * pitch + v * 8));
+    }
+}
+template <int DH>
+__device__ __forceinline__ void put_tile(unsigned char* dst, const uint4 (&reg)[DH / 8], int tid) {
     constexpr int group_stride = (DH / 8) * 128;
 #pragma unroll
     for (int i = 0; i < DH / 8; ++i) {
         const int f = tid + 128 * i;
         const int rg = f / DH, within = f - rg * DH;
-        const int rl = within & 7, v = within >> 3;
-        const int row = rg * 8 + rl;
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (row < rows_valid) val = __ldg(reinterpret_cast<const uint4*>(src + int64_t(row) * pitch + v * 8));
-        *reinterpret_cast<uint4*>(dst + rg * group_stride + v * 128 + rl * 16) = val;
+        *reinterpret_cast<uint4*>(dst + rg * group_stride + (within >> 3) * 128 + (within & 7) * 16) = reg[i];
     }
+}
+template <int DH>
+__device__ __forceinline__ void stage_tile(unsigned char* dst, const __nv_bfloat16* src, int64_t pitch, int rows_valid,
+                                           int tid) {
+    uint4 reg[DH / 8];
+    fetch_tile<DH>(reg, src, pitch, rows_valid, tid);
+    put_tile<DH>(dst, reg, tid);
 }
 
 template <int DH>
@@ -132,13 +146,32 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
     uint32_t phase = 0;
     bool ok = true;
     const int nblocks = (L + kKeyBlock - 1) / kKeyBlock;
+    // The next key block's K and V pieces are requested into registers while the current block's softmax runs (head
+    // widths up to 64: 16 registers per operand), so that their latency is not on the block's critical path.
+    constexpr bool PREFETCH = DH <= 64;
+    uint4 kreg[DH / 8], vreg[DH / 8];
+    if (PREFETCH) {
+        fetch_tile<DH>(kreg, base + C, pitch, L < kKeyBlock ? L : kKeyBlock, tid);
+        fetch_tile<DH>(vreg, base + 2 * C, pitch, L < kKeyBlock ? L : kKeyBlock, tid);
+    }
     for (int j = 0; j < nblocks && ok; ++j) {
         const int k0 = j * kKeyBlock;
         const int kvalid = L - k0 < kKeyBlock ? L - k0 : kKeyBlock;
-        stage_tile<DH>(sK, base + C + int64_t(k0) * pitch, pitch, kvalid, tid);
-        stage_tile<DH>(sV, base + 2 * C + int64_t(k0) * pitch, pitch, kvalid, tid);
+        if (PREFETCH) {
+            put_tile<DH>(sK, kreg, tid);
+            put_tile<DH>(sV, vreg, tid);
+        } else {
+            stage_tile<DH>(sK, base + C + int64_t(k0) * pitch, pitch, kvalid, tid);
+            stage_tile<DH>(sV, base + 2 * C + int64_t(k0) * pitch, pitch, kvalid, tid);
+        }
         fence_proxy_async_smem();
         __syncthreads();
+        if (PREFETCH && j + 1 < nblocks) {
+            const int k1 = k0 + kKeyBlock;
+            const int kv1 = L - k1 < kKeyBlock ? L - k1 : kKeyBlock;
+            fetch_tile<DH>(kreg, base + C + int64_t(k1) * pitch, pitch, kv1, tid);
+            fetch_tile<DH>(vreg, base + 2 * C + int64_t(k1) * pitch, pitch, kv1, tid);
+        }
         // One lane issues; its warp-mates wait for it at the warp barrier instead of polling beside it (a polling loop
         // on the other side of a divergent branch can keep the issuing lane from being scheduled).
         if (warp == 0) {
@@ -160,16 +193,27 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
         if (!ok) break;
         tc_fence_after();
 
-        // ---- row maximum of this block
+        // ---- row maximum of this block (the next 32 columns are requested while the current ones are reduced)
+        const bool full = kvalid == kKeyBlock;
         float mx = -INFINITY;
+        {
+            uint32_t ra[32], rb[32];
+            tmem_ld_32x32(t_s, ra);
 #pragma unroll
-        for (int c = 0; c < kKeyBlock / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld_32x32(t_s + uint32_t(c * 32), r);
-            tmem_ld_wait_32(r);
+            for (int c = 0; c < kKeyBlock / 32; ++c) {
+                uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+                uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+                tmem_ld_wait_32(cur);
+                if (c + 1 < kKeyBlock / 32) tmem_ld_32x32(t_s + uint32_t((c + 1) * 32), nxt);
+                if (full) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-                if (c * 32 + e < kvalid) mx = fmaxf(mx, __uint_as_float(r[e]));
+                    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(cur[e]));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (c * 32 + e < kvalid) mx = fmaxf(mx, __uint_as_float(cur[e]));
+                }
+            }
         }
         const float m_new = fmaxf(m_run, mx);
         const float mc = m_new * p.scale_log2;
@@ -177,28 +221,29 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
         // ---- P = exp2(c (S - m)), row sum, bf16 into shared memory (K-major: 16 key groups of 128 bytes per row group)
         float sum = 0.f;
         unsigned char* prow = sP + (tid >> 3) * 2048 + (tid & 7) * 16;
+        {
+            uint32_t ra[32], rb[32];
+            tmem_ld_32x32(t_s, ra);
 #pragma unroll
-        for (int c = 0; c < kKeyBlock / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld_32x32(t_s + uint32_t(c * 32), r);
-            tmem_ld_wait_32(r);
-            float pv[32];
+            for (int c = 0; c < kKeyBlock / 32; ++c) {
+                uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+                uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+                tmem_ld_wait_32(cur);
+                if (c + 1 < kKeyBlock / 32) tmem_ld_32x32(t_s + uint32_t((c + 1) * 32), nxt);
+                float pv[32];
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                const float v = ex2(fmaf(__uint_as_float(r[e]), p.scale_log2, -mc));
-                pv[e] = (c * 32 + e < kvalid) ? v : 0.f;
-            }
+                for (int e = 0; e < 32; ++e) {
+                    const float v = ex2(fmaf(__uint_as_float(cur[e]), p.scale_log2, -mc));
+                    pv[e] = (full || c * 32 + e < kvalid) ? v : 0.f;
+                    sum += pv[e];
+                }
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                uint4 w;
-                w.x = pack_bf16(pv[8 * g + 0], pv[8 * g + 1]); w.y = pack_bf16(pv[8 * g + 2], pv[8 * g + 3]);
-                w.z = pack_bf16(pv[8 * g + 4], pv[8 * g + 5]); w.w = pack_bf16(pv[8 * g + 6], pv[8 * g + 7]);
-                // the sum runs over the rounded values, the ones the tensor core multiplies with V
-                sum += (__uint_as_float(w.x << 16) + __uint_as_float(w.x & 0xFFFF0000u)) +
-                       (__uint_as_float(w.y << 16) + __uint_as_float(w.y & 0xFFFF0000u)) +
-                       (__uint_as_float(w.z << 16) + __uint_as_float(w.z & 0xFFFF0000u)) +
-                       (__uint_as_float(w.w << 16) + __uint_as_float(w.w & 0xFFFF0000u));
-                *reinterpret_cast<uint4*>(prow + (c * 4 + g) * 128) = w;
+                for (int g = 0; g < 4; ++g) {
+                    uint4 w;
+                    w.x = pack_bf16(pv[8 * g + 0], pv[8 * g + 1]); w.y = pack_bf16(pv[8 * g + 2], pv[8 * g + 3]);
+                    w.z = pack_bf16(pv[8 * g + 4], pv[8 * g + 5]); w.w = pack_bf16(pv[8 * g + 6], pv[8 * g + 7]);
+                    *reinterpret_cast<uint4*>(prow + (c * 4 + g) * 128) = w;
+                }
             }
         }
         l_run = fmaf(l_run, alpha, sum);
