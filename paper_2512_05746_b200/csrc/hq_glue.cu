@@ -120,28 +120,44 @@ __global__ void __launch_bounds__(256) concat_kernel(const uint4* a, int ca8, co
     out[i] = c < ca8 ? __ldcs(a + r * ca8 + c) : __ldcs(b + r * cb8 + (c - ca8));
 }
 
-// y = act((x - mean) rstd gamma + beta) with the statistics of the element's (sample, group)
-__global__ void __launch_bounds__(256) gn_apply_kernel(const uint4* x, uint4* out, int64_t n8, int c8,
-                                                       int64_t vec_per_sample, const float* stats, const float* gamma,
+// y = act((x - mean) rstd gamma + beta) with the statistics of the element's (sample, group).  A thread keeps one channel
+// vector (8 channels) and walks pixels, so gamma / beta / the group's statistics are read once per thread and sample.
+__global__ void __launch_bounds__(256) gn_apply_kernel(const uint4* x, uint4* out, int c8, int64_t pixels_per_sample,
+                                                       int pixel_chunks, const float* stats, const float* gamma,
                                                        const float* beta, int groups, int cg, int act) {
-    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i >= n8) return;
-    const int64_t n = i / vec_per_sample;
-    const int c0 = int(i % c8) * 8;
-    F8 f = unpack8(__ldcs(x + i));
+    const int n = blockIdx.y;
+    const int lanes_c = c8 < 256 ? c8 : 256;           // channel vectors walked side by side
+    const int ppl = 256 / lanes_c;                      // pixels walked side by side
+    const int cv0 = threadIdx.x % lanes_c, pl = threadIdx.x / lanes_c;
+    if (pl >= ppl) return;
+    const int64_t per = (pixels_per_sample + pixel_chunks - 1) / pixel_chunks;
+    const int64_t p0 = int64_t(blockIdx.x) * per, p1 = p0 + per < pixels_per_sample ? p0 + per : pixels_per_sample;
+    for (int cv = cv0; cv < c8; cv += lanes_c) {
+        float a[8], b[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const int c = c0 + e;
-        const float2 st = *reinterpret_cast<const float2*>(stats + (n * groups + c / cg) * 2);
-        const float a = st.y * __ldg(gamma + c);
-        const float y = fmaf(f.v[e], a, fmaf(-st.x, a, __ldg(beta + c)));
-        f.v[e] = act ? silu_f(y) : y;
+        for (int e = 0; e < 8; ++e) {
+            const int c = cv * 8 + e;
+            const float2 st = *reinterpret_cast<const float2*>(stats + (int64_t(n) * groups + c / cg) * 2);
+            a[e] = st.y * __ldg(gamma + c);
+            b[e] = fmaf(-st.x, a[e], __ldg(beta + c));
+        }
+        const uint4* src = x + int64_t(n) * pixels_per_sample * c8 + cv;
+        uint4* dst = out + int64_t(n) * pixels_per_sample * c8 + cv;
+        for (int64_t px = p0 + pl; px < p1; px += ppl) {
+            F8 f = unpack8(__ldcs(src + px * c8));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float y = fmaf(f.v[e], a[e], b[e]);
+                f.v[e] = act ? silu_f(y) : y;
+            }
+            dst[px * c8] = pack8(f);
+        }
     }
-    out[i] = pack8(f);
 }
 
-// Convolution with few input channels (the network's first convolution): a warp takes one output pixel, each lane
-// eight consecutive output channels per round; the weights sit in shared memory as [tap * C + c][Cout].
+// Convolution with few input channels (the network's first convolution): a warp takes four consecutive output pixels of
+// a row, each lane eight consecutive output channels per round; the weights sit in shared memory as [tap * C + c][Cout] and
+// every weight read serves the four pixels.
 template <typename InT>
 __global__ void __launch_bounds__(256) conv_small_cin_kernel(const InT* x, const float* w, const float* bias,
                                                              __nv_bfloat16* out, int Nb, int H, int W, int C, int Cout,
@@ -154,47 +170,65 @@ __global__ void __launch_bounds__(256) conv_small_cin_kernel(const InT* x, const
     }
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const int64_t pixels = int64_t(Nb) * Ho * Wo;
-    for (int64_t p = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); p < pixels;
-         p += int64_t(gridDim.x) * (blockDim.x >> 5)) {
-        const int wo = int(p % Wo);
-        const int ho = int((p / Wo) % Ho);
-        const int n = int(p / (int64_t(Wo) * Ho));
+    const int wq = (Wo + 3) / 4;                       // groups of four pixels per output row
+    const int64_t groups = int64_t(Nb) * Ho * wq;
+    for (int64_t g = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); g < groups;
+         g += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo0 = int(g % wq) * 4;
+        const int ho = int((g / wq) % Ho);
+        const int n = int(g / (int64_t(wq) * Ho));
         for (int co0 = lane * 8; co0 < Cout; co0 += 256) {
-            float acc[8];
+            float acc[4][8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = bias != nullptr ? __ldg(bias + co0 + e) : 0.f;
+            for (int e = 0; e < 8; ++e) {
+                const float b = bias != nullptr ? __ldg(bias + co0 + e) : 0.f;
+#pragma unroll
+                for (int pp = 0; pp < 4; ++pp) acc[pp][e] = b;
+            }
             for (int r = 0; r < R; ++r) {
                 const int hi = ho * stride + r - pad;
                 if (hi < 0 || hi >= H) continue;
-                for (int s = 0; s < R; ++s) {
-                    const int wi = wo * stride + s - pad;
-                    if (wi < 0 || wi >= W) continue;
-                    const InT* px = x + ((int64_t(n) * H + hi) * W + wi) * C;
+                for (int sx = 0; sx < R; ++sx) {
                     for (int c = 0; c < C; ++c) {
-                        float xv;
-                        if (sizeof(InT) == 4) xv = __ldg(reinterpret_cast<const float*>(px) + c);
-                        else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(px)[c]);
-                        const float4* wr = reinterpret_cast<const float4*>(sw + ((r * R + s) * C + c) * Cout + co0);
+                        float xv[4];
+#pragma unroll
+                        for (int pp = 0; pp < 4; ++pp) {
+                            const int wi = (wo0 + pp) * stride + sx - pad;
+                            xv[pp] = 0.f;
+                            if (wi >= 0 && wi < W && wo0 + pp < Wo) {
+                                const InT* px = x + ((int64_t(n) * H + hi) * W + wi) * C + c;
+                                if (sizeof(InT) == 4) xv[pp] = __ldg(reinterpret_cast<const float*>(px));
+                                else xv[pp] = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(px));
+                            }
+                        }
+                        const float4* wr = reinterpret_cast<const float4*>(sw + ((r * R + sx) * C + c) * Cout + co0);
                         const float4 w0 = wr[0], w1 = wr[1];
-                        acc[0] = fmaf(xv, w0.x, acc[0]); acc[1] = fmaf(xv, w0.y, acc[1]);
-                        acc[2] = fmaf(xv, w0.z, acc[2]); acc[3] = fmaf(xv, w0.w, acc[3]);
-                        acc[4] = fmaf(xv, w1.x, acc[4]); acc[5] = fmaf(xv, w1.y, acc[5]);
-                        acc[6] = fmaf(xv, w1.z, acc[6]); acc[7] = fmaf(xv, w1.w, acc[7]);
+#pragma unroll
+                        for (int pp = 0; pp < 4; ++pp) {
+                            acc[pp][0] = fmaf(xv[pp], w0.x, acc[pp][0]); acc[pp][1] = fmaf(xv[pp], w0.y, acc[pp][1]);
+                            acc[pp][2] = fmaf(xv[pp], w0.z, acc[pp][2]); acc[pp][3] = fmaf(xv[pp], w0.w, acc[pp][3]);
+                            acc[pp][4] = fmaf(xv[pp], w1.x, acc[pp][4]); acc[pp][5] = fmaf(xv[pp], w1.y, acc[pp][5]);
+                            acc[pp][6] = fmaf(xv[pp], w1.z, acc[pp][6]); acc[pp][7] = fmaf(xv[pp], w1.w, acc[pp][7]);
+                        }
                     }
                 }
             }
-            F8 f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f.v[e] = acc[e];
-            *reinterpret_cast<uint4*>(out + p * Cout + co0) = pack8(f);
+            for (int pp = 0; pp < 4; ++pp) {
+                if (wo0 + pp >= Wo) continue;
+                F8 f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f.v[e] = acc[pp][e];
+                *reinterpret_cast<uint4*>(out + ((int64_t(n) * Ho + ho) * Wo + wo0 + pp) * Cout + co0) = pack8(f);
+            }
         }
     }
 }
 
-// Convolution with few output channels (the network's last convolution): a warp takes one output pixel, each lane eight
-// input channels per round of 256 for every filter tap (coalesced 512-byte reads), the weights [Cout][R][R][C] sit in
-// shared memory as they are, and the partial sums of the warp are added up by shuffles.  Output fp32.
+// Convolution with few output channels (the network's last convolution): a warp takes four consecutive output pixels of a
+// row, each lane eight input channels per round of 256 for every filter tap (coalesced 512-byte reads); the weights
+// [Cout][R][R][C] sit in shared memory as they are and every weight read serves the four pixels; the partial sums of the
+// warp are added up by shuffles.  Output fp32.
 template <int COUT>
 __global__ void __launch_bounds__(256) conv_small_cout_kernel(const __nv_bfloat16* x, const float* w, const float* bias,
                                                               float* out, int Nb, int H, int W, int C, int R, int stride,
@@ -204,43 +238,59 @@ __global__ void __launch_bounds__(256) conv_small_cout_kernel(const __nv_bfloat1
     for (int i = threadIdx.x; i < wsize; i += blockDim.x) sw[i] = w[i];
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const int64_t pixels = int64_t(Nb) * Ho * Wo;
-    for (int64_t p = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); p < pixels;
-         p += int64_t(gridDim.x) * (blockDim.x >> 5)) {
-        const int wo = int(p % Wo);
-        const int ho = int((p / Wo) % Ho);
-        const int n = int(p / (int64_t(Wo) * Ho));
-        float acc[COUT];
+    const int wq = (Wo + 3) / 4;
+    const int64_t groups = int64_t(Nb) * Ho * wq;
+    for (int64_t g = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); g < groups;
+         g += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo0 = int(g % wq) * 4;
+        const int ho = int((g / wq) % Ho);
+        const int n = int(g / (int64_t(wq) * Ho));
+        float acc[4][COUT];
 #pragma unroll
-        for (int o = 0; o < COUT; ++o) acc[o] = 0.f;
+        for (int pp = 0; pp < 4; ++pp)
+#pragma unroll
+            for (int o = 0; o < COUT; ++o) acc[pp][o] = 0.f;
         for (int r = 0; r < R; ++r) {
             const int hi = ho * stride + r - pad;
             if (hi < 0 || hi >= H) continue;
-            for (int s = 0; s < R; ++s) {
-                const int wi = wo * stride + s - pad;
-                if (wi < 0 || wi >= W) continue;
-                const __nv_bfloat16* px = x + ((int64_t(n) * H + hi) * W + wi) * C;
+            for (int sx = 0; sx < R; ++sx) {
                 for (int c0 = lane * 8; c0 < C; c0 += 256) {
-                    const F8 f = unpack8(__ldg(reinterpret_cast<const uint4*>(px + c0)));
+                    F8 f[4];
+#pragma unroll
+                    for (int pp = 0; pp < 4; ++pp) {
+                        const int wi = (wo0 + pp) * stride + sx - pad;
+                        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                        if (wi >= 0 && wi < W && wo0 + pp < Wo)
+                            raw = __ldg(reinterpret_cast<const uint4*>(x + ((int64_t(n) * H + hi) * W + wi) * C + c0));
+                        f[pp] = unpack8(raw);
+                    }
 #pragma unroll
                     for (int o = 0; o < COUT; ++o) {
-                        const float4* wr = reinterpret_cast<const float4*>(sw + (o * R * R + r * R + s) * C + c0);
+                        const float4* wr = reinterpret_cast<const float4*>(sw + (o * R * R + r * R + sx) * C + c0);
                         const float4 w0 = wr[0], w1 = wr[1];
-                        acc[o] = fmaf(f.v[0], w0.x, fmaf(f.v[1], w0.y, fmaf(f.v[2], w0.z, fmaf(f.v[3], w0.w, acc[o]))));
-                        acc[o] = fmaf(f.v[4], w1.x, fmaf(f.v[5], w1.y, fmaf(f.v[6], w1.z, fmaf(f.v[7], w1.w, acc[o]))));
+#pragma unroll
+                        for (int pp = 0; pp < 4; ++pp) {
+                            acc[pp][o] = fmaf(f[pp].v[0], w0.x, fmaf(f[pp].v[1], w0.y, fmaf(f[pp].v[2], w0.z, fmaf(f[pp].v[3], w0.w, acc[pp][o]))));
+                            acc[pp][o] = fmaf(f[pp].v[4], w1.x, fmaf(f[pp].v[5], w1.y, fmaf(f[pp].v[6], w1.z, fmaf(f[pp].v[7], w1.w, acc[pp][o]))));
+                        }
                     }
                 }
             }
         }
 #pragma unroll
-        for (int o = 0; o < COUT; ++o) {
+        for (int pp = 0; pp < 4; ++pp)
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc[o] += __shfl_xor_sync(0xffffffffu, acc[o], off);
-        }
-        if (lane == 0) {
+            for (int o = 0; o < COUT; ++o) {
 #pragma unroll
-            for (int o = 0; o < COUT; ++o) out[p * COUT + o] = acc[o] + (bias != nullptr ? __ldg(bias + o) : 0.f);
-        }
+                for (int off = 16; off > 0; off >>= 1) acc[pp][o] += __shfl_xor_sync(0xffffffffu, acc[pp][o], off);
+            }
+        // lane pp * COUT + o writes output o of pixel pp
+#pragma unroll
+        for (int pp = 0; pp < 4; ++pp)
+#pragma unroll
+            for (int o = 0; o < COUT; ++o)
+                if (lane == pp * COUT + o && wo0 + pp < Wo)
+                    out[((int64_t(n) * Ho + ho) * Wo + wo0 + pp) * COUT + o] = acc[pp][o] + (bias != nullptr ? __ldg(bias + o) : 0.f);
     }
 }
 
@@ -339,10 +389,15 @@ extern "C" hq_status hq_groupnorm_act(const void* x, int64_t Nb, int64_t H, int6
     const float* stats = nullptr;
     hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st);
     if (s != HQ_OK) return s;
-    const int64_t n8 = Nb * H * W * (C / 8);
-    gn_apply_kernel<<<blocks_for(n8, 256), 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(out), n8,
-                                                         int(C / 8), H * W * (C / 8), stats, gamma, beta, groups,
-                                                         int(C / groups), silu != 0);
+    if (Nb > 65535) return HQ_ERR_UNSUPPORTED;
+    const int c8 = int(C / 8);
+    const int64_t hw = H * W;
+    const int64_t ppl = c8 < 256 ? 256 / c8 : 1;
+    int64_t chunks = hw / (ppl * 8);                   // about 8 pixels per thread
+    chunks = chunks < 1 ? 1 : (chunks > 2048 ? 2048 : chunks);
+    gn_apply_kernel<<<dim3(unsigned(chunks), unsigned(Nb)), 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(out),
+                                                                         c8, hw, int(chunks), stats, gamma, beta, groups,
+                                                                         int(C / groups), silu != 0);
     return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
@@ -358,8 +413,8 @@ extern "C" hq_status hq_conv2d_direct(const void* x, hq_dtype xdt, const float* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t smem = size_t(R) * R * C * Cout * sizeof(float);
     if (smem > 160 * 1024) return HQ_ERR_UNSUPPORTED;
-    const int64_t pixels = Nb * Ho * Wo;
-    const int grid = int(pixels / 8 < 148 * 16 ? (pixels + 7) / 8 : 148 * 16);
+    const int64_t pixel_groups = Nb * Ho * ((Wo + 3) / 4);                    // a warp takes four pixels at a time
+    const int grid = int(pixel_groups / 8 < 148 * 16 ? (pixel_groups + 7) / 8 : 148 * 16);
     if (ydt == HQ_BF16 && C <= 16 && Cout % 8 == 0) {                          // few input channels
         if (!aligned16(y)) return HQ_ERR_ALIGNMENT;
         if (xdt == HQ_F32) {
