@@ -57,15 +57,19 @@ def ws_views(torch, ws, rows, cols):
     return ws[: rows * pitch].view(rows, pitch), ws[off: off + rows * 4].view(torch.float32)
 
 
+STEP_KERNEL_SOURCES = ("hq_common.cuh", "hq_fwht.cuh", "hq_quant.cu", "hq_gemm_kernel.cuh", "hq_gemm.cu", "hq_api.cu",
+                       "hq_gemm_inst_i8_gemm.cu", "hq_gemm_inst_i8_conv.cu", "hq_gemm_inst_nibble_gemm.cu",
+                       "hq_gemm_inst_nibble_conv.cu")
+
+
 def csrc_digest():
-    """SHA-256 over the CUDA sources and the C header, in name order: identifies the kernels a profile was taken with."""
-    import glob
+    """SHA-256 over the sources of the kernels the default step launches (transform + quantize, integer GEMM / conv and
+    their launchers): identifies the kernels a profile was taken with."""
     import hashlib
     h = hashlib.sha256()
-    files = sorted(glob.glob(os.path.join(ROOT, "paper_2512_05746_b200", "csrc", "*"))) + [os.path.join(ROOT, "include", "hq.h")]
-    for f in files:
-        with open(f, "rb") as fh:
-            h.update(os.path.basename(f).encode() + b"\0" + fh.read())
+    for name in STEP_KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2512_05746_b200", "csrc", name), "rb") as fh:
+            h.update(name.encode() + b"\0" + fh.read())
     return h.hexdigest()[:16]
 
 
