@@ -768,6 +768,38 @@ def main_sweep(args):
                           points=points)))
 
 
+def main_attn(args):
+    """The self-attention core of the UNet's 32x32 level (1024 tokens, 8 heads of 64) on its own: TFLOP/s of hq_attention.
+    --rows sets the batch (default 64; smaller for profiler captures)."""
+    import torch
+    from paper_2512_05746_b200 import binding as hq
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Nb = 64 if args.rows == 32768 else max(1, int(args.rows))
+    L, Cc, heads = 1024, 512, 8
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    sets = [(torch.randn((Nb * L, 3 * Cc), generator=gen, device=dev).to(torch.bfloat16),
+             torch.empty((Nb * L, Cc), dtype=torch.bfloat16, device=dev)) for _ in range(2)]
+    i = [0]
+
+    def call():
+        i[0] ^= 1
+        hq.hq_attention(sets[i[0]][0], Nb, heads, sets[i[0]][1], dev_status=status)
+
+    steps, warmup = max(1, min(args.steps, 50)), max(3, min(args.warmup, 5))
+    for _ in range(warmup):
+        call()
+    ms = timed_region(torch, call, steps, torch.cuda.current_stream()) / steps
+    hq.hq_check_status(status)
+    flops = 4.0 * Nb * L * L * Cc
+    print(json.dumps(dict(metric="TFLOP/s of the self-attention core (bf16 tensor cores, 4 L^2 C per sample)",
+                          value=flops / (ms * 1e-3) / 1e12, unit="TFLOP/s", n_gpus=1, steps=steps, warmup=warmup, ms_per_step=ms,
+                          higher_is_better=True, dtype="bf16", data="synthetic", vs_baseline=None,
+                          config=dict(workload=f"attention core: batch {Nb}, 1024 tokens, 8 heads x 64"), gpu_launches=steps)))
+
+
 def main_gn(args):
     """GroupNorm(32) + SiLU + transform + quantize on one NHWC bf16 tensor (64 x 64 x 64 x 256, the input of a UNet
     residual-block convolution), beside the plain transform + quantize of the same tensor."""
@@ -866,7 +898,7 @@ def main():
                     help="skip the variant measurements (nibble container, INT3, per-pixel conv, one-limb weights, probe)")
     ap.add_argument("--passes-per-step", type=int, default=PASSES_PER_STEP,
                     help="passes over the batch that make up one step (profiler captures use 1)")
-    ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep", "gn"],
+    ap.add_argument("--workload", default="step", choices=["step", "unet", "dit", "sweep", "gn", "attn"],
                     help="step: the benchmark step (default); unet: one denoising step of the UNet-shaped network; dit: the "
                          "quantized linears of the DiT-shaped workload; sweep: the M x K x N shape sweep; gn: the "
                          "GroupNorm+SiLU prologue on one tensor")
@@ -910,6 +942,8 @@ def main():
         return main_sweep(args)
     if args.workload == "gn":
         return main_gn(args)
+    if args.workload == "attn":
+        return main_attn(args)
 
     import torch
     import torch.distributed as dist
