@@ -909,6 +909,8 @@ def main():
                          "byte (default, the faster one) or two per byte (half the workspace)")
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
+    ap.add_argument("--pair-gemm", action="store_true",
+                    help="run the short-reduction products on pairs of SMs (tcgen05.mma.cta_group::2; hq_set_pair_gemm)")
     ap.add_argument("--print-csrc-digest", action="store_true", help="print the digest profiles/dram_traffic.json records")
     args = ap.parse_args()
     if args.print_csrc_digest:
@@ -964,6 +966,9 @@ def main():
 
     warmup = max(args.warmup, 3)
     R = max(1, args.passes_per_step)
+    if args.pair_gemm:
+        hq.hq_set_pair_gemm(True)
+        WORKLOAD = WORKLOAD + ", K <= 512 products on SM pairs"
     layers = build_layers(torch, hq, device, seed=rank)
     status = torch.zeros((1,), dtype=torch.int32, device=device)
     stream = torch.cuda.current_stream()

@@ -70,7 +70,9 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
     return a;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    // default (CTA-scope release) semantics: what the arrival orders are this warp's tensor-memory reads, which the
+    // tcgen05 fence in front of it covers; a cluster-scope release here drains the thread's whole memory pipeline
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load whose completion bytes are credited to the barrier at `bar_cluster_addr` (this CTA's or the leader's).
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int x, int y) {
