@@ -264,13 +264,61 @@ __device__ __forceinline__ void store_row16(void* out_row, const uint32_t (&v)[1
 // out in the 64-byte swizzle of the output tensor map); every 32 columns one lane hands the buffer to the copy
 // engine, which clips rows and columns beyond the output, and the warp carries on with the next columns.  Before
 // the buffer is written again the lane waits until the engine has read it.
-template <int LIMBS>
+template <int LIMBS, bool EARLY = false>
 __device__ __forceinline__ void epilogue_fast(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
                                               const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0,
                                               int row0, uint64_t* tempty_bar) {
     constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
     const uint32_t wsw = (lane >> 1) & 3;
     unsigned char* wr = stg + lane * 64;
+    if constexpr (EARLY) {
+        // All of this warp's accumulator columns are requested at once (128 registers) and the accumulator is handed
+        // back to the MMA warp as soon as they have arrived, before any of the arithmetic and stores below.
+        constexpr int NL = LIMBS == 2 ? 2 * NSTEPS : NSTEPS;
+        uint32_t acc[NL][16];
+#pragma unroll
+        for (int st = 0; st < NSTEPS; ++st) {
+            tmem_ld_32x16(t_row + uint32_t(st * 16), acc[st]);
+            if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2 + st * 16), acc[NSTEPS + st]);
+        }
+#pragma unroll
+        for (int l = 0; l < NL; ++l) tmem_ld_wait_16(acc[l]);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar);
+#pragma unroll
+        for (int st = 0; st < NSTEPS; ++st) {
+            int32_t w[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                w[j] = LIMBS == 2 ? int32_t(acc[st][j]) * 256 + int32_t(acc[NSTEPS + st][j]) : int32_t(acc[st][j]);
+            if ((st & 1) == 0) {                           // the copy engine must be done reading the staging buffer
+                if (lane == 0) bulk_wait_read_all();
+                __syncwarp();
+            }
+            const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
+            const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const float4 s0 = sw4[2 * j], s1 = sw4[2 * j + 1], c0 = b4[2 * j], c1 = b4[2 * j + 1];
+                uint4 o;
+                o.x = pack_bf16x2(fmaf(float(w[8 * j + 0]) * s0.x, sa_eff, c0.x), fmaf(float(w[8 * j + 1]) * s0.y, sa_eff, c0.y));
+                o.y = pack_bf16x2(fmaf(float(w[8 * j + 2]) * s0.z, sa_eff, c0.z), fmaf(float(w[8 * j + 3]) * s0.w, sa_eff, c0.w));
+                o.z = pack_bf16x2(fmaf(float(w[8 * j + 4]) * s1.x, sa_eff, c1.x), fmaf(float(w[8 * j + 5]) * s1.y, sa_eff, c1.y));
+                o.w = pack_bf16x2(fmaf(float(w[8 * j + 6]) * s1.z, sa_eff, c1.z), fmaf(float(w[8 * j + 7]) * s1.w, sa_eff, c1.w));
+                *reinterpret_cast<uint4*>(wr + (((2 * (st & 1) + j) ^ wsw) << 4)) = o;
+            }
+            if (st & 1) {
+                fence_proxy_async_smem();                  // the lanes' writes become visible to the copy engine
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(tmY, stg, col0 + (st >> 1) * 32, row0);
+                    bulk_commit_group();
+                }
+            }
+        }
+        return;
+    }
     uint32_t hi[16], lo[16];
     tmem_ld_32x16(t_row, hi);
     if (LIMBS == 2) tmem_ld_32x16(t_row + uint32_t(kBN / 2), lo);
@@ -788,7 +836,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 // rows of the tile are consecutive output rows (checked on the host); this warp owns 32 of them
                 const int row0 = out_row_of<CONV>(p, tc, 0) + q * 32;
                 const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
-                epilogue_fast<LIMBS_T>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
+                epilogue_fast<LIMBS_T, !NIBBLE>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, &ctl->tempty[as]);
                 continue;
             }
 
