@@ -841,7 +841,7 @@ def main_gn(args):
                           higher_is_better=True, dtype="f32", data="synthetic", vs_baseline=None,
                           config=dict(workload=f"GroupNorm(32)+SiLU prologue on {Nb}x{H}x{W}x{Cc} bf16, {codes_name()} codes"),
                           plain_transform_quantize_ms=plain_ms, frac_of_copy_bandwidth=gbytes / gn_ms / 1e6 / pk["hbm_gbs"],
-                          gpu_launches=3 * steps)))
+                          gpu_launches=2 * steps)))
 
 
 def launch_command(n_gpus, argv, port=None):

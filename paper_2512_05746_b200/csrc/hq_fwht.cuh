@@ -19,6 +19,9 @@ __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { f32x2 r; asm("sub.rn.f
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
 __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { f32x2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
 
+// The largest of three values in one instruction.
+__device__ __forceinline__ float max3(float a, float b, float c) { float r; asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c)); return r; }
+
 // Butterflies over pair-index bits: element distance 2*h for h = LO .. HI (pairs stay pairs).
 template <int P, int LO, int HI>
 __device__ __forceinline__ void butterflies_pairs(f32x2 (&v)[P]) {
@@ -48,32 +51,35 @@ __device__ __forceinline__ void butterfly_within_pairs(f32x2 (&v)[P]) {
 __host__ __device__ constexpr int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
 
 // Rounds E values held as pairs (ties to even, optional clamp) and packs them in register order into words: 8
-// four-bit codes or 4 bytes per word.  Each rounded value is kMagicBits + (code + bias); summing the shifted bit
-// patterns and removing the shifted constants leaves the biased fields, which one XOR turns into two's complement.
+// four-bit codes or 4 bytes per word.  Adding kMagic + bias leaves code + bias in the low mantissa bits.  The second
+// value of every pair is rounded F times larger (F = 256 for bytes, 16 for four-bit codes): scaling the multiplier and
+// the magic number by a power of two scales the sum exactly, so the code is the same, and it lands F units up.  Taking
+// the scaled magic number off again (exact) and adding the first value (exact: the sum stays below 2^22 units) leaves
+// both biased codes side by side in the low bits of one float, on the floating-point pipe; byte permutes then gather
+// the fields of a word, and one XOR turns the biased fields into two's complement.
 template <int E, bool INT8_OUT, bool CLAMP>
 __device__ __forceinline__ void round_pack(const f32x2 (&v)[E / 2], float inv, int bits, uint32_t (&out)[INT8_OUT ? E / 4 : E / 8]) {
+    constexpr float F = INT8_OUT ? 256.0f : 16.0f;
     const float bias = INT8_OUT ? 128.0f : 8.0f;
     const float mb = kMagic + bias;
     const float lo = mb + float(-(1 << (bits - 1))), hi = mb + float((1 << (bits - 1)) - 1);
-    const f32x2 inv2 = pk2(inv, inv), mb2 = pk2(mb, mb);
-    constexpr int PER_WORD = INT8_OUT ? 4 : 8;
-    constexpr int SHIFT = INT8_OUT ? 8 : 4;
-    uint32_t cst = 0;
+    const f32x2 inv2 = pk2(inv, F * inv), mb2 = pk2(mb, F * mb);
+    uint32_t u[E / 2];                                 // per pair: kMagicBits + (c0 + bias) + F (c1 + bias)
 #pragma unroll
-    for (int e = 0; e < PER_WORD; ++e) cst += kMagicBits << (SHIFT * e);
-    constexpr uint32_t UNBIAS = INT8_OUT ? 0x80808080u : 0x88888888u;
+    for (int e = 0; e < E / 2; ++e) {
+        float f0, f1;
+        upk2(fma2(v[e], inv2, mb2), f0, f1);
+        if (CLAMP) { f0 = fminf(fmaxf(f0, lo), hi); f1 = fminf(fmaxf(f1, F * lo), F * hi); }
+        u[e] = __float_as_uint(f0 + (f1 - F * kMagic));
+    }
+    if (INT8_OUT) {
 #pragma unroll
-    for (int w = 0; w < E / PER_WORD; ++w) {
-        uint32_t acc = 0;
+        for (int w = 0; w < E / 4; ++w) out[w] = __byte_perm(u[2 * w], u[2 * w + 1], 0x5410) ^ 0x80808080u;
+    } else {
 #pragma unroll
-        for (int e = 0; e < PER_WORD; e += 2) {
-            float f0, f1;
-            upk2(fma2(v[(w * PER_WORD + e) / 2], inv2, mb2), f0, f1);
-            if (CLAMP) { f0 = fminf(fmaxf(f0, lo), hi); f1 = fminf(fmaxf(f1, lo), hi); }
-            acc += __float_as_uint(f0) << (SHIFT * e);
-            acc += __float_as_uint(f1) << (SHIFT * (e + 1));
-        }
-        out[w] = (acc - cst) ^ UNBIAS;
+        for (int w = 0; w < E / 8; ++w)
+            out[w] = __byte_perm(__byte_perm(u[4 * w], u[4 * w + 1], 0x0040), __byte_perm(u[4 * w + 2], u[4 * w + 3], 0x0040),
+                                 0x5410) ^ 0x88888888u;
     }
 }
 

@@ -21,7 +21,14 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
-__device__ __forceinline__ float silu_f(float y) { return y / (1.0f + __expf(-y)); }
+// y * sigmoid(y) with one special-function instruction each for the exponential and the reciprocal (every caller rounds
+// the result to bf16)
+__device__ __forceinline__ float silu_f(float y) {
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(y * -1.4426950408889634f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+    return y * r;
+}
 
 struct F8 { float v[8]; };
 __device__ __forceinline__ F8 unpack8(const uint4 w) {

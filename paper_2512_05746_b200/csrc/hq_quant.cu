@@ -11,14 +11,17 @@
 //   fwht_quant_generic  every other block size, including the identity: one row per CTA in shared memory.
 //   width_quant_kernel  the transform along the width axis of an NHWC tensor (Eq. 13-14 as stated), static scale,
 //                       followed by the integer factor q * H_raw.
-//   gn_stats_kernel / gn_finalize_kernel   per-(sample, group) statistics for the GroupNorm prologue.
+//   gn_stats_kernel     per-(sample, group) mean and 1/sqrt(var + eps) for the GroupNorm prologue, in one launch.
 // The butterflies run unnormalised (H_raw); 2^(-k/2) is folded into the scale (Eq. 7).
+#include <type_traits>
+
 #include "hq_common.cuh"
 #include "hq_fwht.cuh"
 
 namespace hq {
-namespace {
+int sm_count();             // hq_gemm.cu: SM count of the current device
 
+namespace {
 
 struct QuantParams {
     const void* x;
@@ -38,7 +41,9 @@ struct QuantParams {
     const float* gn_beta;    // [cols]
     int gn_groups;
     int gn_silu;             // 1: SiLU after the normalisation, 0: none
-    int64_t gn_rows_per_sample;
+    int gn_sets_per_sample;  // CTAs per sample (a CTA never straddles two samples)
+    int gn_cg;               // channels per group, and its log2 when it is a power of two (else -1)
+    int gn_cg_shift;
     // optional LayerNorm over each row with a per-sample affine, applied before the transform (ln_on != 0)
     int ln_on;
     const float* ln_w;       // [groups][cols] or nullptr (= 1)
@@ -47,15 +52,21 @@ struct QuantParams {
     float ln_eps;
 };
 
-__device__ __forceinline__ float silu(float y) { return __fdividef(y, 1.0f + __expf(-y)); }
+// y * sigmoid(y) = y / (1 + 2^(-y log2 e)) for two values: the exponential and the reciprocal are one special-function
+// instruction each (the flush-to-zero forms: the plain forms are expanded into sequences that rescale subnormal operands,
+// which tripled the instruction count of the prologue); everything else is two-wide.  A large negative y gives
+// 2^(...) = inf, 1 / inf = 0 and y * 0 = -0; a subnormal exponential is flushed to 0 and leaves y.
+__device__ __forceinline__ float ex2_ftz(float x) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float rcp_ftz(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ f32x2 silu2(f32x2 y) {
+    constexpr float kNegLog2e = -1.4426950408889634f;
+    float z0, z1, d0, d1;
+    upk2(mul2(y, pk2(kNegLog2e, kNegLog2e)), z0, z1);
+    upk2(add2(pk2(ex2_ftz(z0), ex2_ftz(z1)), pk2(1.0f, 1.0f)), d0, d1);
+    return mul2(y, pk2(rcp_ftz(d0), rcp_ftz(d1)));
+}
 
 __device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ float4 load4_keep(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ float4 load4_keep(const __nv_bfloat16* p) {
-    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p));
-    return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u), __uint_as_float(raw.y << 16),
-                       __uint_as_float(raw.y & 0xFFFF0000u));
-}
 __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
     uint2 raw = __ldcs(reinterpret_cast<const uint2*>(p));
     float4 f;
@@ -107,27 +118,14 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     const int tr = tid - row_in_cta * p.threads_per_row;
     const int blk = tr / TB;
     const int tb = tr & (TB - 1);
-    const int64_t row = int64_t(blockIdx.x) * p.rows_per_cta + row_in_cta;
-    const bool valid = row < p.rows;
     const bool shared_max = (p.m > 1) || (TB > 32);
 
     if (!STATIC && tid < p.rows_per_cta) rowmax[tid] = 0u;
 
     // GroupNorm + SiLU prologue: per-channel y = x * a[c] + b[c] with a = rstd * gamma, b = beta - mean * a of the
-    // sample this CTA's rows belong to (the host makes sure a CTA never straddles two samples), then y * sigmoid(y).
+    // sample the CTA's rows belong to (the host makes sure a CTA never straddles two samples), then y * sigmoid(y).
     float* gn_a = reinterpret_cast<float*>(rowmax + ((p.rows_per_cta + 3) & ~3));
     float* gn_b = gn_a + p.cols;
-    if (GN) {
-        const int64_t sample = (int64_t(blockIdx.x) * p.rows_per_cta) / p.gn_rows_per_sample;
-        const int cg = int(p.cols) / p.gn_groups;
-        for (int c = tid; c < int(p.cols); c += blockDim.x) {
-            const float2 st = *reinterpret_cast<const float2*>(p.gn_stats + (sample * p.gn_groups + c / cg) * 2);
-            const float a = st.y * __ldg(p.gn_gamma + c);
-            gn_a[c] = a;
-            gn_b[c] = fmaf(-st.x, a, __ldg(p.gn_beta + c));
-        }
-        __syncthreads();
-    }
     // LayerNorm prologue: two sums per row, gathered in shared memory (the affine vectors of the CTA's sample are read
     // from global memory as they are used: a CTA holds only a few rows, a table of its own would cost more than it saves)
     float* lnacc = gn_a;                               // [rows_per_cta][2]
@@ -136,23 +134,52 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
         __syncthreads();
     }
 
-    f32x2 v[P];
+    // The rows' values are requested first, so that the table below is built while they are on their way.
+    using Raw = typename std::conditional<sizeof(InT) == 4, float4, uint2>::type;
+    const int64_t row = int64_t(blockIdx.x) * p.rows_per_cta + row_in_cta;
+    const bool valid = row < p.rows;                   // rows past the end work on row 0's values and store nothing
+    Raw cur[E / 4];
     {
         const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
 #pragma unroll
+        for (int i = 0; i < E / 4; ++i) cur[i] = __ldcs(reinterpret_cast<const Raw*>(src + 4 * (tb + TB * i)));
+    }
+    if (GN) {
+        const unsigned sample = blockIdx.x / unsigned(p.gn_sets_per_sample);
+        const float2* st = reinterpret_cast<const float2*>(p.gn_stats) + size_t(sample) * p.gn_groups;
+        for (int c = 4 * tid; c < int(p.cols); c += 4 * blockDim.x) {      // a channel quad lies in one group
+            const float2 ms = __ldg(st + (p.gn_cg_shift >= 0 ? c >> p.gn_cg_shift : c / p.gn_cg));
+            const float4 gm = __ldg(reinterpret_cast<const float4*>(p.gn_gamma + c));
+            const float4 bt = __ldg(reinterpret_cast<const float4*>(p.gn_beta + c));
+            const float4 a = make_float4(ms.y * gm.x, ms.y * gm.y, ms.y * gm.z, ms.y * gm.w);
+            *reinterpret_cast<float4*>(gn_a + c) = a;
+            *reinterpret_cast<float4*>(gn_b + c) = make_float4(fmaf(-ms.x, a.x, bt.x), fmaf(-ms.x, a.y, bt.y),
+                                                               fmaf(-ms.x, a.z, bt.z), fmaf(-ms.x, a.w, bt.w));
+        }
+        __syncthreads();
+    }
+
+    f32x2 v[P];
+    {
+#pragma unroll
         for (int i = 0; i < E / 4; ++i) {
-            float4 f = load4(src + 4 * (tb + TB * i));
+            float4 f;
+            if constexpr (sizeof(InT) == 4) {
+                f = cur[i];
+            } else {
+                f = make_float4(__uint_as_float(cur[i].x << 16), __uint_as_float(cur[i].x & 0xFFFF0000u),
+                                __uint_as_float(cur[i].y << 16), __uint_as_float(cur[i].y & 0xFFFF0000u));
+            }
+            v[2 * i] = pk2(f.x, f.y);
+            v[2 * i + 1] = pk2(f.z, f.w);
             if (GN) {
                 const int ch = blk * N + 4 * (tb + TB * i);
                 const float4 a4 = *reinterpret_cast<const float4*>(gn_a + ch);
                 const float4 b4 = *reinterpret_cast<const float4*>(gn_b + ch);
-                f.x = fmaf(f.x, a4.x, b4.x); f.y = fmaf(f.y, a4.y, b4.y);
-                f.z = fmaf(f.z, a4.z, b4.z); f.w = fmaf(f.w, a4.w, b4.w);
-                if (GN_SILU) { f.x = silu(f.x); f.y = silu(f.y); f.z = silu(f.z); f.w = silu(f.w); }
+                v[2 * i] = fma2(v[2 * i], pk2(a4.x, a4.y), pk2(b4.x, b4.y));
+                v[2 * i + 1] = fma2(v[2 * i + 1], pk2(a4.z, a4.w), pk2(b4.z, b4.w));
+                if (GN_SILU) { v[2 * i] = silu2(v[2 * i]); v[2 * i + 1] = silu2(v[2 * i + 1]); }
             }
-            if (!valid) f = make_float4(0.f, 0.f, 0.f, 0.f);
-            v[2 * i] = pk2(f.x, f.y);
-            v[2 * i + 1] = pk2(f.z, f.w);
         }
     }
     if (LN) {
@@ -205,7 +232,7 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
         for (int e = 0; e < P; ++e) {
             float a, b;
             upk2(v[e], a, b);
-            amax = fmaxf(fmaxf(amax, fabsf(a)), fabsf(b));
+            amax = max3(amax, fabsf(a), fabsf(b));
         }
 #pragma unroll
         for (int off = 1; off < (TB < 32 ? TB : 32); off <<= 1)
@@ -479,63 +506,146 @@ __global__ void __launch_bounds__(128) width_quant2_kernel(const Width2Params p)
 }
 
 // ---- GroupNorm statistics: sums and sums of squares per (sample, group), then mean and 1/sqrt(var + eps) --------
-// x NHWC; grid (chunks, samples); a thread owns channel quads (coalesced over channels) and walks the pixels of its
-// chunk, accumulating in fp64; per-CTA shared-memory reduction per group, one fp64 atomic pair per group and CTA.
-template <typename InT>
-__global__ void __launch_bounds__(256) gn_stats_kernel(const InT* x, int64_t hw, int C, int groups, int chunks,
-                                                       double* sums) {
-    extern __shared__ double s_acc[];                  // [groups][2]
-    for (int i = threadIdx.x; i < 2 * groups; i += blockDim.x) s_acc[i] = 0.0;
-    __syncthreads();
-    const int nq = C / 4 < 256 ? C / 4 : 256;          // channel quads walked side by side
-    const int ppl = 256 / nq;                          // pixels walked side by side
-    const int qd0 = threadIdx.x % nq, pl = threadIdx.x / nq;
-    const int64_t per = (hw + chunks - 1) / chunks;
-    const int64_t p0 = int64_t(blockIdx.x) * per, p1 = p0 + per < hw ? p0 + per : hw;
-    const int cg = C / groups;
-    const InT* base = x + int64_t(blockIdx.y) * hw * C;
-    if (pl < ppl) {
-        for (int qd = qd0; qd < C / 4; qd += nq) {
-            double s1 = 0.0, s2 = 0.0;
-            int64_t px = p0 + pl;
-            for (; px + 3 * ppl < p1; px += 4 * ppl) {     // four independent loads in flight
-                float4 f[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) f[u] = load4_keep(base + (px + u * ppl) * C + 4 * qd);   // read again by the quantize kernel: keep in L2
-                // sixteen values at a time in fp32 (relative error about 1e-7), then into the fp64 running sums:
-                // the fp32 -> fp64 conversions are the slow instructions here
-                float a1 = 0.f, a2 = 0.f;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    a1 += (f[u].x + f[u].y) + (f[u].z + f[u].w);
-                    a2 = fmaf(f[u].x, f[u].x, fmaf(f[u].y, f[u].y, fmaf(f[u].z, f[u].z, fmaf(f[u].w, f[u].w, a2))));
-                }
-                s1 += double(a1);
-                s2 += double(a2);
-            }
-            for (; px < p1; px += ppl) {
-                const float4 f = load4_keep(base + px * C + 4 * qd);
-                s1 += double(f.x) + double(f.y) + double(f.z) + double(f.w);
-                s2 += double(f.x) * f.x + double(f.y) * f.y + double(f.z) * f.z + double(f.w) * f.w;
-            }
-            const int g = 4 * qd / cg;                 // cg is a multiple of 4 (checked on the host)
-            atomicAdd(&s_acc[2 * g], s1);
-            atomicAdd(&s_acc[2 * g + 1], s2);
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < 2 * groups; i += blockDim.x)
-        atomicAdd(&sums[int64_t(blockIdx.y) * 2 * groups + i], s_acc[i]);
+// x NHWC; one wave of CTAs, each with an equal share of the pixels of all samples, cut into segments where it crosses a
+// sample boundary.  A thread owns one 16-byte (bf16 with VEC = 4: 8-byte) piece of a pixel's
+// channels -- VEC / 4 channel quads, and a quad never straddles two groups -- and walks the pixels of the segment
+// with eight loads in flight; the 32 values a quad collects per round are added two-wide in fp32 and then carried in
+// fp64.  The pixel lanes of the CTA meet in shared memory, one fp64 atomic pair per quad (per piece when it lies in one
+// group) and segment goes to global memory, and the CTA whose segment completes a sample's pixel count turns the
+// sample's sums into the statistics.  The pixel counter is the sample's first statistics word (cleared with the sums by the host,
+// overwritten by the mean at the end).
+template <int VEC>
+struct GnPiece;
+template <>
+struct GnPiece<4> { float4 d; };
+template <>
+struct GnPiece<8> { uint4 d; };
+__device__ __forceinline__ GnPiece<4> gn_load(const float* p, GnPiece<4>*) { return {__ldg(reinterpret_cast<const float4*>(p))}; }
+__device__ __forceinline__ GnPiece<4> gn_load(const __nv_bfloat16* p, GnPiece<4>*) {
+    const uint2 r = __ldg(reinterpret_cast<const uint2*>(p));
+    return {make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u), __uint_as_float(r.y << 16),
+                        __uint_as_float(r.y & 0xFFFF0000u))};
+}
+__device__ __forceinline__ GnPiece<8> gn_load(const __nv_bfloat16* p, GnPiece<8>*) { return {__ldg(reinterpret_cast<const uint4*>(p))}; }
+// The two value pairs of quad q of a piece.
+__device__ __forceinline__ void gn_quad(const GnPiece<4>& r, int, f32x2& lo, f32x2& hi) {
+    lo = pk2(r.d.x, r.d.y);
+    hi = pk2(r.d.z, r.d.w);
+}
+__device__ __forceinline__ void gn_quad(const GnPiece<8>& r, int q, f32x2& lo, f32x2& hi) {
+    const uint32_t w0 = q == 0 ? r.d.x : r.d.z, w1 = q == 0 ? r.d.y : r.d.w;
+    lo = pk2(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xFFFF0000u));
+    hi = pk2(__uint_as_float(w1 << 16), __uint_as_float(w1 & 0xFFFF0000u));
 }
 
-__global__ void gn_finalize_kernel(const double* sums, int64_t count, double eps, int total, float* stats) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const double mean = sums[2 * i] / double(count);
-    double var = sums[2 * i + 1] / double(count) - mean * mean;
-    if (var < 0.0) var = 0.0;
-    stats[2 * i] = float(mean);
-    stats[2 * i + 1] = float(1.0 / sqrt(var + eps));
+template <typename InT, int VEC>
+__global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, int64_t hw, int64_t total_px, int64_t span, int C,
+                                                          int groups, double* sums, float* stats, double inv_count,
+                                                          double eps) {
+    constexpr int Q = VEC / 4;                         // channel quads per piece
+    constexpr int U = 8;                               // loads in flight per thread
+    __shared__ double red[2 * Q][256];
+    __shared__ int s_last;
+    const int tid = threadIdx.x;
+    const int pieces = C / VEC;
+    const int nq = pieces < 256 ? pieces : 256;        // pieces walked side by side
+    const int ppl = 256 / nq;                          // pixels walked side by side
+    const int col0 = tid % nq, pl = tid / nq;
+    const int cg = C / groups;
+    // the CTA's share of the pixels of all samples, cut into segments at the sample boundaries
+    int64_t r0 = int64_t(blockIdx.x) * span;
+    const int64_t r1 = r0 + span < total_px ? r0 + span : total_px;
+    while (r0 < r1) {
+        const int64_t sample = r0 / hw;
+        const int64_t seg_end = (sample + 1) * hw < r1 ? (sample + 1) * hw : r1;
+        double* out = sums + sample * 2 * groups;
+        for (int cbase = 0; cbase < pieces; cbase += nq) {
+            const int col = cbase + col0;
+            double s1[Q], s2[Q];
+#pragma unroll
+            for (int q = 0; q < Q; ++q) { s1[q] = 0.0; s2[q] = 0.0; }
+            if (pl < ppl && col < pieces) {
+                const InT* src = x + int64_t(col) * VEC;
+                int64_t px = r0 + pl;
+                for (; px + (U - 1) * ppl < seg_end; px += U * ppl) {
+                    GnPiece<VEC> raw[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) raw[u] = gn_load(src + (px + u * ppl) * C, static_cast<GnPiece<VEC>*>(nullptr));
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        f32x2 a = pk2(0.f, 0.f), b = pk2(0.f, 0.f);
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            f32x2 lo, hi;
+                            gn_quad(raw[u], q, lo, hi);
+                            a = add2(a, add2(lo, hi));
+                            b = fma2(lo, lo, fma2(hi, hi, b));
+                        }
+                        float a0, a1, b0, b1;
+                        upk2(a, a0, a1);
+                        upk2(b, b0, b1);
+                        s1[q] += double(a0 + a1);
+                        s2[q] += double(b0 + b1);
+                    }
+                }
+                for (; px < seg_end; px += ppl) {
+                    const GnPiece<VEC> raw = gn_load(src + px * C, static_cast<GnPiece<VEC>*>(nullptr));
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        f32x2 lo, hi;
+                        gn_quad(raw, q, lo, hi);
+                        float a0, a1, b0, b1;
+                        upk2(add2(lo, hi), a0, a1);
+                        upk2(fma2(lo, lo, mul2(hi, hi)), b0, b1);
+                        s1[q] += double(a0 + a1);
+                        s2[q] += double(b0 + b1);
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < Q; ++q) { red[2 * q][tid] = s1[q]; red[2 * q + 1][tid] = s2[q]; }
+            __syncthreads();
+            if (pl == 0 && col < pieces) {
+                double t[2 * Q];
+#pragma unroll
+                for (int k = 0; k < 2 * Q; ++k) {
+                    t[k] = 0.0;
+                    for (int j = 0; j < ppl; ++j) t[k] += red[k][j * nq + col0];
+                }
+                const int g0 = col * VEC / cg;
+                const int g1 = (col * VEC + 4 * (Q - 1)) / cg;
+                if (g1 == g0) {
+                    atomicAdd(out + 2 * g0, Q == 2 ? t[0] + t[2 * (Q - 1)] : t[0]);
+                    atomicAdd(out + 2 * g0 + 1, Q == 2 ? t[1] + t[2 * (Q - 1) + 1] : t[1]);
+                } else {
+                    atomicAdd(out + 2 * g0, t[0]);
+                    atomicAdd(out + 2 * g0 + 1, t[1]);
+                    atomicAdd(out + 2 * g1, t[2 * (Q - 1)]);
+                    atomicAdd(out + 2 * g1 + 1, t[2 * (Q - 1) + 1]);
+                }
+                __threadfence();
+            }
+            __syncthreads();
+        }
+        // tickets count pixels: the CTA whose segment completes the sample sees every CTA's sums
+        float* st = stats + sample * 2 * groups;
+        if (tid == 0) {
+            const unsigned int cnt = unsigned(seg_end - r0);
+            s_last = atomicAdd(reinterpret_cast<unsigned int*>(st), cnt) + cnt == unsigned(hw);
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int g = tid; g < groups; g += 256) {
+                const double mean = __ldcg(out + 2 * g) * inv_count;
+                double var = __ldcg(out + 2 * g + 1) * inv_count - mean * mean;
+                if (var < 0.0) var = 0.0;
+                *reinterpret_cast<float2*>(st + 2 * g) = make_float2(float(mean), float(1.0 / sqrt(var + eps)));
+            }
+        }
+        __syncthreads();                               // s_last is written again by the next segment
+        r0 = seg_end;
+    }
 }
 
 template <int KLOG, int E, typename InT>
@@ -621,7 +731,9 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
     p.scales = scales;
     if (gn != nullptr) {
         p.gn_stats = gn->stats; p.gn_gamma = gn->gamma; p.gn_beta = gn->beta; p.gn_groups = gn->groups;
-        p.gn_rows_per_sample = gn->rows_per_sample; p.gn_silu = gn->silu;
+        p.gn_silu = gn->silu;
+        p.gn_cg = int(cols / gn->groups);
+        p.gn_cg_shift = is_pow2(p.gn_cg) ? ilog2(p.gn_cg) : -1;
     }
     if (ln != nullptr) {
         p.ln_on = 1; p.ln_w = ln->w; p.ln_b = ln->b; p.ln_rows_per_group = ln->rows_per_group; p.ln_eps = ln->eps;
@@ -643,7 +755,12 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
         p.threads_per_row = tr;
         p.rows_per_cta = rpc;
         const int threads = rpc * tr;
-        if (gn != nullptr && gn->rows_per_sample % rpc != 0) return HQ_ERR_UNSUPPORTED;   // a CTA must stay in one sample
+        if (gn != nullptr) {
+            if (gn->rows_per_sample % rpc != 0) return HQ_ERR_UNSUPPORTED;               // a CTA must stay in one sample
+            if (gn->rows_per_sample / rpc > 0x7fffffff || cols % 4 != 0) return HQ_ERR_UNSUPPORTED;
+            if (!aligned16(gn->gamma) || !aligned16(gn->beta)) return HQ_ERR_ALIGNMENT;
+            p.gn_sets_per_sample = int(gn->rows_per_sample / rpc);
+        }
         if (ln != nullptr && ln->rows_per_group > 0 && ln->rows_per_group % rpc != 0) return HQ_ERR_UNSUPPORTED;
         if (threads <= 320) {                               // otherwise the generic kernel below takes the row shape
         // exchange buffer: per Hadamard block n/4 float4 slots plus one slot of padding per J (J = E/2 or E/4)
@@ -700,23 +817,30 @@ hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, i
     if (reinterpret_cast<uintptr_t>(x) % (4 * elt) != 0) return HQ_ERR_ALIGNMENT;
     double* sums = static_cast<double*>(scratch);
     float* stats = reinterpret_cast<float*>(sums + size_t(Nb) * groups * 2);
-    HQ_CUDA_OK(cudaMemsetAsync(sums, 0, size_t(Nb) * groups * 2 * sizeof(double), st));
-    // enough CTAs that a thread walks about 16 pixels per channel quad (short dependent chains, many loads in flight)
-    const int64_t ppl = C / 4 < 256 ? 256 / (C / 4) : 1;
-    int64_t chunks = hw / (ppl * 16);
-    if (chunks > 1024) chunks = 1024;
-    if (chunks < 1) chunks = 1;
-    if (Nb > 65535) return HQ_ERR_UNSUPPORTED;
-    const dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(Nb));
-    const size_t smem = size_t(groups) * 2 * sizeof(double);
+    HQ_CUDA_OK(cudaMemsetAsync(scratch, 0, need, st));             // the sums and the ticket counters
+    if (hw > 0x7fffffff) return HQ_ERR_UNSUPPORTED;                // the tickets count pixels in 32 bits
+    // 16-byte pieces (bf16: eight channels) where the shape allows them
+    const bool wide = xdt == HQ_BF16 && C % 8 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
+    const int64_t pieces = C / (wide ? 8 : 4);
+    const int64_t ppl = pieces < 256 ? 256 / pieces : 1;
+    // one wave of CTAs (four per SM) that share the pixels of all samples evenly, in whole rounds of loads; small
+    // tensors get fewer CTAs so that a thread still walks a round of eight pixels
+    const int64_t total_px = Nb * hw;
+    const int64_t round = ppl * 8;
+    int64_t ctas = int64_t(sm_count()) * 4;
+    int64_t span = ((total_px + ctas - 1) / ctas + round - 1) / round * round;
+    ctas = (total_px + span - 1) / span;
+    const double inv_count = 1.0 / (double(hw) * double(C / groups));
+    const unsigned grid = unsigned(ctas);
     if (xdt == HQ_F32)
-        gn_stats_kernel<float><<<grid, 256, smem, st>>>(static_cast<const float*>(x), hw, int(C), groups, int(chunks), sums);
+        gn_stats_kernel<float, 4><<<grid, 256, 0, st>>>(static_cast<const float*>(x), hw, total_px, span, int(C), groups, sums,
+                                                       stats, inv_count, double(eps));
+    else if (wide)
+        gn_stats_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), hw, total_px, span, int(C),
+                                                               groups, sums, stats, inv_count, double(eps));
     else
-        gn_stats_kernel<__nv_bfloat16><<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(x), hw, int(C), groups,
-                                                                 int(chunks), sums);
-    if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
-    const int total = int(Nb * groups);
-    gn_finalize_kernel<<<(total + 127) / 128, 128, 0, st>>>(sums, hw * (C / groups), double(eps), total, stats);
+        gn_stats_kernel<__nv_bfloat16, 4><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), hw, total_px, span, int(C),
+                                                               groups, sums, stats, inv_count, double(eps));
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
     *stats_out = stats;
     return HQ_OK;
