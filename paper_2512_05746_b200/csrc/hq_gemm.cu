@@ -78,30 +78,73 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// A tensor map is a pure function of the arguments it is encoded from (address, extents, pitch, box, swizzle), so the
+// encoded 128 bytes are kept per calling thread in a small direct-mapped table keyed by those arguments: a layer that
+// is called again on the same buffers (every step of a sampler) pays for a lookup and a copy instead of three driver
+// calls, which matters for the few-row layers whose kernels are as short as their host-side set-up.
+struct TmapKey {
+    uint64_t v[8];
+    bool operator==(const TmapKey& o) const {
+        for (int i = 0; i < 8; ++i)
+            if (v[i] != o.v[i]) return false;
+        return true;
+    }
+};
+struct TmapSlot { TmapKey key; CUtensorMap map; bool used; };
+constexpr int kTmapSlots = 512;
+
+template <typename Encode>
+bool cached_tensor_map(CUtensorMap* tm, const TmapKey& key, Encode&& encode) {
+    static thread_local TmapSlot table[kTmapSlots] = {};
+    uint64_t h = 0x9E3779B97F4A7C15ull;
+    for (int i = 0; i < 8; ++i) h = (h ^ key.v[i]) * 0xFF51AFD7ED558CCDull + (h >> 29);
+    TmapSlot& slot = table[(h >> 20) % kTmapSlots];
+    if (slot.used && slot.key == key) {
+        *tm = slot.map;
+        return true;
+    }
+    if (!encode(tm)) return false;
+    slot.key = key;
+    slot.map = *tm;
+    slot.used = true;
+    return true;
+}
+
 bool encode_2d(CUtensorMap* tm, const void* base, uint64_t inner_bytes, uint64_t rows, uint64_t pitch_bytes,
                uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[2] = {inner_bytes, rows};
-    cuuint64_t strides[1] = {pitch_bytes};
-    cuuint32_t box[2] = {box_inner, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const TmapKey key{{1, reinterpret_cast<uint64_t>(base), inner_bytes, rows, pitch_bytes,
+                       (uint64_t(box_inner) << 32) | box_rows, uint64_t(swizzle128), 0}};
+    return cached_tensor_map(tm, key, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {inner_bytes, rows};
+        cuuint64_t strides[1] = {pitch_bytes};
+        cuuint32_t box[2] = {box_inner, box_rows};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 bool encode_4d(CUtensorMap* tm, const void* base, const uint64_t dims_in[4], const uint32_t box_in[4],
                const uint32_t estr_in[4], bool swizzle128) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[4] = {dims_in[0], dims_in[1], dims_in[2], dims_in[3]};
-    cuuint64_t strides[3] = {dims_in[0], dims_in[0] * dims_in[1], dims_in[0] * dims_in[1] * dims_in[2]};
-    cuuint32_t box[4] = {box_in[0], box_in[1], box_in[2], box_in[3]};
-    cuuint32_t estr[4] = {estr_in[0], estr_in[1], estr_in[2], estr_in[3]};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    // boxes and element strides are small numbers: 16 bits each in the key
+    const TmapKey key{{3, reinterpret_cast<uint64_t>(base), dims_in[0], dims_in[1], dims_in[2], dims_in[3],
+                       (uint64_t(box_in[0]) << 48) | (uint64_t(box_in[1]) << 32) | (uint64_t(box_in[2]) << 16) | box_in[3],
+                       (uint64_t(estr_in[0]) << 48) | (uint64_t(estr_in[1]) << 32) | (uint64_t(estr_in[2]) << 16) |
+                           (uint64_t(estr_in[3]) << 1) | uint64_t(swizzle128)}};
+    return cached_tensor_map(tm, key, [&](CUtensorMap* out) {
+        cuuint64_t dims[4] = {dims_in[0], dims_in[1], dims_in[2], dims_in[3]};
+        cuuint64_t strides[3] = {dims_in[0], dims_in[0] * dims_in[1], dims_in[0] * dims_in[1] * dims_in[2]};
+        cuuint32_t box[4] = {box_in[0], box_in[1], box_in[2], box_in[3]};
+        cuuint32_t estr[4] = {estr_in[0], estr_in[1], estr_in[2], estr_in[3]};
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Output tensor map for the epilogue's bulk stores: bf16 [rows][N] with pitch ldy, boxes of 32 rows x 32 columns
@@ -109,13 +152,16 @@ bool encode_4d(CUtensorMap* tm, const void* base, const uint64_t dims_in[4], con
 bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[2] = {N, rows};
-    cuuint64_t strides[1] = {ldy * 2};
-    cuuint32_t box[2] = {32, 32};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(y), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const TmapKey key{{2, reinterpret_cast<uint64_t>(y), N, rows, ldy, 0, 0, 0}};
+    return cached_tensor_map(tm, key, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {N, rows};
+        cuuint64_t strides[1] = {ldy * 2};
+        cuuint32_t box[2] = {32, 32};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(y), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 int sm_count() {
