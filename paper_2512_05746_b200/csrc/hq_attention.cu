@@ -11,14 +11,22 @@
 // and finally O / sum goes out as bf16.  Operands are staged by plain 16-byte loads into the unswizzled canonical
 // layout of the tensor core (8 x 16-byte core matrices).  Several CTAs are resident per SM and overlap one another's
 // load, tensor and softmax phases; every wait is bounded.
+#include <cuda.h>
+
 #include "hq_common.cuh"
+#include "hq_fwht.cuh"
 
 namespace hq {
+// hq_gemm.cu: bf16 [rows][cols] with a row pitch, boxes of box_rows x 64 columns in the 128-byte swizzle
+bool encode_2d_bf16_sw128(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
+                          uint32_t box_rows);
+
 namespace {
 
 constexpr int kQTile = 128;      // queries per CTA (tensor-memory lanes)
-constexpr int kKeyBlock = 128;   // keys per step
-constexpr int kAttnTmemCols = 256;
+constexpr int kKeyBlock = 64;    // keys per step: S (64 columns) and O (dh columns) fit 128 columns of tensor memory up to
+                                 // dh = 64, and a CTA's tiles 48 KB of shared memory, so that four CTAs share an SM
+__host__ __device__ constexpr int attn_tmem_cols(int dh) { return kKeyBlock + dh <= 128 ? 128 : 256; }
 constexpr int32_t kStatusAttnWait = 0x600;
 
 struct AttnParams {
@@ -81,10 +89,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // core-matrix layout: the 16-byte piece (row, v) lands at (row / 8) * group_stride + v * 128 + (row % 8) * 16.  Rows beyond
 // rows_valid are zero.  Consecutive lanes take consecutive rows of a group, so the shared-memory stores of a warp fall
 // into four 128-byte runs.
-template <int DH>
-__device__ __forceinline__ void fetch_tile(uint4 (&reg)[DH / 8], const __nv_bfloat16* src, int64_t pitch, int rows_valid, int tid) {
+template <int DH, int ROWS>
+__device__ __forceinline__ void fetch_tile(uint4 (&reg)[ROWS * DH / 1024], const __nv_bfloat16* src, int64_t pitch, int rows_valid,
+                                           int tid) {
+    static_assert((ROWS * DH / 8) % 128 == 0, "the tile's 16-byte pieces are dealt to 128 threads");
 #pragma unroll
-    for (int i = 0; i < DH / 8; ++i) {
+    for (int i = 0; i < ROWS * DH / 1024; ++i) {
         const int f = tid + 128 * i;
         const int rg = f / DH, within = f - rg * DH;
         const int row = rg * 8 + (within & 7), v = within >> 3;
@@ -92,32 +102,34 @@ __device__ __forceinline__ void fetch_tile(uint4 (&reg)[DH / 8], const __nv_bflo
         if (row < rows_valid) reg[i] = __ldg(reinterpret_cast<const uint4*>(src + int64_t(row) * pitch + v * 8));
     }
 }
-template <int DH>
-__device__ __forceinline__ void put_tile(unsigned char* dst, const uint4 (&reg)[DH / 8], int tid) {
+template <int DH, int ROWS>
+__device__ __forceinline__ void put_tile(unsigned char* dst, const uint4 (&reg)[ROWS * DH / 1024], int tid) {
     constexpr int group_stride = (DH / 8) * 128;
 #pragma unroll
-    for (int i = 0; i < DH / 8; ++i) {
+    for (int i = 0; i < ROWS * DH / 1024; ++i) {
         const int f = tid + 128 * i;
         const int rg = f / DH, within = f - rg * DH;
         *reinterpret_cast<uint4*>(dst + rg * group_stride + (within >> 3) * 128 + (within & 7) * 16) = reg[i];
     }
 }
-template <int DH>
+template <int DH, int ROWS>
 __device__ __forceinline__ void stage_tile(unsigned char* dst, const __nv_bfloat16* src, int64_t pitch, int rows_valid,
                                            int tid) {
-    uint4 reg[DH / 8];
-    fetch_tile<DH>(reg, src, pitch, rows_valid, tid);
-    put_tile<DH>(dst, reg, tid);
+    uint4 reg[ROWS * DH / 1024];
+    fetch_tile<DH, ROWS>(reg, src, pitch, rows_valid, tid);
+    put_tile<DH, ROWS>(dst, reg, tid);
 }
 
 template <int DH>
-__global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(128, (DH <= 64 ? 4 : 2)) attention_kernel(const AttnParams p) {
     extern __shared__ __align__(128) unsigned char smem_attn[];
-    constexpr int kTileBytes = kQTile * DH * 2;
+    constexpr int KB = kKeyBlock;
+    constexpr int kQBytes = kQTile * DH * 2, kKVBytes = KB * DH * 2;
+    constexpr int kTmemCols = attn_tmem_cols(DH);
     unsigned char* sQ = smem_attn;
-    unsigned char* sK = sQ + kTileBytes;
-    unsigned char* sV = sK + kTileBytes;
-    unsigned char* sP = sV + kTileBytes;                       // 128 x 128 bf16
+    unsigned char* sK = sQ + kQBytes;
+    unsigned char* sV = sK + kKVBytes;
+    unsigned char* sP = sV + kKVBytes;                         // 128 x KB bf16
     __shared__ uint64_t bar;
     __shared__ uint32_t tmem_slot;
 
@@ -129,48 +141,42 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
 
     if (tid == 0) { mbar_init(&bar, 1); fence_barrier_init(); }
     // the allocation is a warp-wide (.sync.aligned) instruction: it runs in a warp none of whose lanes took another path
-    if (warp == 1) { __syncwarp(); tmem_alloc(&tmem_slot, kAttnTmemCols); tmem_relinquish(); }
-    stage_tile<DH>(sQ, base + int64_t(q0) * pitch, pitch, L - q0 < kQTile ? L - q0 : kQTile, tid);
+    if (warp == 1) { __syncwarp(); tmem_alloc(&tmem_slot, kTmemCols); tmem_relinquish(); }
+    stage_tile<DH, kQTile>(sQ, base + int64_t(q0) * pitch, pitch, L - q0 < kQTile ? L - q0 : kQTile, tid);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
-    const uint32_t t_s = tmem_base + (uint32_t(warp * 32) << 16);          // this warp's lanes, S at columns 0..127
-    const uint32_t t_o = t_s + uint32_t(kKeyBlock);                        // O at columns 128..128+DH
+    const uint32_t t_s = tmem_base + (uint32_t(warp * 32) << 16);          // this warp's lanes, S at columns 0..KB-1
+    const uint32_t t_o = t_s + uint32_t(KB);                               // O at columns KB..KB+DH-1
 
     constexpr uint32_t kGroup = (DH / 8) * 128;                            // bytes of one 8-row group of a DH-wide tile
-    const uint32_t idesc_s = make_idesc_bf16(kQTile, kKeyBlock, false);
+    constexpr uint32_t kPGroup = (KB / 8) * 128;                           // bytes of one 8-row group of P
+    const uint32_t idesc_s = make_idesc_bf16(kQTile, KB, false);
     const uint32_t idesc_o = make_idesc_bf16(kQTile, DH, true);
 
     float m_run = -INFINITY, l_run = 0.f;
     uint32_t phase = 0;
     bool ok = true;
-    const int nblocks = (L + kKeyBlock - 1) / kKeyBlock;
-    // The next key block's K and V pieces are requested into registers while the current block's softmax runs (head
-    // widths up to 64: 16 registers per operand), so that their latency is not on the block's critical path.
-    constexpr bool PREFETCH = DH <= 64;
-    uint4 kreg[DH / 8], vreg[DH / 8];
-    if (PREFETCH) {
-        fetch_tile<DH>(kreg, base + C, pitch, L < kKeyBlock ? L : kKeyBlock, tid);
-        fetch_tile<DH>(vreg, base + 2 * C, pitch, L < kKeyBlock ? L : kKeyBlock, tid);
-    }
+    const int nblocks = (L + KB - 1) / KB;
+    // The next key block's K and V pieces are requested into registers while the current block's softmax runs, so that
+    // their latency is not on the block's critical path.
+    constexpr int NR = KB * DH / 1024;
+    uint4 kreg[NR], vreg[NR];
+    fetch_tile<DH, KB>(kreg, base + C, pitch, L < KB ? L : KB, tid);
+    fetch_tile<DH, KB>(vreg, base + 2 * C, pitch, L < KB ? L : KB, tid);
     for (int j = 0; j < nblocks && ok; ++j) {
-        const int k0 = j * kKeyBlock;
-        const int kvalid = L - k0 < kKeyBlock ? L - k0 : kKeyBlock;
-        if (PREFETCH) {
-            put_tile<DH>(sK, kreg, tid);
-            put_tile<DH>(sV, vreg, tid);
-        } else {
-            stage_tile<DH>(sK, base + C + int64_t(k0) * pitch, pitch, kvalid, tid);
-            stage_tile<DH>(sV, base + 2 * C + int64_t(k0) * pitch, pitch, kvalid, tid);
-        }
+        const int k0 = j * KB;
+        const int kvalid = L - k0 < KB ? L - k0 : KB;
+        put_tile<DH, KB>(sK, kreg, tid);
+        put_tile<DH, KB>(sV, vreg, tid);
         fence_proxy_async_smem();
         __syncthreads();
-        if (PREFETCH && j + 1 < nblocks) {
-            const int k1 = k0 + kKeyBlock;
-            const int kv1 = L - k1 < kKeyBlock ? L - k1 : kKeyBlock;
-            fetch_tile<DH>(kreg, base + C + int64_t(k1) * pitch, pitch, kv1, tid);
-            fetch_tile<DH>(vreg, base + 2 * C + int64_t(k1) * pitch, pitch, kv1, tid);
+        if (j + 1 < nblocks) {
+            const int k1 = k0 + KB;
+            const int kv1 = L - k1 < KB ? L - k1 : KB;
+            fetch_tile<DH, KB>(kreg, base + C + int64_t(k1) * pitch, pitch, kv1, tid);
+            fetch_tile<DH, KB>(vreg, base + 2 * C + int64_t(k1) * pitch, pitch, kv1, tid);
         }
         // One lane issues; its warp-mates wait for it at the warp barrier instead of polling beside it (a polling loop
         // on the other side of a divergent branch can keep the issuing lane from being scheduled).
@@ -193,60 +199,44 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
         if (!ok) break;
         tc_fence_after();
 
-        // ---- row maximum of this block (the next 32 columns are requested while the current ones are reduced)
-        const bool full = kvalid == kKeyBlock;
-        float mx = -INFINITY;
-        {
-            uint32_t ra[32], rb[32];
-            tmem_ld_32x32(t_s, ra);
+        // ---- the row's KB scores come into registers once: maximum, then P = exp2(c (S - m)), the row sum, and P as bf16
+        // into shared memory (K-major: KB / 8 key groups of 128 bytes per row group)
+        const bool full = kvalid == KB;
+        uint32_t sreg[KB];
 #pragma unroll
-            for (int c = 0; c < kKeyBlock / 32; ++c) {
-                uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-                uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
-                tmem_ld_wait_32(cur);
-                if (c + 1 < kKeyBlock / 32) tmem_ld_32x32(t_s + uint32_t((c + 1) * 32), nxt);
-                if (full) {
+        for (int c = 0; c < KB / 32; ++c) tmem_ld_32x32(t_s + uint32_t(c * 32), *reinterpret_cast<uint32_t (*)[32]>(&sreg[32 * c]));
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(cur[e]));
-                } else {
+        for (int c = 0; c < KB / 32; ++c) tmem_ld_wait_32(*reinterpret_cast<uint32_t (*)[32]>(&sreg[32 * c]));
+        if (!full) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (c * 32 + e < kvalid) mx = fmaxf(mx, __uint_as_float(cur[e]));
-                }
-            }
+            for (int e = 0; e < KB; ++e)
+                if (e >= kvalid) sreg[e] = 0xFF800000u;                   // -inf: no part in the maximum, weight 0
         }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < KB; e += 2) mx = max3(mx, __uint_as_float(sreg[e]), __uint_as_float(sreg[e + 1]));
         const float m_new = fmaxf(m_run, mx);
         const float mc = m_new * p.scale_log2;
         const float alpha = ex2(m_run * p.scale_log2 - mc);              // 0 on the first block (m_run = -inf)
-        // ---- P = exp2(c (S - m)), row sum, bf16 into shared memory (K-major: 16 key groups of 128 bytes per row group)
-        float sum = 0.f;
-        unsigned char* prow = sP + (tid >> 3) * 2048 + (tid & 7) * 16;
-        {
-            uint32_t ra[32], rb[32];
-            tmem_ld_32x32(t_s, ra);
+        f32x2 sum2 = pk2(0.f, 0.f);
+        const f32x2 sc2 = pk2(p.scale_log2, p.scale_log2), nmc2 = pk2(-mc, -mc);
+        unsigned char* prow = sP + (tid >> 3) * kPGroup + (tid & 7) * 16;
 #pragma unroll
-            for (int c = 0; c < kKeyBlock / 32; ++c) {
-                uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-                uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
-                tmem_ld_wait_32(cur);
-                if (c + 1 < kKeyBlock / 32) tmem_ld_32x32(t_s + uint32_t((c + 1) * 32), nxt);
-                float pv[32];
+        for (int g = 0; g < KB / 8; ++g) {
+            uint32_t w[4];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float v = ex2(fmaf(__uint_as_float(cur[e]), p.scale_log2, -mc));
-                    pv[e] = (full || c * 32 + e < kvalid) ? v : 0.f;
-                    sum += pv[e];
-                }
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    uint4 w;
-                    w.x = pack_bf16(pv[8 * g + 0], pv[8 * g + 1]); w.y = pack_bf16(pv[8 * g + 2], pv[8 * g + 3]);
-                    w.z = pack_bf16(pv[8 * g + 4], pv[8 * g + 5]); w.w = pack_bf16(pv[8 * g + 6], pv[8 * g + 7]);
-                    *reinterpret_cast<uint4*>(prow + (c * 4 + g) * 128) = w;
-                }
+            for (int h = 0; h < 4; ++h) {
+                float z0, z1;
+                upk2(fma2(pk2(__uint_as_float(sreg[8 * g + 2 * h]), __uint_as_float(sreg[8 * g + 2 * h + 1])), sc2, nmc2), z0, z1);
+                const float p0 = ex2(z0), p1 = ex2(z1);
+                sum2 = add2(sum2, pk2(p0, p1));
+                w[h] = pack_bf16(p0, p1);
             }
+            *reinterpret_cast<uint4*>(prow + g * 128) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        l_run = fmaf(l_run, alpha, sum);
+        float sum_lo, sum_hi;
+        upk2(sum2, sum_lo, sum_hi);
+        l_run = fmaf(l_run, alpha, sum_lo + sum_hi);
         m_run = m_new;
         // ---- the output accumulator follows the running maximum (skipped when no row of the warp moved)
         if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
@@ -267,12 +257,12 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
         if (warp == 0) {
             if (tid == 0) {
                 tc_fence_after();
-                // P: K-major, row groups 2048 bytes apart.  V: MN-major, key groups kGroup apart (lbo), dh groups 128 (sbo).
-                const uint64_t a = make_desc_noswizzle(smem_u32(sP), 128, 2048);
+                // P: K-major, row groups kPGroup bytes apart.  V: MN-major, key groups kGroup apart (lbo), dh groups 128 (sbo).
+                const uint64_t a = make_desc_noswizzle(smem_u32(sP), 128, kPGroup);
                 const uint64_t b = make_desc_noswizzle(smem_u32(sV), kGroup, 128);
 #pragma unroll
-                for (int k = 0; k < kKeyBlock / 16; ++k)
-                    mma_bf16(tmem_base + uint32_t(kKeyBlock), a + uint64_t(k * 16), b + uint64_t(k * 2 * (kGroup >> 4)), idesc_o,
+                for (int k = 0; k < KB / 16; ++k)
+                    mma_bf16(tmem_base + uint32_t(KB), a + uint64_t(k * 16), b + uint64_t(k * 2 * (kGroup >> 4)), idesc_o,
                              (j | k) != 0 ? 1u : 0u);
                 mma_commit(&bar);
             }
@@ -312,12 +302,259 @@ __global__ void __launch_bounds__(128) attention_kernel(const AttnParams p) {
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, kAttnTmemCols);
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ---- head widths of 64 and 128: operands by TMA -----------------------------------------------------------------
+// Q, K and V tiles come in by bulk tensor loads in the 128-byte swizzle (rows of 64 head channels = 128 bytes; a width
+// of 128 takes two such column halves per tile), issued by one thread as soon as the MMAs that read the buffer have
+// completed: the next K block lands during the softmax, the next V block during the next S product, no registers or
+// shared-memory stores are spent on staging, and a CTA needs 48 KB of shared memory and 128 columns of tensor memory at
+// width 64, so that four share an SM.  Q and K are K-major operands (8-row groups 1024 bytes apart); V is read as an
+// MN-major operand (8-key groups 1024 bytes apart, the two 64-channel halves one tile apart).
+// The running maximum of a row moves only when a block's maximum exceeds it by more than 2^8 in the exponent: the
+// weights then stay below 2^8 (exact in bf16's range), the normalisation by the row sum at the end is unchanged, and
+// the read-modify-write of the output accumulator in tensor memory is almost never needed after the first block.
+constexpr int32_t kStatusAttnTma = 0x601;
+
+__device__ __forceinline__ uint64_t make_sw128_mnmajor_desc(uint32_t smem_addr, uint32_t atom_stride_bytes) {
+    uint64_t d = 0;
+    d |= uint64_t((smem_addr & 0x3FFFFu) >> 4);
+    d |= uint64_t((atom_stride_bytes >> 4) & 0x3FFFu) << 16;   // between 64-element groups along N
+    d |= uint64_t(1024 >> 4) << 32;                            // between 8-row groups along K
+    d |= uint64_t(1) << 46;
+    d |= uint64_t(2) << 61;
+    return d;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(128, (DH <= 64 ? 4 : 2))
+attention_tma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const AttnParams p) {
+    extern __shared__ __align__(1024) unsigned char smem_attn_tma[];
+    constexpr int KB = kKeyBlock, NH = DH / 64;                // column halves per tile
+    constexpr int kQHalf = kQTile * 128, kKVHalf = KB * 128;   // bytes of one 64-channel half of a tile
+    constexpr int kTmemCols = attn_tmem_cols(DH);
+    unsigned char* sQ = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_attn_tma) + 1023) & ~uintptr_t(1023));
+    unsigned char* sK = sQ + NH * kQHalf;
+    unsigned char* sV = sK + NH * kKVHalf;
+    unsigned char* sP = sV + NH * kKVHalf;                     // 128 x KB bf16, unswizzled core matrices
+    __shared__ uint64_t bar_mma, bar_q, bar_k, bar_v;
+    __shared__ uint32_t tmem_slot;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int q0 = blockIdx.x * kQTile, head = blockIdx.y, n = blockIdx.z;
+    const int L = p.L, C = p.C;
+    const int row0 = n * L;                                    // the sample's first row of the [Nb L][3 C] matrix
+    const int nblocks = (L + KB - 1) / KB;
+
+    if (tid == 0) {
+        mbar_init(&bar_mma, 1); mbar_init(&bar_q, 1); mbar_init(&bar_k, 1); mbar_init(&bar_v, 1);
+        fence_barrier_init();
+        tma_prefetch_desc(&tmQ);
+        tma_prefetch_desc(&tmKV);
+    }
+    if (warp == 1) { __syncwarp(); tmem_alloc(&tmem_slot, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    bool q_flying = false, k_flying = false, v_flying = false;  // thread 0: a load into the buffer is outstanding
+    uint32_t k_par = 0, v_par = 0;                              // ... and the barrier phase it completes
+    if (tid == 0) {
+        mbar_expect_tx(&bar_q, NH * kQHalf);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) tma_load_2d(sQ + h * kQHalf, &tmQ, &bar_q, head * DH + 64 * h, row0 + q0);
+        mbar_expect_tx(&bar_k, NH * kKVHalf);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) tma_load_2d(sK + h * kKVHalf, &tmKV, &bar_k, C + head * DH + 64 * h, row0);
+        mbar_expect_tx(&bar_v, NH * kKVHalf);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) tma_load_2d(sV + h * kKVHalf, &tmKV, &bar_v, 2 * C + head * DH + 64 * h, row0);
+        q_flying = k_flying = v_flying = true;
+    }
+    const uint32_t tmem_base = tmem_slot;
+    const uint32_t t_s = tmem_base + (uint32_t(warp * 32) << 16);
+    const uint32_t t_o = t_s + uint32_t(KB);
+    constexpr uint32_t kPGroup = (KB / 8) * 128;
+    const uint32_t idesc_s = make_idesc_bf16(kQTile, KB, false);
+    const uint32_t idesc_o = make_idesc_bf16(kQTile, DH, true);
+
+    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t ph_mma = 0, ph_kv = 0;
+    bool ok = true;
+    for (int j = 0; j < nblocks && ok; ++j) {
+        const int k0 = j * KB;
+        const int kvalid = L - k0 < KB ? L - k0 : KB;
+        // ---- S = Q K^T
+        if (warp == 0) {
+            if (tid == 0) {
+                bool ready = j > 0 || mbar_wait(&bar_q, 0, p.dev_status, kStatusAttnTma);
+                if (ready) q_flying = false;
+                ready = ready && mbar_wait(&bar_k, ph_kv, p.dev_status, kStatusAttnTma);
+                if (ready) {
+                    k_flying = false;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < DH / 16; ++k) {
+                        const uint64_t a = make_sw128_kmajor_desc(smem_u32(sQ + (k / 4) * kQHalf)) + uint64_t(2 * (k & 3));
+                        const uint64_t b = make_sw128_kmajor_desc(smem_u32(sK + (k / 4) * kKVHalf)) + uint64_t(2 * (k & 3));
+                        mma_bf16(tmem_base, a, b, idesc_s, k != 0 ? 1u : 0u);
+                    }
+                    mma_commit(&bar_mma);
+                }
+            }
+            __syncwarp();
+        }
+        ok = mbar_wait(&bar_mma, ph_mma, p.dev_status, kStatusAttnWait);
+        ph_mma ^= 1;
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        tc_fence_after();
+        if (tid == 0 && j + 1 < nblocks) {                     // the K buffer is free: the next block's keys
+            mbar_expect_tx(&bar_k, NH * kKVHalf);
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+                tma_load_2d(sK + h * kKVHalf, &tmKV, &bar_k, C + head * DH + 64 * h, row0 + k0 + KB);
+            k_flying = true;
+            k_par = uint32_t(j + 1) & 1u;
+        }
+        // ---- the row's KB scores come into registers once: maximum, P = exp2(c (S - m)), row sum, P as bf16 to smem
+        const bool full = kvalid == KB;
+        uint32_t sreg[KB];
+#pragma unroll
+        for (int c = 0; c < KB / 32; ++c) tmem_ld_32x32(t_s + uint32_t(c * 32), *reinterpret_cast<uint32_t (*)[32]>(&sreg[32 * c]));
+#pragma unroll
+        for (int c = 0; c < KB / 32; ++c) tmem_ld_wait_32(*reinterpret_cast<uint32_t (*)[32]>(&sreg[32 * c]));
+        if (!full) {
+#pragma unroll
+            for (int e = 0; e < KB; ++e)
+                if (e >= kvalid) sreg[e] = 0xFF800000u;                   // -inf: no part in the maximum, weight 0
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < KB; e += 2) mx = max3(mx, __uint_as_float(sreg[e]), __uint_as_float(sreg[e + 1]));
+        const float m_new = (mx - m_run) * p.scale_log2 > 8.0f ? mx : m_run;     // first block: inf > 8
+        const float mc = m_new * p.scale_log2;
+        const float alpha = ex2(m_run * p.scale_log2 - mc);              // 1 when the maximum stays, 0 on the first block
+        f32x2 sum2 = pk2(0.f, 0.f);
+        const f32x2 sc2 = pk2(p.scale_log2, p.scale_log2), nmc2 = pk2(-mc, -mc);
+        unsigned char* prow = sP + (tid >> 3) * kPGroup + (tid & 7) * 16;
+#pragma unroll
+        for (int g = 0; g < KB / 8; ++g) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                float z0, z1;
+                upk2(fma2(pk2(__uint_as_float(sreg[8 * g + 2 * h]), __uint_as_float(sreg[8 * g + 2 * h + 1])), sc2, nmc2), z0, z1);
+                const float p0 = ex2(z0), p1 = ex2(z1);
+                sum2 = add2(sum2, pk2(p0, p1));
+                w[h] = pack_bf16(p0, p1);
+            }
+            *reinterpret_cast<uint4*>(prow + g * 128) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        float sum_lo, sum_hi;
+        upk2(sum2, sum_lo, sum_hi);
+        l_run = fmaf(l_run, alpha, sum_lo + sum_hi);
+        m_run = m_new;
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+#pragma unroll
+            for (int c = 0; c < DH / 16; ++c) {
+                uint32_t r[16];
+                tmem_ld_32x16(t_o + uint32_t(c * 16), r);
+                tmem_ld_wait_16(r);
+#pragma unroll
+                for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                tmem_st_32x16(t_o + uint32_t(c * 16), r);
+            }
+            tmem_st_wait();
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        // ---- O += P V
+        if (warp == 0) {
+            if (tid == 0) {
+                if (mbar_wait(&bar_v, ph_kv, p.dev_status, kStatusAttnTma)) {
+                    v_flying = false;
+                    tc_fence_after();
+                    const uint64_t a = make_desc_noswizzle(smem_u32(sP), 128, kPGroup);
+                    const uint64_t b = make_sw128_mnmajor_desc(smem_u32(sV), kKVHalf);
+#pragma unroll
+                    for (int k = 0; k < KB / 16; ++k)        // 16 keys on: two core-matrix columns of P, 16 rows of V
+                        mma_bf16(tmem_base + uint32_t(KB), a + uint64_t(k * 16), b + uint64_t(k * 128), idesc_o,
+                                 (j | k) != 0 ? 1u : 0u);
+                    mma_commit(&bar_mma);
+                }
+            }
+            __syncwarp();
+        }
+        ph_kv ^= 1;
+        ok = mbar_wait(&bar_mma, ph_mma, p.dev_status, kStatusAttnWait);
+        ph_mma ^= 1;
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        tc_fence_after();
+        if (tid == 0 && j + 1 < nblocks) {                     // the V buffer is free: the next block's values
+            mbar_expect_tx(&bar_v, NH * kKVHalf);
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+                tma_load_2d(sV + h * kKVHalf, &tmKV, &bar_v, 2 * C + head * DH + 64 * h, row0 + k0 + KB);
+            v_flying = true;
+            v_par = uint32_t(j + 1) & 1u;
+        }
+    }
+    if (!ok && tid == 0) {
+        // a wait ran out: the loads still on their way must land before the CTA's shared memory is given up
+        if (q_flying) mbar_wait(&bar_q, 0, nullptr, 0);
+        if (k_flying) mbar_wait(&bar_k, k_par, nullptr, 0);
+        if (v_flying) mbar_wait(&bar_v, v_par, nullptr, 0);
+    }
+
+    if (ok) {
+        const bool row_ok = q0 + tid < L;
+        const float inv = 1.0f / l_run;
+        __nv_bfloat16* dst = p.out + (int64_t(n) * L + (row_ok ? q0 + tid : 0)) * C + head * DH;
+#pragma unroll
+        for (int c = 0; c < DH / 16; ++c) {
+            uint32_t r[16];
+            tmem_ld_32x16(t_o + uint32_t(c * 16), r);
+            tmem_ld_wait_16(r);
+            uint4 w0, w1;
+            w0.x = pack_bf16(__uint_as_float(r[0]) * inv, __uint_as_float(r[1]) * inv);
+            w0.y = pack_bf16(__uint_as_float(r[2]) * inv, __uint_as_float(r[3]) * inv);
+            w0.z = pack_bf16(__uint_as_float(r[4]) * inv, __uint_as_float(r[5]) * inv);
+            w0.w = pack_bf16(__uint_as_float(r[6]) * inv, __uint_as_float(r[7]) * inv);
+            w1.x = pack_bf16(__uint_as_float(r[8]) * inv, __uint_as_float(r[9]) * inv);
+            w1.y = pack_bf16(__uint_as_float(r[10]) * inv, __uint_as_float(r[11]) * inv);
+            w1.z = pack_bf16(__uint_as_float(r[12]) * inv, __uint_as_float(r[13]) * inv);
+            w1.w = pack_bf16(__uint_as_float(r[14]) * inv, __uint_as_float(r[15]) * inv);
+            if (row_ok) {
+                reinterpret_cast<uint4*>(dst + c * 16)[0] = w0;
+                reinterpret_cast<uint4*>(dst + c * 16)[1] = w1;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+template <int DH>
+hq_status launch_attention_tma(const AttnParams& p, int Nb, cudaStream_t st) {
+    CUtensorMap tmQ, tmKV;
+    const uint64_t rows = uint64_t(Nb) * p.L, cols = 3 * uint64_t(p.C);
+    if (!encode_2d_bf16_sw128(&tmQ, p.qkv, cols, rows, cols * 2, kQTile)) return HQ_ERR_CUDA;
+    if (!encode_2d_bf16_sw128(&tmKV, p.qkv, cols, rows, cols * 2, kKeyBlock)) return HQ_ERR_CUDA;
+    const size_t smem = size_t(DH / 64) * (kQTile + 2 * kKeyBlock) * 128 + size_t(kQTile) * kKeyBlock * 2 + 1024;
+    if (cudaFuncSetAttribute(attention_tma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+        return HQ_ERR_CUDA;
+    const dim3 grid(unsigned((p.L + kQTile - 1) / kQTile), unsigned(p.heads), unsigned(Nb));
+    attention_tma_kernel<DH><<<grid, 128, smem, st>>>(tmQ, tmKV, p);
+    return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
 template <int DH>
 cudaError_t launch_attention(const AttnParams& p, int Nb, cudaStream_t st) {
-    const size_t smem = size_t(3) * kQTile * DH * 2 + size_t(kQTile) * kKeyBlock * 2 + 128;
+    const size_t smem = size_t(kQTile + 2 * kKeyBlock) * DH * 2 + size_t(kQTile) * kKeyBlock * 2 + 128;
     cudaError_t e = cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
     const dim3 grid(unsigned((p.L + kQTile - 1) / kQTile), unsigned(p.heads), unsigned(Nb));
@@ -335,7 +572,7 @@ extern "C" hq_status hq_attention(const void* qkv, int64_t Nb, int64_t L, int64_
     if (Nb == 0) return HQ_OK;
     if (qkv == nullptr || out == nullptr) return HQ_ERR_INVALID_ARG;
     if (!aligned16(qkv) || !aligned16(out) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
-    if (Nb > 65535 || heads > 65535 || L > (1 << 24)) return HQ_ERR_UNSUPPORTED;
+    if (Nb > 65535 || heads > 65535 || L > (1 << 24) || Nb * L > 0x7fffffff) return HQ_ERR_UNSUPPORTED;
     const int dh = int(C / heads);
     AttnParams p{};
     p.qkv = static_cast<const __nv_bfloat16*>(qkv);
@@ -348,9 +585,9 @@ extern "C" hq_status hq_attention(const void* qkv, int64_t Nb, int64_t L, int64_
     switch (dh) {
         case 32: e = launch_attention<32>(p, int(Nb), st); break;
         case 48: e = launch_attention<48>(p, int(Nb), st); break;
-        case 64: e = launch_attention<64>(p, int(Nb), st); break;
+        case 64: return launch_attention_tma<64>(p, int(Nb), st);
         case 96: e = launch_attention<96>(p, int(Nb), st); break;
-        case 128: e = launch_attention<128>(p, int(Nb), st); break;
+        case 128: return launch_attention_tma<128>(p, int(Nb), st);
         default: return HQ_ERR_UNSUPPORTED;      // head widths the tensor-core tile shapes here cover: 32, 48, 64, 96, 128
     }
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;

@@ -147,6 +147,24 @@ bool encode_4d(CUtensorMap* tm, const void* base, const uint64_t dims_in[4], con
     });
 }
 
+// bf16 matrix [rows][cols] with a row pitch, boxes of box_rows x 64 columns (128 bytes) in the 128-byte swizzle: the
+// operand tiles of the attention kernel.
+bool encode_2d_bf16_sw128(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
+                          uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const TmapKey key{{4, reinterpret_cast<uint64_t>(base), cols, rows, pitch_bytes, box_rows, 0, 0}};
+    return cached_tensor_map(tm, key, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {cols, rows};
+        cuuint64_t strides[1] = {pitch_bytes};
+        cuuint32_t box[2] = {64, box_rows};
+        cuuint32_t estr[2] = {1, 1};
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
+}
+
 // Output tensor map for the epilogue's bulk stores: bf16 [rows][N] with pitch ldy, boxes of 32 rows x 32 columns
 // in the 64-byte swizzle the staging buffers are written in.
 bool encode_y(CUtensorMap* tm, const void* y, uint64_t N, uint64_t rows, uint64_t ldy) {

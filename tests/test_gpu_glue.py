@@ -127,6 +127,8 @@ ATTN_CASES = [
     (3, 64, 1024, 8),       # dh 128: the 8x8 level
     (1, 200, 128, 2),       # ragged: 200 = 128 + 72 queries and keys
     (1, 16, 64, 2),         # a 4x4 map
+    (3, 200, 128, 2),       # dh 64, ragged, several samples: the last key block of a sample reaches into the next one's rows
+    (2, 72, 256, 2),        # dh 128, ragged, two samples
 ]
 
 
@@ -147,6 +149,27 @@ def test_attention_matches_oracle(env, oracle, Nb, L, C, heads):
                              rms_rel=float(np.sqrt((err ** 2).mean() / (want ** 2).mean()))))
     assert np.all(err <= bound), f"largest error / bound = {(err / bound).max():.3f}"
     assert np.sqrt((err ** 2).mean() / (want ** 2).mean()) <= Y_BF16_RTOL
+
+
+@pytest.mark.parametrize("C,heads", [(128, 2), (256, 2), (96, 2)])
+def test_attention_follows_a_late_maximum(env, oracle, C, heads):
+    """Scores that grow by far more than the kernel's lazy-rescale threshold from one key block to the next: the keys of
+    each block of 64 are scaled up block by block, so the running maximum of every row has to move (and the output
+    accumulator has to be rescaled) at every block."""
+    torch, hq = env
+    Nb, L = 2, 320
+    x = inputs.activations((Nb * L, 3 * C), seed=77).reshape(Nb, L, 3 * C).copy()
+    x[:, :, :C] = np.abs(x[:, :, :C])                    # q, k >= 0: every score of a later block is larger
+    x[:, :, C:2 * C] = np.abs(x[:, :, C:2 * C]) * (1.0 + 1.5 * (np.arange(L) // 64))[None, :, None]
+    qkv, qr = bf16(torch, x.reshape(Nb * L, 3 * C).astype(np.float32))
+    out = torch.empty((Nb * L, C), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    hq.hq_attention(qkv, Nb, heads, out, dev_status=status)
+    torch.cuda.synchronize()
+    hq.hq_check_status(status)
+    want = oracle.attention(qr.reshape(Nb, L, 3 * C), heads).reshape(Nb * L, C)
+    err = np.abs(out.float().cpu().numpy().astype(np.float64) - want)
+    assert np.all(err <= attention_bound(oracle, qr, Nb, L, C, heads, want))
 
 
 def test_attention_refuses_unsupported_head_width(env):
