@@ -379,43 +379,56 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t idesc_o = make_idesc_bf16(kQTile, DH, true);
 
     float m_run = -INFINITY, l_run = 0.f;
-    uint32_t ph_mma = 0, ph_kv = 0;
+    uint32_t ph_mma = 0;
     bool ok = true;
+    // S of block 0
+    if (warp == 0) {
+        if (tid == 0) {
+            bool ready = mbar_wait(&bar_q, 0, p.dev_status, kStatusAttnTma);
+            if (ready) q_flying = false;
+            ready = ready && mbar_wait(&bar_k, 0, p.dev_status, kStatusAttnTma);
+            if (ready) {
+                k_flying = false;
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < DH / 16; ++k) {
+                    const uint64_t a = make_sw128_kmajor_desc(smem_u32(sQ + (k / 4) * kQHalf)) + uint64_t(2 * (k & 3));
+                    const uint64_t b = make_sw128_kmajor_desc(smem_u32(sK + (k / 4) * kKVHalf)) + uint64_t(2 * (k & 3));
+                    mma_bf16(tmem_base, a, b, idesc_s, k != 0 ? 1u : 0u);
+                }
+                mma_commit(&bar_mma);
+            }
+        }
+        __syncwarp();
+    }
+    // Block j: wait for S(j) (and O += P V of block j - 1, issued in the same batch), refill the buffers those MMAs have
+    // read, softmax from registers, then one batch of MMAs again: O += P(j) V(j) and S(j + 1) -- the S columns are free as
+    // soon as every thread holds its row in registers, so the two products share one trip to the tensor core.
     for (int j = 0; j < nblocks && ok; ++j) {
         const int k0 = j * KB;
         const int kvalid = L - k0 < KB ? L - k0 : KB;
-        // ---- S = Q K^T
-        if (warp == 0) {
-            if (tid == 0) {
-                bool ready = j > 0 || mbar_wait(&bar_q, 0, p.dev_status, kStatusAttnTma);
-                if (ready) q_flying = false;
-                ready = ready && mbar_wait(&bar_k, ph_kv, p.dev_status, kStatusAttnTma);
-                if (ready) {
-                    k_flying = false;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < DH / 16; ++k) {
-                        const uint64_t a = make_sw128_kmajor_desc(smem_u32(sQ + (k / 4) * kQHalf)) + uint64_t(2 * (k & 3));
-                        const uint64_t b = make_sw128_kmajor_desc(smem_u32(sK + (k / 4) * kKVHalf)) + uint64_t(2 * (k & 3));
-                        mma_bf16(tmem_base, a, b, idesc_s, k != 0 ? 1u : 0u);
-                    }
-                    mma_commit(&bar_mma);
-                }
-            }
-            __syncwarp();
-        }
         ok = mbar_wait(&bar_mma, ph_mma, p.dev_status, kStatusAttnWait);
         ph_mma ^= 1;
         ok = __syncthreads_and(ok);
         if (!ok) break;
         tc_fence_after();
-        if (tid == 0 && j + 1 < nblocks) {                     // the K buffer is free: the next block's keys
-            mbar_expect_tx(&bar_k, NH * kKVHalf);
+        if (tid == 0) {
+            if (j + 1 < nblocks) {                             // the K buffer is free: the next block's keys
+                mbar_expect_tx(&bar_k, NH * kKVHalf);
 #pragma unroll
-            for (int h = 0; h < NH; ++h)
-                tma_load_2d(sK + h * kKVHalf, &tmKV, &bar_k, C + head * DH + 64 * h, row0 + k0 + KB);
-            k_flying = true;
-            k_par = uint32_t(j + 1) & 1u;
+                for (int h = 0; h < NH; ++h)
+                    tma_load_2d(sK + h * kKVHalf, &tmKV, &bar_k, C + head * DH + 64 * h, row0 + k0 + KB);
+                k_flying = true;
+                k_par = uint32_t(j + 1) & 1u;
+            }
+            if (j > 0) {                                       // the V buffer is free: this block's values
+                mbar_expect_tx(&bar_v, NH * kKVHalf);
+#pragma unroll
+                for (int h = 0; h < NH; ++h)
+                    tma_load_2d(sV + h * kKVHalf, &tmKV, &bar_v, 2 * C + head * DH + 64 * h, row0 + k0);
+                v_flying = true;
+                v_par = uint32_t(j) & 1u;
+            }
         }
         // ---- the row's KB scores come into registers once: maximum, P = exp2(c (S - m)), row sum, P as bf16 to smem
         const bool full = kvalid == KB;
@@ -470,11 +483,15 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         fence_proxy_async_smem();
         tc_fence_before();
         __syncthreads();
-        // ---- O += P V
         if (warp == 0) {
             if (tid == 0) {
-                if (mbar_wait(&bar_v, ph_kv, p.dev_status, kStatusAttnTma)) {
-                    v_flying = false;
+                bool ready = mbar_wait(&bar_v, uint32_t(j) & 1u, p.dev_status, kStatusAttnTma);
+                if (ready) v_flying = false;
+                if (ready && j + 1 < nblocks) {
+                    ready = mbar_wait(&bar_k, uint32_t(j + 1) & 1u, p.dev_status, kStatusAttnTma);
+                    if (ready) k_flying = false;
+                }
+                if (ready) {
                     tc_fence_after();
                     const uint64_t a = make_desc_noswizzle(smem_u32(sP), 128, kPGroup);
                     const uint64_t b = make_sw128_mnmajor_desc(smem_u32(sV), kKVHalf);
@@ -482,25 +499,24 @@ attention_tma_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     for (int k = 0; k < KB / 16; ++k)        // 16 keys on: two core-matrix columns of P, 16 rows of V
                         mma_bf16(tmem_base + uint32_t(KB), a + uint64_t(k * 16), b + uint64_t(k * 128), idesc_o,
                                  (j | k) != 0 ? 1u : 0u);
+                    if (j + 1 < nblocks) {
+#pragma unroll
+                        for (int k = 0; k < DH / 16; ++k) {
+                            const uint64_t qa = make_sw128_kmajor_desc(smem_u32(sQ + (k / 4) * kQHalf)) + uint64_t(2 * (k & 3));
+                            const uint64_t kb = make_sw128_kmajor_desc(smem_u32(sK + (k / 4) * kKVHalf)) + uint64_t(2 * (k & 3));
+                            mma_bf16(tmem_base, qa, kb, idesc_s, k != 0 ? 1u : 0u);
+                        }
+                    }
                     mma_commit(&bar_mma);
                 }
             }
             __syncwarp();
         }
-        ph_kv ^= 1;
+    }
+    if (ok) {                                                  // the last O += P V
         ok = mbar_wait(&bar_mma, ph_mma, p.dev_status, kStatusAttnWait);
-        ph_mma ^= 1;
         ok = __syncthreads_and(ok);
-        if (!ok) break;
         tc_fence_after();
-        if (tid == 0 && j + 1 < nblocks) {                     // the V buffer is free: the next block's values
-            mbar_expect_tx(&bar_v, NH * kKVHalf);
-#pragma unroll
-            for (int h = 0; h < NH; ++h)
-                tma_load_2d(sV + h * kKVHalf, &tmKV, &bar_v, 2 * C + head * DH + 64 * h, row0 + k0 + KB);
-            v_flying = true;
-            v_par = uint32_t(j + 1) & 1u;
-        }
     }
     if (!ok && tid == 0) {
         // a wait ran out: the loads still on their way must land before the CTA's shared memory is given up
