@@ -629,6 +629,15 @@ def main_unet(args):
     stream = torch.cuda.current_stream()
     for _ in range(max(3, min(args.warmup, 5))):
         net.run()
+    if args.profile_forward:
+        torch.cuda.synchronize()
+        torch.cuda.profiler.start()
+        net.run()
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
+        hq.hq_check_status(net.status)
+        print(json.dumps(dict(workload="unet", batch=batch, profiled_forwards=1, library_calls=len(net.tape))))
+        return
     t_one = timed_region(torch, net.run, 2, stream) / 2
     steps = max(args.steps, int(600.0 / max(t_one, 1e-3)) + 1)          # at least 0.6 s in the timed region
     sampler = ClockSampler(0)
@@ -912,6 +921,9 @@ def main():
     ap.add_argument("--pair-gemm", action="store_true",
                     help="run the short-reduction products on pairs of SMs (tcgen05.mma.cta_group::2; hq_set_pair_gemm)")
     ap.add_argument("--print-csrc-digest", action="store_true", help="print the digest profiles/dram_traffic.json records")
+    ap.add_argument("--profile-forward", action="store_true",
+                    help="--workload unet: run one forward between cudaProfilerStart / Stop and exit (for a profiler's "
+                         "launch list with --profile-from-start off)")
     args = ap.parse_args()
     if args.print_csrc_digest:
         print(csrc_digest())
