@@ -75,7 +75,13 @@ def test_upsample_and_concat(env, oracle):
 
 
 @pytest.mark.parametrize("silu", [False, True])
-@pytest.mark.parametrize("Nb,H,W,C,G", [(2, 8, 8, 128, 32), (3, 4, 4, 384, 32), (1, 16, 16, 64, 8)])
+@pytest.mark.parametrize("Nb,H,W,C,G", [
+    (2, 8, 8, 128, 32),         # four channels per group: the two channel quads of a 16-byte piece lie in different groups
+    (3, 4, 4, 384, 32),         # twelve channels per group, 48 pieces per pixel (not a divisor of the CTA size)
+    (1, 16, 16, 64, 8),
+    (70, 3, 7, 64, 8),          # 21 pixels per sample: a CTA's share of the pixels crosses several sample boundaries
+    (2, 40, 40, 256, 32),       # 1600 pixels per sample: shares end inside a sample, rounds of loads with a ragged tail
+])
 def test_groupnorm_act(env, oracle, silu, Nb, H, W, C, G):
     torch, hq = env
     x, xr = bf16(torch, inputs.activations((Nb, H, W, C), outlier_count=2, outlier_scale=8.0, seed=C) + np.float32(0.4))

@@ -1,5 +1,5 @@
 """GPU parity of GroupNorm + SiLU fused in front of the transform + quantization (hq_gn_silu_quant) against the CPU
-oracle.  The prologue runs in fp32 with the hardware's fast exponential and division; the transform that follows sums
+oracle.  The prologue runs in fp32 with the hardware's approximate exponential and reciprocal; the transform that follows sums
 a whole block of such values, over which their independent errors average out, so the codes are held to the same rule
 as the plain kernel's (one step of difference only within 1e-6 of the row's full scale from a rounding boundary, for at
 most 1e-4 of the codes) and the scales to the same 1e-6.  Measured on these cases: no differing code in 1.0 M codes
@@ -69,6 +69,33 @@ def test_gn_silu_quant_matches_oracle(env, oracle, Nb, H, W, C, G, n, bits, dt, 
     s_gpu = scales.cpu().numpy()[:, None] if not static else np.float32(s0)
     inside = np.abs(v) < oracle.qmax(bits)
     assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)
+
+
+def test_gn_silu_quant_on_an_input_aligned_to_8_bytes_only(env, oracle):
+    """A bf16 tensor that starts 8 bytes into an allocation: the statistics pass then reads four channels per load."""
+    torch, hq = env
+    Nb, H, W, C, G, n = 2, 8, 8, 128, 32, 128
+    x = inputs.activations((Nb, H, W, C), outlier_count=1, outlier_scale=8.0, seed=3) + np.float32(0.5)
+    rng = np.random.default_rng(5)
+    gamma = (1.0 + 0.2 * rng.standard_normal(C)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(C)).astype(np.float32)
+    store = torch.zeros((x.size + 4,), dtype=torch.bfloat16, device="cuda")
+    xt = store[4:].view(Nb, H, W, C)
+    xt.copy_(torch.from_numpy(x).cuda().to(torch.bfloat16))
+    assert xt.data_ptr() % 16 == 8
+    x = xt.float().cpu().numpy()
+    rows = Nb * H * W
+    codes = torch.zeros((rows, C // 2), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((rows,), dtype=torch.float32, device="cuda")
+    scratch = torch.empty((Nb * G * 24,), dtype=torch.uint8, device="cuda")
+    hq.hq_gn_silu_quant(xt, G, torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), 1e-6, n, 4, codes,
+                        hq.HQ_CODES_NIBBLE, scratch, scales=scales)
+    torch.cuda.synchronize()
+    u = oracle.transform(oracle.groupnorm_silu(x, G, gamma, beta, 1e-6).reshape(rows, C), n)
+    q_ref, s_ref, v = oracle.quantize(u, 4, want_v=True)
+    assert float(np.abs(scales.cpu().numpy() / s_ref - 1.0).max()) <= GN_SCALE_RTOL
+    check_codes(unpack_nibbles_np(codes.cpu().numpy()), q_ref, v, "groupnorm prologue, 8-byte aligned input",
+                tie_rel=GN_TIE_REL, mismatch_frac=GN_MISMATCH_FRAC)
 
 
 LN_TIE_REL = CODE_TIE_REL
