@@ -234,18 +234,22 @@ hq_status hq_ln_qlinear(const void* x, hq_dtype xdt, int64_t M, int64_t K, int64
  * groups   groups of C/groups consecutive channels (a multiple of 4 each); statistics per (sample, group) over
  *          H*W*(C/groups) values: y = (x - mean) / sqrt(var + eps) * gamma[c] + beta[c]; then y * sigmoid(y).
  * gamma, beta  device [C].   The rest as hq_hadamard_quant with rows = Nb*H*W, cols = C (transform over channels).
+ * pre_bias device bf16 [Nb][C], 8-byte aligned, or NULL: a per-sample, per-channel addend (the projected step
+ *          embedding of a residual block) that is added to x BEFORE the normalisation -- the statistics are those of
+ *          x + pre_bias -- without the sum ever being written: the statistics pass adds it as it reads, and the
+ *          quantize pass folds it into its per-channel offset.  Read only.
  * scratch  device, 16-byte aligned, Nb * groups * 24 bytes: fp64 sums (cleared by the call) and the statistics.
  * Restrictions: had_block in 32..4096 with at most 320 threads per CTA shape (else HQ_ERR_UNSUPPORTED), and the
  * rows of a sample must be a multiple of the rows one CTA takes (any H*W that is a multiple of 32 is). */
 hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
-                           const float* gamma, const float* beta, float eps, int had_block, int bits,
+                           const float* gamma, const float* beta, const void* pre_bias, float eps, int had_block, int bits,
                            hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                            int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, void* stream);
 
 /* The fused convolution layer with that prologue: GroupNorm + SiLU -> transform -> quantize -> integer convolution ->
  * rescale.  Arguments as hq_gn_silu_quant and hq_qconv. */
 hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
-                           const float* gamma, const float* beta, float eps, const hq_weight_desc* desc,
+                           const float* gamma, const float* beta, const void* pre_bias, float eps, const hq_weight_desc* desc,
                            const void* w_dev, int R, int S, int stride, int pad, const float* scale_w,
                            const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale, void* y,
                            hq_dtype ydt, void* workspace, size_t ws_bytes, void* scratch, size_t scratch_bytes,

@@ -56,7 +56,7 @@ def forward(cfg: dict, P: dict, x, t, y, static: dict, a_bits: int = 4, w_bits: 
     def resblock(name, h, semb):
         cin, cout = h.shape[-1], P[name + ".conv1.w"].shape[0]
         a = conv3(name + ".conv1", h, norm=name + ".norm1")
-        a = st(a + linear(name + ".emb", semb)[:, None, None, :])
+        a = a + linear(name + ".emb", semb)[:, None, None, :]     # feeds the normalisation directly: not a kept tensor
         a = conv3(name + ".conv2", a, norm=name + ".norm2")
         skip = h if cin == cout else conv1(name + ".skip", h)
         return keep(name, st(skip + a))

@@ -81,12 +81,12 @@ def _load():
     L.hq_hadamard_quant_width2.restype = C.c_int
     L.hq_qconv_width.argtypes = [p, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32, i32,
                                  p, p, i32, p, C.c_size_t, p, p]
-    L.hq_gn_silu_quant.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, i32, i32, i32, p, p, i32, i64, p, p,
+    L.hq_gn_silu_quant.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, p, C.c_float, i32, i32, i32, p, p, i32, i64, p, p,
                                    C.c_size_t, p]
     L.hq_ln_quant.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, i32, i32, i32, p, p, i32, i64, p, p]
     L.hq_ln_qlinear.argtypes = [p, i32, i64, i64, i64, p, p, i64, C.c_float, C.POINTER(WeightDesc), p, p, p, i32, p, i32, i64,
                                 p, C.c_size_t, p, p]
-    L.hq_gn_silu_qconv.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, C.c_float, C.POINTER(WeightDesc), p, i32, i32, i32,
+    L.hq_gn_silu_qconv.argtypes = [p, i32, i64, i64, i64, i64, i32, p, p, p, C.c_float, C.POINTER(WeightDesc), p, i32, i32, i32,
                                    i32, p, p, i32, i32, p, p, i32, p, C.c_size_t, p, C.c_size_t, p, p]
     L.hq_gn_qlinear.argtypes = [p, i32, i64, i64, i64, i32, p, p, C.c_float, i32, C.POINTER(WeightDesc), p, p, p, i32, p, i32,
                                 i64, p, C.c_size_t, p, C.c_size_t, p, p]
@@ -262,22 +262,25 @@ def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias,
 
 
 def hq_gn_silu_quant(x, groups: int, gamma, beta, eps: float, had_block: int, bits: int, codes, container: int,
-                     scratch, scales=None, static_scale=None, stream=None) -> None:
-    """GroupNorm(groups) + SiLU of x NHWC, then transform over channels + quantization into codes [Nb*H*W, pitch]."""
+                     scratch, scales=None, static_scale=None, stream=None, pre_bias=None) -> None:
+    """GroupNorm(groups) + SiLU of x NHWC (of x + pre_bias[n, c] when a bf16 [Nb, C] addend is given), then transform
+    over channels + quantization into codes [Nb*H*W, pitch]."""
     Nb, H, W, Cin = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
-    _check(lib.hq_gn_silu_quant(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), eps, had_block,
+    _check(lib.hq_gn_silu_quant(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps, had_block,
                                 bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
                                 _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)),
            "hq_gn_silu_quant")
 
 
 def hq_gn_silu_qconv(x, groups: int, gamma, beta, eps: float, pw: PreparedWeight, R: int, S: int, stride: int, pad: int,
-                     bias, a_bits: int, y, workspace, scratch, static_scale=None, dev_status=None, stream=None) -> None:
-    """The fused convolution layer with GroupNorm + SiLU in front (x NHWC)."""
+                     bias, a_bits: int, y, workspace, scratch, static_scale=None, dev_status=None, stream=None,
+                     pre_bias=None) -> None:
+    """The fused convolution layer with GroupNorm + SiLU in front (x NHWC; pre_bias: bf16 [Nb, C] added to x before the
+    normalisation, or None)."""
     Nb, H, W, Cin = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
-    _check(lib.hq_gn_silu_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), eps,
+    _check(lib.hq_gn_silu_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps,
                                 C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride, pad, _dptr(pw.s_w_dev), _dptr(bias),
                                 a_bits, mode, _dptr(static_scale), _dptr(y), _dtype_code(y), _dptr(workspace),
                                 workspace.numel() * workspace.element_size(), _dptr(scratch),

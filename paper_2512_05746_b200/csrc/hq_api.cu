@@ -26,7 +26,7 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
                                const float* gamma, const float* beta, float eps, int had_block, int bits,
                                hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                                int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
-                               int silu);
+                               int silu, const void* pre_bias);
 hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
                           const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
                           hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
@@ -128,7 +128,8 @@ extern "C" hq_status hq_ln_qlinear(const void* x, hq_dtype xdt, int64_t M, int64
 }
 
 extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
-                                      const float* gamma, const float* beta, float eps, const hq_weight_desc* desc,
+                                      const float* gamma, const float* beta, const void* pre_bias, float eps,
+                                      const hq_weight_desc* desc,
                                       const void* w_dev, int R, int S, int stride, int pad, const float* scale_w,
                                       const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale, void* y,
                                       hq_dtype ydt, void* workspace, size_t ws_bytes, void* scratch, size_t scratch_bytes,
@@ -148,7 +149,7 @@ extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, i
     unsigned char* codes = static_cast<unsigned char*>(workspace);
     float* scales = reinterpret_cast<float*>(codes + scales_offset(rows, C, cont));
     s = launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, desc->had_block, a_bits, mode, static_scale, codes,
-                             cont, ldc, scales, scratch, scratch_bytes, st, 1);
+                             cont, ldc, scales, scratch, scratch_bytes, st, 1, pre_bias);
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st, true);
@@ -176,7 +177,8 @@ extern "C" hq_status hq_gn_qlinear(const void* x, hq_dtype xdt, int64_t Nb, int6
     float* scales = reinterpret_cast<float*>(codes + scales_offset(M, C, cont));
     const int64_t ldc = code_pitch(C, cont);
     s = launch_gn_silu_quant(x, xdt, Nb, rows_per_sample, 1, C, groups, gamma, beta, eps, desc->had_block, a_bits,
-                             HQ_SCALE_PER_ROW, nullptr, codes, cont, ldc, scales, scratch, scratch_bytes, st, silu != 0);
+                             HQ_SCALE_PER_ROW, nullptr, codes, cont, ldc, scales, scratch, scratch_bytes, st, silu != 0,
+                             nullptr);
     if (s != HQ_OK) return s;
     return launch_qgemm(codes, cont, a_bits, M, C, ldc, desc, w_dev, scales, 0, scale_w, bias, hq_alpha_for(desc), nullptr,
                         y, ydt, ldy, dev_status, st, true);

@@ -11,7 +11,8 @@ namespace hq {
 // GroupNorm statistics of an NHWC tensor into `scratch` (defined in hq_quant.cu): [samples][groups][2] fp64 sums,
 // followed by [samples][groups][2] floats (mean, 1/sqrt(var + eps)).
 hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
-                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st);
+                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st,
+                          const void* pre_bias);
 
 namespace {
 
@@ -394,7 +395,7 @@ extern "C" hq_status hq_groupnorm_act(const void* x, int64_t Nb, int64_t H, int6
     if (!aligned16(x) || !aligned16(out) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float* stats = nullptr;
-    hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st);
+    hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st, nullptr);
     if (s != HQ_OK) return s;
     if (Nb > 65535) return HQ_ERR_UNSUPPORTED;
     const int c8 = int(C / 8);

@@ -41,6 +41,7 @@ struct QuantParams {
     const float* gn_beta;    // [cols]
     int gn_groups;
     int gn_silu;             // 1: SiLU after the normalisation, 0: none
+    const __nv_bfloat16* gn_pre_bias;   // [samples][cols] added to x before the normalisation, or nullptr
     int gn_sets_per_sample;  // CTAs per sample (a CTA never straddles two samples)
     int gn_cg;               // channels per group, and its log2 when it is a power of two (else -1)
     int gn_cg_shift;
@@ -152,9 +153,16 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
             const float4 gm = __ldg(reinterpret_cast<const float4*>(p.gn_gamma + c));
             const float4 bt = __ldg(reinterpret_cast<const float4*>(p.gn_beta + c));
             const float4 a = make_float4(ms.y * gm.x, ms.y * gm.y, ms.y * gm.z, ms.y * gm.w);
+            // (x + e - mean) a + beta = x a + (beta + (e - mean) a): the per-sample addend e costs nothing per element
+            float4 sh = make_float4(-ms.x, -ms.x, -ms.x, -ms.x);
+            if (p.gn_pre_bias != nullptr) {
+                const uint2 er = __ldg(reinterpret_cast<const uint2*>(p.gn_pre_bias + size_t(sample) * p.cols + c));
+                sh.x += __uint_as_float(er.x << 16); sh.y += __uint_as_float(er.x & 0xFFFF0000u);
+                sh.z += __uint_as_float(er.y << 16); sh.w += __uint_as_float(er.y & 0xFFFF0000u);
+            }
             *reinterpret_cast<float4*>(gn_a + c) = a;
-            *reinterpret_cast<float4*>(gn_b + c) = make_float4(fmaf(-ms.x, a.x, bt.x), fmaf(-ms.x, a.y, bt.y),
-                                                               fmaf(-ms.x, a.z, bt.z), fmaf(-ms.x, a.w, bt.w));
+            *reinterpret_cast<float4*>(gn_b + c) = make_float4(fmaf(sh.x, a.x, bt.x), fmaf(sh.y, a.y, bt.y),
+                                                               fmaf(sh.z, a.z, bt.z), fmaf(sh.w, a.w, bt.w));
         }
         __syncthreads();
     }
@@ -539,9 +547,9 @@ __device__ __forceinline__ void gn_quad(const GnPiece<8>& r, int q, f32x2& lo, f
 }
 
 template <typename InT, int VEC>
-__global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, int64_t hw, int64_t total_px, int64_t span, int C,
-                                                          int groups, double* sums, float* stats, double inv_count,
-                                                          double eps) {
+__global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, const __nv_bfloat16* pre_bias, int64_t hw,
+                                                          int64_t total_px, int64_t span, int C, int groups, double* sums,
+                                                          float* stats, double inv_count, double eps) {
     constexpr int Q = VEC / 4;                         // channel quads per piece
     constexpr int U = 8;                               // loads in flight per thread
     __shared__ double red[2 * Q][256];
@@ -562,9 +570,18 @@ __global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, int64_t 
         for (int cbase = 0; cbase < pieces; cbase += nq) {
             const int col = cbase + col0;
             double s1[Q], s2[Q];
+            f32x2 e_lo[Q], e_hi[Q];                    // the sample's addend on this thread's channels (zero: none)
 #pragma unroll
-            for (int q = 0; q < Q; ++q) { s1[q] = 0.0; s2[q] = 0.0; }
+            for (int q = 0; q < Q; ++q) { s1[q] = 0.0; s2[q] = 0.0; e_lo[q] = pk2(0.f, 0.f); e_hi[q] = pk2(0.f, 0.f); }
             if (pl < ppl && col < pieces) {
+                if (pre_bias != nullptr) {
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        const uint2 er = __ldg(reinterpret_cast<const uint2*>(pre_bias + sample * C + int64_t(col) * VEC + 4 * q));
+                        e_lo[q] = pk2(__uint_as_float(er.x << 16), __uint_as_float(er.x & 0xFFFF0000u));
+                        e_hi[q] = pk2(__uint_as_float(er.y << 16), __uint_as_float(er.y & 0xFFFF0000u));
+                    }
+                }
                 const InT* src = x + int64_t(col) * VEC;
                 int64_t px = r0 + pl;
                 for (; px + (U - 1) * ppl < seg_end; px += U * ppl) {
@@ -578,6 +595,8 @@ __global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, int64_t 
                         for (int u = 0; u < U; ++u) {
                             f32x2 lo, hi;
                             gn_quad(raw[u], q, lo, hi);
+                            lo = add2(lo, e_lo[q]);
+                            hi = add2(hi, e_hi[q]);
                             a = add2(a, add2(lo, hi));
                             b = fma2(lo, lo, fma2(hi, hi, b));
                         }
@@ -594,6 +613,8 @@ __global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, int64_t 
                     for (int q = 0; q < Q; ++q) {
                         f32x2 lo, hi;
                         gn_quad(raw, q, lo, hi);
+                        lo = add2(lo, e_lo[q]);
+                        hi = add2(hi, e_hi[q]);
                         float a0, a1, b0, b1;
                         upk2(add2(lo, hi), a0, a1);
                         upk2(fma2(lo, lo, mul2(hi, hi)), b0, b1);
@@ -697,7 +718,8 @@ cudaError_t dispatch_fast(int klog, const QuantParams& p, bool int8_out, int gri
 }  // namespace
 
 // Launches the transform+quantize kernel; shared by the public entry point and the fused layer calls.
-struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; int silu; };
+struct GnArgs { const float* stats; const float* gamma; const float* beta; int groups; int64_t rows_per_sample; int silu;
+                const __nv_bfloat16* pre_bias; };
 struct LnArgs { const float* w; const float* b; int64_t rows_per_group; float eps; };
 
 static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
@@ -732,6 +754,7 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
     if (gn != nullptr) {
         p.gn_stats = gn->stats; p.gn_gamma = gn->gamma; p.gn_beta = gn->beta; p.gn_groups = gn->groups;
         p.gn_silu = gn->silu;
+        p.gn_pre_bias = gn->pre_bias;
         p.gn_cg = int(cols / gn->groups);
         p.gn_cg_shift = is_pow2(p.gn_cg) ? ilog2(p.gn_cg) : -1;
     }
@@ -804,7 +827,8 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
 // GroupNorm statistics of an NHWC tensor (hw pixels per sample): fp64 sums per (sample, group) in `scratch` (cleared
 // here), then mean and 1/sqrt(var + eps) as floats behind them.  scratch: Nb * groups * (2 doubles + 2 floats).
 hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
-                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st) {
+                          void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st,
+                          const void* pre_bias) {
     if (x == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
     if (Nb <= 0 || hw <= 0 || C <= 0 || groups <= 0) return HQ_ERR_SHAPE;
@@ -815,6 +839,8 @@ hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, i
     if (reinterpret_cast<uintptr_t>(scratch) % 16 != 0) return HQ_ERR_ALIGNMENT;
     const int elt = xdt == HQ_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(x) % (4 * elt) != 0) return HQ_ERR_ALIGNMENT;
+    if (pre_bias != nullptr && reinterpret_cast<uintptr_t>(pre_bias) % 8 != 0) return HQ_ERR_ALIGNMENT;
+    const __nv_bfloat16* pre = static_cast<const __nv_bfloat16*>(pre_bias);
     double* sums = static_cast<double*>(scratch);
     float* stats = reinterpret_cast<float*>(sums + size_t(Nb) * groups * 2);
     HQ_CUDA_OK(cudaMemsetAsync(scratch, 0, need, st));             // the sums and the ticket counters
@@ -833,13 +859,13 @@ hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, i
     const double inv_count = 1.0 / (double(hw) * double(C / groups));
     const unsigned grid = unsigned(ctas);
     if (xdt == HQ_F32)
-        gn_stats_kernel<float, 4><<<grid, 256, 0, st>>>(static_cast<const float*>(x), hw, total_px, span, int(C), groups, sums,
+        gn_stats_kernel<float, 4><<<grid, 256, 0, st>>>(static_cast<const float*>(x), pre, hw, total_px, span, int(C), groups, sums,
                                                        stats, inv_count, double(eps));
     else if (wide)
-        gn_stats_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), hw, total_px, span, int(C),
+        gn_stats_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), pre, hw, total_px, span, int(C),
                                                                groups, sums, stats, inv_count, double(eps));
     else
-        gn_stats_kernel<__nv_bfloat16, 4><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), hw, total_px, span, int(C),
+        gn_stats_kernel<__nv_bfloat16, 4><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), pre, hw, total_px, span, int(C),
                                                                groups, sums, stats, inv_count, double(eps));
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
     *stats_out = stats;
@@ -852,14 +878,14 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
                                const float* gamma, const float* beta, float eps, int had_block, int bits,
                                hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                                int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
-                               int silu) {
+                               int silu, const void* pre_bias) {
     if (gamma == nullptr || beta == nullptr) return HQ_ERR_INVALID_ARG;
     if (H <= 0 || W <= 0) return HQ_ERR_SHAPE;
     const int64_t hw = H * W;
     const float* stats = nullptr;
-    hq_status s = launch_gn_stats(x, xdt, Nb, hw, C, groups, eps, scratch, scratch_bytes, &stats, st);
+    hq_status s = launch_gn_stats(x, xdt, Nb, hw, C, groups, eps, scratch, scratch_bytes, &stats, st, pre_bias);
     if (s != HQ_OK) return s;
-    const GnArgs gn{stats, gamma, beta, groups, hw, silu};
+    const GnArgs gn{stats, gamma, beta, groups, hw, silu, static_cast<const __nv_bfloat16*>(pre_bias)};
     return launch_quant_impl(x, xdt, Nb * hw, C, C, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales, &gn,
                              st);
 }
@@ -964,12 +990,13 @@ extern "C" hq_status hq_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int6
 }
 
 extern "C" hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
-                                      int groups, const float* gamma, const float* beta, float eps, int had_block,
-                                      int bits, hq_scale_mode mode, const float* static_scale, void* codes,
+                                      int groups, const float* gamma, const float* beta, const void* pre_bias, float eps,
+                                      int had_block, int bits, hq_scale_mode mode, const float* static_scale, void* codes,
                                       hq_container cont, int64_t ld_codes, float* scales, void* scratch,
                                       size_t scratch_bytes, void* stream) {
     return hq::launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, had_block, bits, mode, static_scale, codes,
-                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream), 1);
+                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream), 1,
+                                    pre_bias);
 }
 
 extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,

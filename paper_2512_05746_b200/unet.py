@@ -156,7 +156,7 @@ class UNet:
         return self.ws[: rows * pitch].view(rows, pitch), self.ws[off: off + rows * 4].view(self.torch.float32)
 
     # ------------------------------------------------------------------ layers
-    def _conv3(self, name, x, norm=None, stride=1):
+    def _conv3(self, name, x, norm=None, stride=1, pre_bias=None):
         hq, t = self.hq, self.torch
         Nb, H, W, Cin = x.shape
         pw = self.pw[name]
@@ -173,7 +173,7 @@ class UNet:
             codes, sc = self._ws_views(Nb * H * W, Cin)
             if g:
                 hq.hq_gn_silu_quant(x, G, g[0], g[1], self.EPS, pw.desc.had_block, self.a_bits, codes, self.cont, self.scratch,
-                                    scales=sc)
+                                    scales=sc, pre_bias=pre_bias)
             else:
                 hq.hq_hadamard_quant(x.view(-1, Cin), pw.desc.had_block, self.a_bits, codes, self.cont, scales=sc)
             ss.copy_(sc.max().reshape(1))
@@ -182,11 +182,11 @@ class UNet:
             calibrate()
             if g:
                 hq.hq_gn_silu_qconv(x, G, g[0], g[1], self.EPS, pw, 3, 3, stride, 1, bias, self.a_bits, y, self.ws, self.scratch,
-                                    static_scale=ss, dev_status=self.status)
+                                    static_scale=ss, dev_status=self.status, pre_bias=pre_bias)
             else:
                 hq.hq_qconv(x, pw, 3, 3, stride, 1, bias, self.a_bits, y, self.ws, static_scale=ss, dev_status=self.status)
 
-        self._emit("q", name, run, lambda: dict(op="conv3", x=x, y=y, norm=norm, stride=stride, static=ss,
+        self._emit("q", name, run, lambda: dict(op="conv3", x=x, y=y, norm=norm, stride=stride, static=ss, pre_bias=pre_bias,
                                                 codes=self._ws_views(Nb * H * W, Cin)[0]))
         return y
 
@@ -227,8 +227,8 @@ class UNet:
         cin, cout = x.shape[-1], self.pw[name + ".conv1"].desc.N
         h = self._conv3(name + ".conv1", x, norm=name + ".norm1")
         e = self._linear(name + ".emb", semb)
-        self._glue(name + ".emb_add", "add_rows_bcast", lambda: hq.hq_add_rows_bcast(h, e), e=e, out=h)
-        h2 = self._conv3(name + ".conv2", h, norm=name + ".norm2")
+        # h + e is never stored: the second convolution's normalisation takes the embedding as a per-sample addend
+        h2 = self._conv3(name + ".conv2", h, norm=name + ".norm2", pre_bias=e)
         xs = x if cin == cout else self._conv1(name + ".skip", x)
         out = self._new(h2.shape)
         self._glue(name + ".residual", "add", lambda: hq.hq_add(xs, h2, out), a=xs, b=h2, out=out)

@@ -71,6 +71,43 @@ def test_gn_silu_quant_matches_oracle(env, oracle, Nb, H, W, C, G, n, bits, dt, 
     assert np.all(np.abs(u - s_gpu * q)[inside] <= 0.5 * np.max(s_gpu) * (1 + 1e-3) + 1e-6)
 
 
+@pytest.mark.parametrize("Nb,H,W,C,G,n,dt", [(3, 8, 8, 256, 32, 256, "bf16"), (2, 8, 8, 128, 32, 128, "f32"),
+                                             (5, 4, 8, 512, 32, 256, "bf16")])
+def test_gn_silu_quant_with_a_per_sample_addend(env, oracle, Nb, H, W, C, G, n, dt):
+    """pre_bias[n, c] (the projected step embedding of a residual block) is added in front of the normalisation without
+    the sum being stored: codes and scales against the oracle applied to x + pre_bias."""
+    torch, hq = env
+    x = inputs.activations((Nb, H, W, C), outlier_count=2, outlier_scale=8.0, seed=C + Nb) + np.float32(0.3)
+    e = (1.5 * inputs.activations((Nb, C), seed=Nb)).astype(np.float32)
+    rng = np.random.default_rng(C)
+    gamma = (1.0 + 0.2 * rng.standard_normal(C)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(C)).astype(np.float32)
+    xt = torch.from_numpy(x).cuda()
+    if dt == "bf16":
+        xt = xt.to(torch.bfloat16)
+        x = xt.float().cpu().numpy()
+    et = torch.from_numpy(e).cuda().to(torch.bfloat16)
+    e = et.float().cpu().numpy()
+    rows = Nb * H * W
+    codes = torch.zeros((rows, C // 2), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((rows,), dtype=torch.float32, device="cuda")
+    scratch = torch.empty((Nb * G * 24,), dtype=torch.uint8, device="cuda")
+    hq.hq_gn_silu_quant(xt, G, torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), 1e-5, n, 4, codes,
+                        hq.HQ_CODES_NIBBLE, scratch, scales=scales, pre_bias=et)
+    torch.cuda.synchronize()
+    xe = x.astype(np.float64) + e.astype(np.float64)[:, None, None, :]
+    u = oracle.transform(oracle.groupnorm_silu(xe, G, gamma, beta, 1e-5).reshape(rows, C), n)
+    q_ref, s_ref, v = oracle.quantize(u, 4, want_v=True)
+    assert float(np.abs(scales.cpu().numpy() / s_ref - 1.0).max()) <= GN_SCALE_RTOL
+    check_codes(unpack_nibbles_np(codes.cpu().numpy()), q_ref, v, f"groupnorm prologue with addend {Nb}x{H}x{W}x{C} {dt}",
+                tie_rel=GN_TIE_REL, mismatch_frac=GN_MISMATCH_FRAC)
+    # and the addend matters: without it the codes are others
+    hq.hq_gn_silu_quant(xt, G, torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), 1e-5, n, 4, codes,
+                        hq.HQ_CODES_NIBBLE, scratch, scales=scales)
+    torch.cuda.synchronize()
+    assert (unpack_nibbles_np(codes.cpu().numpy()) != q_ref).mean() > 0.2
+
+
 def test_gn_silu_quant_on_an_input_aligned_to_8_bytes_only(env, oracle):
     """A bf16 tensor that starts 8 bytes into an allocation: the statistics pass then reads four channels per load."""
     torch, hq = env

@@ -61,6 +61,8 @@ def test_every_layer_matches_the_oracle_on_the_devices_own_input(run, oracle):
             Nb, H, W, C = x.shape
             w, b = P[name + ".w"], P[name + ".b"]
             stride = r.get("stride", 1)
+            if r.get("pre_bias") is not None:                      # the step embedding, added in front of the normalisation
+                x = x + host(r["pre_bias"])[:, None, None, :]
             xin = oracle.groupnorm(x, G, P[r["norm"] + ".gamma"], P[r["norm"] + ".beta"], net.EPS, "silu") if r.get("norm") else x
             pw = net.pw[name]
             static = float(r["static"].cpu()[0]) if op == "conv3" else None
@@ -112,9 +114,6 @@ def test_every_layer_matches_the_oracle_on_the_devices_own_input(run, oracle):
                 before = host(by_name["time_embed.2"]["y"])
                 table = host(net.bf["label_emb"])
                 assert rel_err(out, before + table[r["labels"].cpu().numpy()]) <= Y_BF16_RTOL, name
-            elif op == "add_rows_bcast":
-                before = host(by_name[name.replace(".emb_add", ".conv1")]["y"])
-                assert rel_err(out, before + host(r["e"])[:, None, None, :]) <= Y_BF16_RTOL, name
             elif op == "add":
                 assert rel_err(out, (host(r["a"]) + host(r["b"])).reshape(out.shape)) <= Y_BF16_RTOL, name
             elif op == "concat":
@@ -139,6 +138,8 @@ def test_every_layer_matches_the_oracle_on_the_devices_own_input(run, oracle):
     # every call of the forward was checked: 16 residual blocks x 3-4 layers, 11 attention blocks x 2, 6 resampling convs, 2 embedding linears
     assert checked["q"] == len([1 for tag, _, _ in net.tape if tag == "q"]) and checked["q"] >= 80
     assert checked["g"] == len([1 for tag, _, _ in net.tape if tag == "g"])
+    # every residual block's second convolution took the block's embedding as its addend
+    assert [r["name"] for r in run["rec"] if r.get("pre_bias") is not None] == [r["name"] for r in run["rec"] if r["name"].endswith(".conv2")]
 
 
 def oracle_forward(run, oracle, a_bits, x=None):
