@@ -5,6 +5,7 @@
 // All activations are bf16, row-major with the channel axis contiguous (NHWC); arithmetic is fp32.
 // Every kernel is HBM-bound element-wise work: 16-byte loads and stores, one element group per thread.
 #include "hq_common.cuh"
+#include "hq_fwht.cuh"
 
 namespace hq {
 
@@ -302,6 +303,178 @@ __global__ void __launch_bounds__(256) conv_small_cout_kernel(const __nv_bfloat1
     }
 }
 
+// The 3x3, stride 1, pad 1 shapes of the network's first and last convolution.  What bounds them is the shared-memory
+// traffic of the weights (a warp-wide 16-byte read costs four wavefronts), so a warp of the first convolution takes EIGHT consecutive output
+// pixels of a row per weight read (the last one four), the input columns they touch in one filter row are fetched once per row (not once per
+// tap), the weights are laid out so that the 32 lanes of a 16-byte read touch consecutive addresses (a lane's eight
+// channels as two quads half a round apart: no bank conflicts), and the multiply-adds run two wide (`fma.f32x2`: an
+// input value is paired with itself or, for the last convolution, with its channel neighbour).
+constexpr int kConvPx = 8;      // first convolution (few registers per pixel)
+constexpr int kConvPxOut = 4;   // last convolution (ten input-column pieces of eight channels per row are already 40 registers)
+
+// Position of channel ch (of a round of up to 256 channels, eight per lane) in the conflict-free order.
+__device__ __forceinline__ int conv_slot(int ch, int half_stride) {
+    const int rnd = ch >> 8, cl = ch & 255;
+    return rnd * 256 + ((cl >> 2) & 1) * half_stride + (cl >> 3) * 4 + (cl & 3);
+}
+
+template <typename InT, int CIN>
+__global__ void __launch_bounds__(256) conv3x3_small_cin_kernel(const InT* x, const float* w, const float* bias,
+                                                                __nv_bfloat16* out, int Nb, int H, int W, int Cout) {
+    extern __shared__ float sw[];                      // [9 * CIN][Cout], channels in conflict-free order
+    constexpr int taps = 9 * CIN;
+    const int hs = (Cout < 256 ? Cout : 256) / 2;
+    for (int i = threadIdx.x; i < taps * Cout; i += blockDim.x) {
+        const int co = i / taps, k = i - co * taps;   // global layout [Cout][3][3][CIN]
+        sw[k * Cout + conv_slot(co, hs)] = w[i];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int wq = (W + kConvPx - 1) / kConvPx;        // groups of eight pixels per output row
+    const int64_t groups = int64_t(Nb) * H * wq;
+    for (int64_t g = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); g < groups;
+         g += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo0 = int(g % wq) * kConvPx;
+        const int ho = int((g / wq) % H);
+        const int n = int(g / (int64_t(wq) * H));
+        for (int co0 = lane * 8; co0 < Cout; co0 += 256) {
+            f32x2 acc[kConvPx][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float b0 = bias != nullptr ? __ldg(bias + co0 + 2 * j) : 0.f;
+                const float b1 = bias != nullptr ? __ldg(bias + co0 + 2 * j + 1) : 0.f;
+#pragma unroll
+                for (int pp = 0; pp < kConvPx; ++pp) acc[pp][j] = pk2(b0, b1);
+            }
+            const float* wbase = sw + (co0 & ~255) + lane * 4;
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+                const int hi = ho + r - 1;
+                if (hi < 0 || hi >= H) continue;
+                float xin[kConvPx + 2][CIN];
+                const InT* row = x + (int64_t(n) * H + hi) * W * CIN;
+#pragma unroll
+                for (int j = 0; j < kConvPx + 2; ++j) {
+                    const int wi = wo0 - 1 + j;
+                    const bool in = wi >= 0 && wi < W;
+#pragma unroll
+                    for (int c = 0; c < CIN; ++c) {
+                        float v = 0.f;
+                        if (in) {
+                            if (sizeof(InT) == 4) v = __ldg(reinterpret_cast<const float*>(row + wi * CIN + c));
+                            else v = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(row + wi * CIN + c));
+                        }
+                        xin[j][c] = v;
+                    }
+                }
+#pragma unroll
+                for (int sx = 0; sx < 3; ++sx) {
+#pragma unroll
+                    for (int c = 0; c < CIN; ++c) {
+                        const float* wr = wbase + ((r * 3 + sx) * CIN + c) * Cout;
+                        const ulonglong2 w0 = *reinterpret_cast<const ulonglong2*>(wr);
+                        const ulonglong2 w1 = *reinterpret_cast<const ulonglong2*>(wr + hs);
+#pragma unroll
+                        for (int pp = 0; pp < kConvPx; ++pp) {
+                            const f32x2 xv = pk2(xin[pp + sx][c], xin[pp + sx][c]);
+                            acc[pp][0] = fma2(w0.x, xv, acc[pp][0]);
+                            acc[pp][1] = fma2(w0.y, xv, acc[pp][1]);
+                            acc[pp][2] = fma2(w1.x, xv, acc[pp][2]);
+                            acc[pp][3] = fma2(w1.y, xv, acc[pp][3]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int pp = 0; pp < kConvPx; ++pp) {
+                if (wo0 + pp >= W) continue;
+                F8 f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) upk2(acc[pp][j], f.v[2 * j], f.v[2 * j + 1]);
+                *reinterpret_cast<uint4*>(out + ((int64_t(n) * H + ho) * W + wo0 + pp) * Cout + co0) = pack8(f);
+            }
+        }
+    }
+}
+
+template <int COUT>
+__global__ void __launch_bounds__(256) conv3x3_small_cout_kernel(const __nv_bfloat16* x, const float* w, const float* bias,
+                                                                 float* out, int Nb, int H, int W, int C) {
+    extern __shared__ float sw[];                      // [COUT][9][C], channels in conflict-free order
+    const int wsize = COUT * 9 * C;
+    const int hs = (C < 256 ? C : 256) / 2;
+    for (int i = threadIdx.x; i < wsize; i += blockDim.x) {
+        const int ot = i / C, c = i - ot * C;
+        sw[ot * C + conv_slot(c, hs)] = w[i];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int wq = (W + kConvPxOut - 1) / kConvPxOut;
+    const int64_t groups = int64_t(Nb) * H * wq;
+    for (int64_t g = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); g < groups;
+         g += int64_t(gridDim.x) * (blockDim.x >> 5)) {
+        const int wo0 = int(g % wq) * kConvPxOut;
+        const int ho = int((g / wq) % H);
+        const int n = int(g / (int64_t(wq) * H));
+        f32x2 acc[kConvPxOut][COUT];                      // even and odd input channels side by side
+#pragma unroll
+        for (int pp = 0; pp < kConvPxOut; ++pp)
+#pragma unroll
+            for (int o = 0; o < COUT; ++o) acc[pp][o] = pk2(0.f, 0.f);
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+            const int hi = ho + r - 1;
+            if (hi < 0 || hi >= H) continue;
+            const __nv_bfloat16* row = x + (int64_t(n) * H + hi) * W * C;
+            for (int c0 = lane * 8; c0 < C; c0 += 256) {
+                f32x2 xin[kConvPxOut + 2][4];
+#pragma unroll
+                for (int j = 0; j < kConvPxOut + 2; ++j) {
+                    const int wi = wo0 - 1 + j;
+                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                    if (wi >= 0 && wi < W) raw = __ldg(reinterpret_cast<const uint4*>(row + int64_t(wi) * C + c0));
+                    xin[j][0] = pk2(bf16_lo(raw.x), bf16_hi(raw.x));
+                    xin[j][1] = pk2(bf16_lo(raw.y), bf16_hi(raw.y));
+                    xin[j][2] = pk2(bf16_lo(raw.z), bf16_hi(raw.z));
+                    xin[j][3] = pk2(bf16_lo(raw.w), bf16_hi(raw.w));
+                }
+                const float* wbase = sw + (c0 & ~255) + lane * 4;
+#pragma unroll
+                for (int sx = 0; sx < 3; ++sx) {
+#pragma unroll
+                    for (int o = 0; o < COUT; ++o) {
+                        const float* wr = wbase + (o * 9 + r * 3 + sx) * C;
+                        const ulonglong2 w0 = *reinterpret_cast<const ulonglong2*>(wr);
+                        const ulonglong2 w1 = *reinterpret_cast<const ulonglong2*>(wr + hs);
+#pragma unroll
+                        for (int pp = 0; pp < kConvPxOut; ++pp)
+                            acc[pp][o] = fma2(xin[pp + sx][0], w0.x, fma2(xin[pp + sx][1], w0.y,
+                                         fma2(xin[pp + sx][2], w1.x, fma2(xin[pp + sx][3], w1.y, acc[pp][o]))));
+                    }
+                }
+            }
+        }
+        float red[kConvPxOut][COUT];
+#pragma unroll
+        for (int pp = 0; pp < kConvPxOut; ++pp)
+#pragma unroll
+            for (int o = 0; o < COUT; ++o) {
+                float a, b;
+                upk2(acc[pp][o], a, b);
+                red[pp][o] = a + b;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) red[pp][o] += __shfl_xor_sync(0xffffffffu, red[pp][o], off);
+            }
+        // lane pp * COUT + o writes output o of pixel pp
+#pragma unroll
+        for (int pp = 0; pp < kConvPxOut; ++pp)
+#pragma unroll
+            for (int o = 0; o < COUT; ++o)
+                if (lane == pp * COUT + o && wo0 + pp < W)
+                    out[((int64_t(n) * H + ho) * W + wo0 + pp) * COUT + o] = red[pp][o] + (bias != nullptr ? __ldg(bias + o) : 0.f);
+    }
+}
+
 inline int blocks_for(int64_t n, int threads) { return int((n + threads - 1) / threads); }
 
 }  // namespace
@@ -423,8 +596,21 @@ extern "C" hq_status hq_conv2d_direct(const void* x, hq_dtype xdt, const float* 
     if (smem > 160 * 1024) return HQ_ERR_UNSUPPORTED;
     const int64_t pixel_groups = Nb * Ho * ((Wo + 3) / 4);                    // a warp takes four pixels at a time
     const int grid = int(pixel_groups / 8 < 148 * 16 ? (pixel_groups + 7) / 8 : 148 * 16);
+    const bool same3x3 = R == 3 && stride == 1 && pad == 1;
+    const int64_t groups8 = Nb * Ho * ((Wo + 7) / 8);                          // the first 3x3 convolution: eight pixels per warp
+    const int grid8 = int(groups8 / 8 < 148 * 16 ? (groups8 + 7) / 8 : 148 * 16);
     if (ydt == HQ_BF16 && C <= 16 && Cout % 8 == 0) {                          // few input channels
         if (!aligned16(y)) return HQ_ERR_ALIGNMENT;
+        if (same3x3 && (C == 3 || C == 4) && (Cout <= 256 || Cout % 256 == 0)) {
+#define HQ_CIN_CASE(T, N)                                                                                           \
+            HQ_CUDA_OK(cudaFuncSetAttribute(conv3x3_small_cin_kernel<T, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
+            conv3x3_small_cin_kernel<T, N><<<grid8, 256, smem, st>>>(static_cast<const T*>(x), w, bias,              \
+                static_cast<__nv_bfloat16*>(y), int(Nb), int(H), int(W), int(Cout));
+            if (xdt == HQ_F32) { if (C == 3) { HQ_CIN_CASE(float, 3) } else { HQ_CIN_CASE(float, 4) } }
+            else { if (C == 3) { HQ_CIN_CASE(__nv_bfloat16, 3) } else { HQ_CIN_CASE(__nv_bfloat16, 4) } }
+#undef HQ_CIN_CASE
+            return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+        }
         if (xdt == HQ_F32) {
             HQ_CUDA_OK(cudaFuncSetAttribute(conv_small_cin_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
             conv_small_cin_kernel<float><<<grid, 256, smem, st>>>(static_cast<const float*>(x), w, bias,
@@ -438,6 +624,20 @@ extern "C" hq_status hq_conv2d_direct(const void* x, hq_dtype xdt, const float* 
     }
     if (ydt == HQ_F32 && xdt == HQ_BF16 && Cout <= 4 && C % 8 == 0) {          // few output channels
         if (!aligned16(x)) return HQ_ERR_ALIGNMENT;
+        if (same3x3 && (C <= 256 || C % 256 == 0)) {
+#define HQ_COUT3_CASE(N)                                                                                            \
+            case N:                                                                                                 \
+                HQ_CUDA_OK(cudaFuncSetAttribute(conv3x3_small_cout_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
+                conv3x3_small_cout_kernel<N><<<grid, 256, smem, st>>>(static_cast<const __nv_bfloat16*>(x), w, bias, \
+                    static_cast<float*>(y), int(Nb), int(H), int(W), int(C));                                       \
+                break;
+            switch (int(Cout)) {
+                HQ_COUT3_CASE(1) HQ_COUT3_CASE(2) HQ_COUT3_CASE(3) HQ_COUT3_CASE(4)
+                default: return HQ_ERR_UNSUPPORTED;
+            }
+#undef HQ_COUT3_CASE
+            return cudaGetLastError() == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+        }
 #define HQ_COUT_CASE(N)                                                                                             \
         case N:                                                                                                     \
             HQ_CUDA_OK(cudaFuncSetAttribute(conv_small_cout_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))); \
