@@ -41,7 +41,7 @@ typedef enum {
     HQ_OK = 0,
     HQ_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, unknown enum value */
     HQ_ERR_SHAPE = 2,         /* sizes that contradict each other (cols % had_block, K mismatch ...) */
-    HQ_ERR_UNSUPPORTED = 3,   /* legal request this build has no kernel for */
+    HQ_ERR_UNSUPPORTED = 3,   /* legal request the library has no kernel for */
     HQ_ERR_ALIGNMENT = 4,     /* pointer or pitch not aligned as stated above */
     HQ_ERR_WORKSPACE = 5,     /* workspace too small (ask hq_workspace_size) */
     HQ_ERR_OVERFLOW_RISK = 6, /* int32 accumulators could overflow for these bit-widths and K */
