@@ -256,6 +256,32 @@ hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, i
                            int32_t* dev_status, void* stream);
 
 
+/* ---- The same calls on the channel concatenation of two tensors, read in place (no counterpart in the paper's
+ * equations: the skip connections of the UNet join the up-sampling path by concatenation, and the concatenated tensor is
+ * consumed only by quantized layers, so it need never be written).  x holds channels / columns [0, C1) (pitch C1, for
+ * hq_hadamard_quant_cat ldx), x2 the channels [C1, C) (pitch C - C1, resp. ldx2); C1 must be a multiple of the Hadamard
+ * block (a block never straddles the two tensors) and of 8, both tensors 16-byte aligned.  Everything else as the call
+ * without `_cat`; the results are bit-identical to it applied to the written-out concatenation. */
+hq_status hq_hadamard_quant_cat(const void* x, int64_t ldx, const void* x2, int64_t ldx2, int64_t cols1, hq_dtype xdt,
+                                int64_t rows, int64_t cols, int had_block, int bits, hq_scale_mode mode,
+                                const float* static_scale, void* codes, hq_container cont, int64_t ld_codes, float* scales,
+                                void* stream);
+hq_status hq_gn_silu_quant_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W,
+                               int64_t C, int groups, const float* gamma, const float* beta, const void* pre_bias,
+                               float eps, int had_block, int bits, hq_scale_mode mode, const float* static_scale,
+                               void* codes, hq_container cont, int64_t ld_codes, float* scales, void* scratch,
+                               size_t scratch_bytes, void* stream);
+hq_status hq_gn_silu_qconv_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W,
+                               int64_t C, int groups, const float* gamma, const float* beta, const void* pre_bias,
+                               float eps, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                               const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                               const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                               void* scratch, size_t scratch_bytes, int32_t* dev_status, void* stream);
+hq_status hq_qconv_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                       const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                       const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode, const float* static_scale,
+                       void* y, hq_dtype ydt, void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* ---- Fused linear layer with GroupNorm (optionally + SiLU) in front, on the pixels of an NHWC tensor: the QKV
  * projection of an attention block (no counterpart in the paper's equations; the paper quantizes the projection, the
  * normalisation in front of it is the network's own).  Rows = Nb * rows_per_sample; statistics per (sample, group) over

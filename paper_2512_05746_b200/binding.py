@@ -27,7 +27,8 @@ EXPORTS = ["hq_version", "hq_status_string", "hq_check_status", "hq_hadamard_qua
            "hq_alpha_for", "hq_mma_i8_probe", "hq_qlinear_noalloc", "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant",
            "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv", "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast",
            "hq_class_embed_add", "hq_timestep_embedding", "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act",
-           "hq_conv2d_direct", "hq_attention", "hq_hadamard_quant_width2", "hq_qlinear_fused", "hq_set_pair_gemm", "hq_mma_i8_probe_pair"]
+           "hq_conv2d_direct", "hq_attention", "hq_hadamard_quant_width2", "hq_qlinear_fused", "hq_set_pair_gemm", "hq_mma_i8_probe_pair",
+           "hq_hadamard_quant_cat", "hq_gn_silu_quant_cat", "hq_gn_silu_qconv_cat", "hq_qconv_cat"]
 HQ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 
@@ -101,13 +102,21 @@ def _load():
     L.hq_conv2d_direct.argtypes = [p, i32, p, p, i64, i64, i64, i64, i64, i32, i32, i32, p, i32, p]
     L.hq_attention.argtypes = [p, i64, i64, i64, i32, p, p, p]
     L.hq_alpha_for.restype = C.c_float
+    L.hq_hadamard_quant_cat.argtypes = [p, i64, p, i64, i64, i32, i64, i64, i32, i32, i32, p, p, i32, i64, p, p]
+    L.hq_gn_silu_quant_cat.argtypes = [p, p, i64, i32, i64, i64, i64, i64, i32, p, p, p, C.c_float, i32, i32, i32, p, p, i32,
+                                       i64, p, p, C.c_size_t, p]
+    L.hq_gn_silu_qconv_cat.argtypes = [p, p, i64, i32, i64, i64, i64, i64, i32, p, p, p, C.c_float, C.POINTER(WeightDesc), p,
+                                       i32, i32, i32, i32, p, p, i32, i32, p, p, i32, p, C.c_size_t, p, C.c_size_t, p, p]
+    L.hq_qconv_cat.argtypes = [p, p, i64, i32, i64, i64, i64, i64, C.POINTER(WeightDesc), p, i32, i32, i32, i32, p, p, i32,
+                               i32, p, p, i32, p, C.c_size_t, p, p]
     L.hq_alpha_for.argtypes = [C.POINTER(WeightDesc)]
     L.hq_mma_i8_probe.argtypes = [i32, i32, p, p]
     for name in ("hq_check_status", "hq_hadamard_quant", "hq_weight_prepare", "hq_qgemm", "hq_qconv2d",
                  "hq_workspace_size", "hq_qlinear", "hq_qconv", "hq_mma_i8_probe", "hq_qlinear_noalloc",
                  "hq_hadamard_quant_width", "hq_qconv_width", "hq_gn_silu_quant", "hq_ln_quant", "hq_ln_qlinear", "hq_gn_silu_qconv",
                  "hq_gn_qlinear", "hq_silu", "hq_add", "hq_add_rows_bcast", "hq_class_embed_add", "hq_timestep_embedding",
-                 "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act", "hq_conv2d_direct", "hq_attention"):
+                 "hq_upsample_nearest2x", "hq_concat_channels", "hq_groupnorm_act", "hq_conv2d_direct", "hq_attention",
+                 "hq_hadamard_quant_cat", "hq_gn_silu_quant_cat", "hq_gn_silu_qconv_cat", "hq_qconv_cat"):
         getattr(L, name).restype = C.c_int
     return L
 
@@ -155,10 +164,16 @@ def hq_check_status(dev_status) -> None:
 
 
 def hq_hadamard_quant(x, had_block: int, bits: int, codes, container: int, scales=None, static_scale=None,
-                      stream=None) -> None:
-    """x [rows, cols] (fp32/bf16, last dim contiguous) -> codes (uint8 [rows, pitch]) and scales (fp32)."""
+                      stream=None, x2=None) -> None:
+    """x [rows, cols] (fp32/bf16, last dim contiguous) -> codes (uint8 [rows, pitch]) and scales (fp32).  With x2
+    [rows, cols2] the input is the column concatenation [x | x2], read in place."""
     rows, cols = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    if x2 is not None:
+        _check(lib.hq_hadamard_quant_cat(_dptr(x), x.stride(0), _dptr(x2), x2.stride(0), cols, _dtype_code(x), rows,
+                                         cols + x2.shape[1], had_block, bits, mode, _dptr(static_scale), _dptr(codes),
+                                         container, codes.stride(0), _dptr(scales), _stream(stream)), "hq_hadamard_quant_cat")
+        return
     _check(lib.hq_hadamard_quant(_dptr(x), _dtype_code(x), rows, cols, x.stride(0), had_block, bits, mode,
                                  _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
                                  _stream(stream)), "hq_hadamard_quant")
@@ -252,9 +267,17 @@ def hq_qlinear_noalloc(x, pw: PreparedWeight, bias, a_bits: int, y, static_scale
 
 
 def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias, a_bits: int, y, workspace,
-             static_scale=None, dev_status=None, stream=None) -> None:
+             static_scale=None, dev_status=None, stream=None, x2=None) -> None:
+    """The fused convolution layer on x NHWC, or (x2 given) on the channel concatenation [x | x2] read in place."""
     Nb, H, W, Cin = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    if x2 is not None:
+        _check(lib.hq_qconv_cat(_dptr(x), _dptr(x2), Cin, _dtype_code(x), Nb, H, W, Cin + x2.shape[3], C.byref(pw.desc),
+                                _dptr(pw.blob_dev), R, S, stride, pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode,
+                                _dptr(static_scale), _dptr(y), _dtype_code(y), _dptr(workspace),
+                                workspace.numel() * workspace.element_size(), _dptr(dev_status), _stream(stream)),
+               "hq_qconv_cat")
+        return
     _check(lib.hq_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride,
                         pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale), _dptr(y),
                         _dtype_code(y), _dptr(workspace), workspace.numel() * workspace.element_size(),
@@ -262,11 +285,18 @@ def hq_qconv(x, pw: PreparedWeight, R: int, S: int, stride: int, pad: int, bias,
 
 
 def hq_gn_silu_quant(x, groups: int, gamma, beta, eps: float, had_block: int, bits: int, codes, container: int,
-                     scratch, scales=None, static_scale=None, stream=None, pre_bias=None) -> None:
-    """GroupNorm(groups) + SiLU of x NHWC (of x + pre_bias[n, c] when a bf16 [Nb, C] addend is given), then transform
-    over channels + quantization into codes [Nb*H*W, pitch]."""
+                     scratch, scales=None, static_scale=None, stream=None, pre_bias=None, x2=None) -> None:
+    """GroupNorm(groups) + SiLU of x NHWC (of x + pre_bias[n, c] when a bf16 [Nb, C] addend is given; of the channel
+    concatenation [x | x2] when x2 is given), then transform over channels + quantization into codes [Nb*H*W, pitch]."""
     Nb, H, W, Cin = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    if x2 is not None:
+        _check(lib.hq_gn_silu_quant_cat(_dptr(x), _dptr(x2), Cin, _dtype_code(x), Nb, H, W, Cin + x2.shape[3], groups,
+                                        _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps, had_block, bits, mode,
+                                        _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
+                                        _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)),
+               "hq_gn_silu_quant_cat")
+        return
     _check(lib.hq_gn_silu_quant(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps, had_block,
                                 bits, mode, _dptr(static_scale), _dptr(codes), container, codes.stride(0), _dptr(scales),
                                 _dptr(scratch), scratch.numel() * scratch.element_size(), _stream(stream)),
@@ -275,11 +305,20 @@ def hq_gn_silu_quant(x, groups: int, gamma, beta, eps: float, had_block: int, bi
 
 def hq_gn_silu_qconv(x, groups: int, gamma, beta, eps: float, pw: PreparedWeight, R: int, S: int, stride: int, pad: int,
                      bias, a_bits: int, y, workspace, scratch, static_scale=None, dev_status=None, stream=None,
-                     pre_bias=None) -> None:
+                     pre_bias=None, x2=None) -> None:
     """The fused convolution layer with GroupNorm + SiLU in front (x NHWC; pre_bias: bf16 [Nb, C] added to x before the
-    normalisation, or None)."""
+    normalisation, or None; x2: the input is the channel concatenation [x | x2], read in place)."""
     Nb, H, W, Cin = x.shape
     mode = HQ_SCALE_PER_ROW if static_scale is None else HQ_SCALE_STATIC
+    if x2 is not None:
+        _check(lib.hq_gn_silu_qconv_cat(_dptr(x), _dptr(x2), Cin, _dtype_code(x), Nb, H, W, Cin + x2.shape[3], groups,
+                                        _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps, C.byref(pw.desc), _dptr(pw.blob_dev),
+                                        R, S, stride, pad, _dptr(pw.s_w_dev), _dptr(bias), a_bits, mode, _dptr(static_scale),
+                                        _dptr(y), _dtype_code(y), _dptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _dptr(scratch),
+                                        scratch.numel() * scratch.element_size(), _dptr(dev_status), _stream(stream)),
+               "hq_gn_silu_qconv_cat")
+        return
     _check(lib.hq_gn_silu_qconv(_dptr(x), _dtype_code(x), Nb, H, W, Cin, groups, _dptr(gamma), _dptr(beta), _dptr(pre_bias), eps,
                                 C.byref(pw.desc), _dptr(pw.blob_dev), R, S, stride, pad, _dptr(pw.s_w_dev), _dptr(bias),
                                 a_bits, mode, _dptr(static_scale), _dptr(y), _dtype_code(y), _dptr(workspace),

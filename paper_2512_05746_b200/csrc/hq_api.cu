@@ -26,7 +26,11 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
                                const float* gamma, const float* beta, float eps, int had_block, int bits,
                                hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                                int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
-                               int silu, const void* pre_bias);
+                               int silu, const void* pre_bias, const void* x2, int64_t split);
+hq_status launch_hadamard_quant_cat(const void* x, int64_t ldx, const void* x2, int64_t ldx2, int64_t split, hq_dtype xdt,
+                                    int64_t rows, int64_t cols, int had_block, int bits, hq_scale_mode mode,
+                                    const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
+                                    float* scales, cudaStream_t st);
 hq_status launch_ln_quant(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, const float* weight,
                           const float* bias, int64_t rows_per_group, float eps, int had_block, int bits,
                           hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
@@ -127,7 +131,8 @@ extern "C" hq_status hq_ln_qlinear(const void* x, hq_dtype xdt, int64_t M, int64
                         y, ydt, ldy, dev_status, st, true);
 }
 
-extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+static hq_status gn_silu_qconv_impl(const void* x, const void* x2, int64_t split, hq_dtype xdt, int64_t Nb, int64_t H,
+                                    int64_t W, int64_t C, int groups,
                                       const float* gamma, const float* beta, const void* pre_bias, float eps,
                                       const hq_weight_desc* desc,
                                       const void* w_dev, int R, int S, int stride, int pad, const float* scale_w,
@@ -149,10 +154,36 @@ extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, i
     unsigned char* codes = static_cast<unsigned char*>(workspace);
     float* scales = reinterpret_cast<float*>(codes + scales_offset(rows, C, cont));
     s = launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, desc->had_block, a_bits, mode, static_scale, codes,
-                             cont, ldc, scales, scratch, scratch_bytes, st, 1, pre_bias);
+                             cont, ldc, scales, scratch, scratch_bytes, st, 1, pre_bias, x2, split);
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st, true);
+}
+
+extern "C" hq_status hq_gn_silu_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C, int groups,
+                                      const float* gamma, const float* beta, const void* pre_bias, float eps,
+                                      const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                                      const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                                      const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                                      void* scratch, size_t scratch_bytes, int32_t* dev_status, void* stream) {
+    return gn_silu_qconv_impl(x, nullptr, 0, xdt, Nb, H, W, C, groups, gamma, beta, pre_bias, eps, desc, w_dev, R, S, stride,
+                              pad, scale_w, bias, a_bits, mode, static_scale, y, ydt, workspace, ws_bytes, scratch,
+                              scratch_bytes, dev_status, stream);
+}
+
+// The same layer on the channel concatenation of two NHWC tensors (x: channels [0, C1), x2: channels [C1, C)), read in
+// place: a skip connection joined to the up-sampling path without the concatenated tensor being written.
+extern "C" hq_status hq_gn_silu_qconv_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H,
+                                          int64_t W, int64_t C, int groups, const float* gamma, const float* beta,
+                                          const void* pre_bias, float eps, const hq_weight_desc* desc, const void* w_dev,
+                                          int R, int S, int stride, int pad, const float* scale_w, const float* bias,
+                                          int a_bits, hq_scale_mode mode, const float* static_scale, void* y, hq_dtype ydt,
+                                          void* workspace, size_t ws_bytes, void* scratch, size_t scratch_bytes,
+                                          int32_t* dev_status, void* stream) {
+    if (x2 == nullptr) return HQ_ERR_INVALID_ARG;
+    return gn_silu_qconv_impl(x, x2, C1, xdt, Nb, H, W, C, groups, gamma, beta, pre_bias, eps, desc, w_dev, R, S, stride, pad,
+                              scale_w, bias, a_bits, mode, static_scale, y, ydt, workspace, ws_bytes, scratch, scratch_bytes,
+                              dev_status, stream);
 }
 
 // The fused linear layer on the pixels of an NHWC tensor with GroupNorm (optionally + SiLU) in front: the QKV
@@ -178,13 +209,14 @@ extern "C" hq_status hq_gn_qlinear(const void* x, hq_dtype xdt, int64_t Nb, int6
     const int64_t ldc = code_pitch(C, cont);
     s = launch_gn_silu_quant(x, xdt, Nb, rows_per_sample, 1, C, groups, gamma, beta, eps, desc->had_block, a_bits,
                              HQ_SCALE_PER_ROW, nullptr, codes, cont, ldc, scales, scratch, scratch_bytes, st, silu != 0,
-                             nullptr);
+                             nullptr, nullptr, 0);
     if (s != HQ_OK) return s;
     return launch_qgemm(codes, cont, a_bits, M, C, ldc, desc, w_dev, scales, 0, scale_w, bias, hq_alpha_for(desc), nullptr,
                         y, ydt, ldy, dev_status, st, true);
 }
 
-extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+static hq_status qconv_impl(const void* x, const void* x2, int64_t split, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W,
+                            int64_t C,
                               const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
                               const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
                               const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
@@ -203,10 +235,34 @@ extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char* codes = static_cast<unsigned char*>(workspace);
     float* scales = reinterpret_cast<float*>(codes + scales_offset(rows, C, cont));
-    s = launch_hadamard_quant(x, xdt, rows, C, C, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
+    if (x2 != nullptr)
+        s = launch_hadamard_quant_cat(x, split, x2, C - split, split, xdt, rows, C, desc->had_block, a_bits, mode, static_scale,
+                                      codes, cont, ldc, scales, st);
+    else
+        s = launch_hadamard_quant(x, xdt, rows, C, C, desc->had_block, a_bits, mode, static_scale, codes, cont, ldc, scales, st);
     if (s != HQ_OK) return s;
     return launch_qconv2d(codes, cont, a_bits, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scales,
                           mode == HQ_SCALE_STATIC, scale_w, bias, hq_alpha_for(desc), nullptr, y, ydt, dev_status, st, true);
+}
+
+extern "C" hq_status hq_qconv(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,
+                              const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride, int pad,
+                              const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                              const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                              int32_t* dev_status, void* stream) {
+    return qconv_impl(x, nullptr, 0, xdt, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale_w, bias, a_bits, mode,
+                      static_scale, y, ydt, workspace, ws_bytes, dev_status, stream);
+}
+
+// The fused convolution layer on the channel concatenation of two NHWC tensors read in place (see hq_gn_silu_qconv_cat).
+extern "C" hq_status hq_qconv_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W,
+                                  int64_t C, const hq_weight_desc* desc, const void* w_dev, int R, int S, int stride,
+                                  int pad, const float* scale_w, const float* bias, int a_bits, hq_scale_mode mode,
+                                  const float* static_scale, void* y, hq_dtype ydt, void* workspace, size_t ws_bytes,
+                                  int32_t* dev_status, void* stream) {
+    if (x2 == nullptr) return HQ_ERR_INVALID_ARG;
+    return qconv_impl(x, x2, C1, xdt, Nb, H, W, C, desc, w_dev, R, S, stride, pad, scale_w, bias, a_bits, mode, static_scale,
+                      y, ydt, workspace, ws_bytes, dev_status, stream);
 }
 
 // Convolution exactly as Eq. 13-14 state it: transform along the width axis, quantization with one static scale,

@@ -13,7 +13,7 @@ namespace hq {
 // followed by [samples][groups][2] floats (mean, 1/sqrt(var + eps)).
 hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
                           void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st,
-                          const void* pre_bias);
+                          const void* pre_bias, const void* x2, int64_t split);
 
 namespace {
 
@@ -568,7 +568,7 @@ extern "C" hq_status hq_groupnorm_act(const void* x, int64_t Nb, int64_t H, int6
     if (!aligned16(x) || !aligned16(out) || C % 8 != 0) return HQ_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float* stats = nullptr;
-    hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st, nullptr);
+    hq_status s = launch_gn_stats(x, HQ_BF16, Nb, H * W, C, groups, eps, scratch, scratch_bytes, &stats, st, nullptr, nullptr, 0);
     if (s != HQ_OK) return s;
     if (Nb > 65535) return HQ_ERR_UNSUPPORTED;
     const int c8 = int(C / 8);

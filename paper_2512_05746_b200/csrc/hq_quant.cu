@@ -26,6 +26,10 @@ namespace {
 struct QuantParams {
     const void* x;
     int64_t rows, cols, ldx;
+    // optional second source: columns [split, cols) of every row come from x2 (pitch ldx2), columns [0, split) from x --
+    // the channel concatenation of two tensors read in place (split is a multiple of the Hadamard block)
+    const void* x2;
+    int64_t split, ldx2;
     int m;               // Hadamard blocks per row
     int rows_per_cta;
     int threads_per_row;
@@ -141,7 +145,10 @@ __global__ void __launch_bounds__(320) fwht_quant_fast(const QuantParams p) {
     const bool valid = row < p.rows;                   // rows past the end work on row 0's values and store nothing
     Raw cur[E / 4];
     {
-        const InT* src = reinterpret_cast<const InT*>(p.x) + (valid ? row : 0) * p.ldx + int64_t(blk) * N;
+        const int64_t c0 = int64_t(blk) * N, r = valid ? row : 0;
+        const InT* src = (p.x2 != nullptr && c0 >= p.split)
+                             ? reinterpret_cast<const InT*>(p.x2) + r * p.ldx2 + (c0 - p.split)
+                             : reinterpret_cast<const InT*>(p.x) + r * p.ldx + c0;
 #pragma unroll
         for (int i = 0; i < E / 4; ++i) cur[i] = __ldcs(reinterpret_cast<const Raw*>(src + 4 * (tb + TB * i)));
     }
@@ -547,9 +554,10 @@ __device__ __forceinline__ void gn_quad(const GnPiece<8>& r, int q, f32x2& lo, f
 }
 
 template <typename InT, int VEC>
-__global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, const __nv_bfloat16* pre_bias, int64_t hw,
-                                                          int64_t total_px, int64_t span, int C, int groups, double* sums,
-                                                          float* stats, double inv_count, double eps) {
+__global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, const InT* x2, int split,
+                                                          const __nv_bfloat16* pre_bias, int64_t hw, int64_t total_px,
+                                                          int64_t span, int C, int groups, double* sums, float* stats,
+                                                          double inv_count, double eps) {
     constexpr int Q = VEC / 4;                         // channel quads per piece
     constexpr int U = 8;                               // loads in flight per thread
     __shared__ double red[2 * Q][256];
@@ -582,12 +590,16 @@ __global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, const __
                         e_hi[q] = pk2(__uint_as_float(er.y << 16), __uint_as_float(er.y & 0xFFFF0000u));
                     }
                 }
-                const InT* src = x + int64_t(col) * VEC;
+                // channels [split, C) of a pixel come from the second tensor when there is one (a piece lies in one of them)
+                const int ch = col * VEC;
+                const bool second = x2 != nullptr && ch >= split;
+                const InT* src = second ? x2 + (ch - split) : x + ch;
+                const int64_t pitch = x2 == nullptr ? C : (second ? C - split : split);
                 int64_t px = r0 + pl;
                 for (; px + (U - 1) * ppl < seg_end; px += U * ppl) {
                     GnPiece<VEC> raw[U];
 #pragma unroll
-                    for (int u = 0; u < U; ++u) raw[u] = gn_load(src + (px + u * ppl) * C, static_cast<GnPiece<VEC>*>(nullptr));
+                    for (int u = 0; u < U; ++u) raw[u] = gn_load(src + (px + u * ppl) * pitch, static_cast<GnPiece<VEC>*>(nullptr));
 #pragma unroll
                     for (int q = 0; q < Q; ++q) {
                         f32x2 a = pk2(0.f, 0.f), b = pk2(0.f, 0.f);
@@ -608,7 +620,7 @@ __global__ void __launch_bounds__(256, 4) gn_stats_kernel(const InT* x, const __
                     }
                 }
                 for (; px < seg_end; px += ppl) {
-                    const GnPiece<VEC> raw = gn_load(src + px * C, static_cast<GnPiece<VEC>*>(nullptr));
+                    const GnPiece<VEC> raw = gn_load(src + px * pitch, static_cast<GnPiece<VEC>*>(nullptr));
 #pragma unroll
                     for (int q = 0; q < Q; ++q) {
                         f32x2 lo, hi;
@@ -722,10 +734,12 @@ struct GnArgs { const float* stats; const float* gamma; const float* beta; int g
                 const __nv_bfloat16* pre_bias; };
 struct LnArgs { const float* w; const float* b; int64_t rows_per_group; float eps; };
 
+struct SplitArgs { const void* x2; int64_t split, ldx2; };
+
 static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, int64_t cols, int64_t ldx, int had_block,
                                    int bits, hq_scale_mode mode, const float* static_scale, void* codes,
                                    hq_container cont, int64_t ld_codes, float* scales, const GnArgs* gn,
-                                   cudaStream_t st, const LnArgs* ln = nullptr) {
+                                   cudaStream_t st, const LnArgs* ln = nullptr, const SplitArgs* sp = nullptr) {
     if (rows == 0 && cols > 0) return HQ_OK;                       // nothing to do; pointers may be NULL
     if (x == nullptr || codes == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
@@ -734,7 +748,7 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
     if (mode == HQ_SCALE_STATIC && static_scale == nullptr) return HQ_ERR_INVALID_ARG;
     if (mode == HQ_SCALE_PER_ROW && scales == nullptr) return HQ_ERR_INVALID_ARG;
     if (bits != 3 && bits != 4 && bits != 8) return HQ_ERR_INVALID_ARG;
-    if (rows < 0 || cols <= 0 || ldx < cols) return HQ_ERR_SHAPE;
+    if (rows < 0 || cols <= 0 || ldx < ((sp != nullptr && sp->x2 != nullptr) ? sp->split : cols)) return HQ_ERR_SHAPE;
     if (cont == HQ_CODES_NIBBLE && (bits > 4 || (cols & 1))) return HQ_ERR_SHAPE;
     const int64_t row_bytes = cont == HQ_CODES_NIBBLE ? cols / 2 : cols;
     if (ld_codes < row_bytes) return HQ_ERR_SHAPE;
@@ -744,6 +758,13 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
 
     QuantParams p{};
     p.x = x; p.rows = rows; p.cols = cols; p.ldx = ldx;
+    if (sp != nullptr && sp->x2 != nullptr) {
+        // the two-source form exists in the fast kernel only; a Hadamard block never straddles the two tensors
+        if (sp->split <= 0 || sp->split >= cols || sp->split % n != 0 || sp->ldx2 < cols - sp->split || ldx < sp->split)
+            return HQ_ERR_SHAPE;
+        if (reinterpret_cast<uintptr_t>(sp->x2) % (4 * (xdt == HQ_F32 ? 4 : 2)) != 0 || sp->ldx2 % 4 != 0) return HQ_ERR_ALIGNMENT;
+        p.x2 = sp->x2; p.split = sp->split; p.ldx2 = sp->ldx2;
+    }
     p.m = int(cols / n);
     p.bits = bits;
     p.norm = float(exp2(-0.5 * double(klog)));
@@ -797,7 +818,7 @@ static hq_status launch_quant_impl(const void* x, hq_dtype xdt, int64_t rows, in
         return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
         }
     }
-    if (gn != nullptr || ln != nullptr) return HQ_ERR_UNSUPPORTED;   // the prologues exist in the fast kernel only
+    if (gn != nullptr || ln != nullptr || p.x2 != nullptr) return HQ_ERR_UNSUPPORTED;   // these exist in the fast kernel only
     const size_t smem = size_t(cols) * 4;
     if (smem > 200 * 1024) return HQ_ERR_UNSUPPORTED;
     const int grid = int(rows < 148 * 8 ? rows : 148 * 8);
@@ -824,11 +845,22 @@ hq_status launch_hadamard_quant(const void* x, hq_dtype xdt, int64_t rows, int64
                              nullptr, st);
 }
 
+// The same on the column concatenation [x | x2] of two matrices read in place: x holds columns [0, split), x2 the rest.
+hq_status launch_hadamard_quant_cat(const void* x, int64_t ldx, const void* x2, int64_t ldx2, int64_t split, hq_dtype xdt,
+                                    int64_t rows, int64_t cols, int had_block, int bits, hq_scale_mode mode,
+                                    const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
+                                    float* scales, cudaStream_t st) {
+    if (x2 == nullptr) return HQ_ERR_INVALID_ARG;
+    const SplitArgs sp{x2, split, ldx2};
+    return launch_quant_impl(x, xdt, rows, cols, ldx, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales,
+                             nullptr, st, nullptr, &sp);
+}
+
 // GroupNorm statistics of an NHWC tensor (hw pixels per sample): fp64 sums per (sample, group) in `scratch` (cleared
 // here), then mean and 1/sqrt(var + eps) as floats behind them.  scratch: Nb * groups * (2 doubles + 2 floats).
 hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, int64_t C, int groups, float eps,
                           void* scratch, size_t scratch_bytes, const float** stats_out, cudaStream_t st,
-                          const void* pre_bias) {
+                          const void* pre_bias, const void* x2, int64_t split) {
     if (x == nullptr || scratch == nullptr) return HQ_ERR_INVALID_ARG;
     if (xdt != HQ_F32 && xdt != HQ_BF16) return HQ_ERR_INVALID_ARG;
     if (Nb <= 0 || hw <= 0 || C <= 0 || groups <= 0) return HQ_ERR_SHAPE;
@@ -846,6 +878,10 @@ hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, i
     HQ_CUDA_OK(cudaMemsetAsync(scratch, 0, need, st));             // the sums and the ticket counters
     if (hw > 0x7fffffff) return HQ_ERR_UNSUPPORTED;                // the tickets count pixels in 32 bits
     // 16-byte pieces (bf16: eight channels) where the shape allows them
+    if (x2 != nullptr) {                                           // channels [split, C) of every pixel live in x2
+        if (split <= 0 || split >= C || split % 8 != 0 || (C - split) % 8 != 0) return HQ_ERR_SHAPE;
+        if (reinterpret_cast<uintptr_t>(x2) % 16 != 0 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return HQ_ERR_ALIGNMENT;
+    }
     const bool wide = xdt == HQ_BF16 && C % 8 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0;
     const int64_t pieces = C / (wide ? 8 : 4);
     const int64_t ppl = pieces < 256 ? 256 / pieces : 1;
@@ -859,13 +895,13 @@ hq_status launch_gn_stats(const void* x, hq_dtype xdt, int64_t Nb, int64_t hw, i
     const double inv_count = 1.0 / (double(hw) * double(C / groups));
     const unsigned grid = unsigned(ctas);
     if (xdt == HQ_F32)
-        gn_stats_kernel<float, 4><<<grid, 256, 0, st>>>(static_cast<const float*>(x), pre, hw, total_px, span, int(C), groups, sums,
+        gn_stats_kernel<float, 4><<<grid, 256, 0, st>>>(static_cast<const float*>(x), static_cast<const float*>(x2), int(split), pre, hw, total_px, span, int(C), groups, sums,
                                                        stats, inv_count, double(eps));
     else if (wide)
-        gn_stats_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), pre, hw, total_px, span, int(C),
+        gn_stats_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(x2), int(split), pre, hw, total_px, span, int(C),
                                                                groups, sums, stats, inv_count, double(eps));
     else
-        gn_stats_kernel<__nv_bfloat16, 4><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), pre, hw, total_px, span, int(C),
+        gn_stats_kernel<__nv_bfloat16, 4><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(x2), int(split), pre, hw, total_px, span, int(C),
                                                                groups, sums, stats, inv_count, double(eps));
     if (cudaGetLastError() != cudaSuccess) return HQ_ERR_CUDA;
     *stats_out = stats;
@@ -878,14 +914,19 @@ hq_status launch_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, int64_t 
                                const float* gamma, const float* beta, float eps, int had_block, int bits,
                                hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
                                int64_t ld_codes, float* scales, void* scratch, size_t scratch_bytes, cudaStream_t st,
-                               int silu, const void* pre_bias) {
+                               int silu, const void* pre_bias, const void* x2, int64_t split) {
     if (gamma == nullptr || beta == nullptr) return HQ_ERR_INVALID_ARG;
     if (H <= 0 || W <= 0) return HQ_ERR_SHAPE;
     const int64_t hw = H * W;
     const float* stats = nullptr;
-    hq_status s = launch_gn_stats(x, xdt, Nb, hw, C, groups, eps, scratch, scratch_bytes, &stats, st, pre_bias);
+    hq_status s = launch_gn_stats(x, xdt, Nb, hw, C, groups, eps, scratch, scratch_bytes, &stats, st, pre_bias, x2, split);
     if (s != HQ_OK) return s;
     const GnArgs gn{stats, gamma, beta, groups, hw, silu, static_cast<const __nv_bfloat16*>(pre_bias)};
+    if (x2 != nullptr) {
+        const SplitArgs sp{x2, split, C - split};
+        return launch_quant_impl(x, xdt, Nb * hw, C, split, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales,
+                                 &gn, st, nullptr, &sp);
+    }
     return launch_quant_impl(x, xdt, Nb * hw, C, C, had_block, bits, mode, static_scale, codes, cont, ld_codes, scales, &gn,
                              st);
 }
@@ -996,7 +1037,26 @@ extern "C" hq_status hq_gn_silu_quant(const void* x, hq_dtype xdt, int64_t Nb, i
                                       size_t scratch_bytes, void* stream) {
     return hq::launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, had_block, bits, mode, static_scale, codes,
                                     cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream), 1,
-                                    pre_bias);
+                                    pre_bias, nullptr, 0);
+}
+
+extern "C" hq_status hq_gn_silu_quant_cat(const void* x, const void* x2, int64_t C1, hq_dtype xdt, int64_t Nb, int64_t H,
+                                          int64_t W, int64_t C, int groups, const float* gamma, const float* beta,
+                                          const void* pre_bias, float eps, int had_block, int bits, hq_scale_mode mode,
+                                          const float* static_scale, void* codes, hq_container cont, int64_t ld_codes,
+                                          float* scales, void* scratch, size_t scratch_bytes, void* stream) {
+    if (x2 == nullptr) return HQ_ERR_INVALID_ARG;
+    return hq::launch_gn_silu_quant(x, xdt, Nb, H, W, C, groups, gamma, beta, eps, had_block, bits, mode, static_scale, codes,
+                                    cont, ld_codes, scales, scratch, scratch_bytes, static_cast<cudaStream_t>(stream), 1,
+                                    pre_bias, x2, C1);
+}
+
+extern "C" hq_status hq_hadamard_quant_cat(const void* x, int64_t ldx, const void* x2, int64_t ldx2, int64_t cols1,
+                                           hq_dtype xdt, int64_t rows, int64_t cols, int had_block, int bits,
+                                           hq_scale_mode mode, const float* static_scale, void* codes, hq_container cont,
+                                           int64_t ld_codes, float* scales, void* stream) {
+    return hq::launch_hadamard_quant_cat(x, ldx, x2, ldx2, cols1, xdt, rows, cols, had_block, bits, mode, static_scale, codes,
+                                         cont, ld_codes, scales, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" hq_status hq_hadamard_quant_width(const void* x, hq_dtype xdt, int64_t Nb, int64_t H, int64_t W, int64_t C,

@@ -156,9 +156,11 @@ class UNet:
         return self.ws[: rows * pitch].view(rows, pitch), self.ws[off: off + rows * 4].view(self.torch.float32)
 
     # ------------------------------------------------------------------ layers
-    def _conv3(self, name, x, norm=None, stride=1, pre_bias=None):
+    def _conv3(self, name, x, norm=None, stride=1, pre_bias=None, x2=None):
+        """x2: the layer's input is the channel concatenation [x | x2], which is read in place and never written."""
         hq, t = self.hq, self.torch
         Nb, H, W, Cin = x.shape
+        Cin += x2.shape[3] if x2 is not None else 0
         pw = self.pw[name]
         self._need_ws(Nb * H * W, Cin)
         y = self._new((Nb, H // stride, W // stride, pw.desc.N))
@@ -173,32 +175,36 @@ class UNet:
             codes, sc = self._ws_views(Nb * H * W, Cin)
             if g:
                 hq.hq_gn_silu_quant(x, G, g[0], g[1], self.EPS, pw.desc.had_block, self.a_bits, codes, self.cont, self.scratch,
-                                    scales=sc, pre_bias=pre_bias)
+                                    scales=sc, pre_bias=pre_bias, x2=x2)
             else:
-                hq.hq_hadamard_quant(x.view(-1, Cin), pw.desc.had_block, self.a_bits, codes, self.cont, scales=sc)
+                hq.hq_hadamard_quant(x.view(-1, x.shape[3]), pw.desc.had_block, self.a_bits, codes, self.cont, scales=sc,
+                                     x2=None if x2 is None else x2.view(-1, x2.shape[3]))
             ss.copy_(sc.max().reshape(1))
 
         def run():
             calibrate()
             if g:
                 hq.hq_gn_silu_qconv(x, G, g[0], g[1], self.EPS, pw, 3, 3, stride, 1, bias, self.a_bits, y, self.ws, self.scratch,
-                                    static_scale=ss, dev_status=self.status, pre_bias=pre_bias)
+                                    static_scale=ss, dev_status=self.status, pre_bias=pre_bias, x2=x2)
             else:
-                hq.hq_qconv(x, pw, 3, 3, stride, 1, bias, self.a_bits, y, self.ws, static_scale=ss, dev_status=self.status)
+                hq.hq_qconv(x, pw, 3, 3, stride, 1, bias, self.a_bits, y, self.ws, static_scale=ss, dev_status=self.status,
+                            x2=x2)
 
-        self._emit("q", name, run, lambda: dict(op="conv3", x=x, y=y, norm=norm, stride=stride, static=ss, pre_bias=pre_bias,
+        self._emit("q", name, run, lambda: dict(op="conv3", x=x, x2=x2, y=y, norm=norm, stride=stride, static=ss, pre_bias=pre_bias,
                                                 codes=self._ws_views(Nb * H * W, Cin)[0]))
         return y
 
-    def _conv1(self, name, x):
+    def _conv1(self, name, x, x2=None):
         hq = self.hq
         Nb, H, W, Cin = x.shape
+        Cin += x2.shape[3] if x2 is not None else 0
         pw = self.pw[name]
         self._need_ws(Nb * H * W, Cin)
         y = self._new((Nb, H, W, pw.desc.N))
         bias = self.f32[name + ".b"]
-        self._emit("q", name, lambda: hq.hq_qconv(x, pw, 1, 1, 1, 0, bias, self.a_bits, y, self.ws, dev_status=self.status),
-                   lambda: dict(op="conv1", x=x, y=y, codes=self._ws_views(Nb * H * W, Cin)[0],
+        self._emit("q", name, lambda: hq.hq_qconv(x, pw, 1, 1, 1, 0, bias, self.a_bits, y, self.ws, dev_status=self.status,
+                                                      x2=x2),
+                   lambda: dict(op="conv1", x=x, x2=x2, y=y, codes=self._ws_views(Nb * H * W, Cin)[0],
                                 scales=self._ws_views(Nb * H * W, Cin)[1]))
         return y
 
@@ -222,14 +228,17 @@ class UNet:
     def _glue(self, name, op, fn, **tensors):
         self._emit("g", name, fn, lambda: dict(op=op, **tensors))
 
-    def _resblock(self, name, x, semb):
+    def _resblock(self, name, x, semb, x2=None):
+        """x2: the block's input is the channel concatenation [x | x2] (a skip connection joining the up-sampling path);
+        its two consumers, the first convolution and the 1x1 skip convolution, read the two tensors in place."""
         hq = self.hq
-        cin, cout = x.shape[-1], self.pw[name + ".conv1"].desc.N
-        h = self._conv3(name + ".conv1", x, norm=name + ".norm1")
+        cin, cout = x.shape[-1] + (x2.shape[-1] if x2 is not None else 0), self.pw[name + ".conv1"].desc.N
+        h = self._conv3(name + ".conv1", x, norm=name + ".norm1", x2=x2)
         e = self._linear(name + ".emb", semb)
         # h + e is never stored: the second convolution's normalisation takes the embedding as a per-sample addend
         h2 = self._conv3(name + ".conv2", h, norm=name + ".norm2", pre_bias=e)
-        xs = x if cin == cout else self._conv1(name + ".skip", x)
+        assert x2 is None or cin != cout       # a concatenated input always changes the channel count here
+        xs = x if cin == cout else self._conv1(name + ".skip", x, x2=x2)
         out = self._new(h2.shape)
         self._glue(name + ".residual", "add", lambda: hq.hq_add(xs, h2, out), a=xs, b=h2, out=out)
         return out
@@ -298,10 +307,7 @@ class UNet:
         for lvl in reversed(range(len(mults))):
             for b in range(nres + 1):
                 sk = skips.pop()
-                cat = self._new(h.shape[:3] + (h.shape[3] + sk.shape[3],))
-                self._glue(f"up{lvl}.res{b}.concat", "concat", (lambda a=h, bb=sk, o=cat: hq.hq_concat_channels(a, bb, o)),
-                           a=h, b=sk, out=cat)
-                h = self._resblock(f"up{lvl}.res{b}", cat, semb)
+                h = self._resblock(f"up{lvl}.res{b}", h, semb, x2=sk)         # [h | skip], never written out
                 if res in cfg["attn_resolutions"]:
                     h = self._attention(f"up{lvl}.attn{b}", h)
             if lvl > 0:

@@ -108,6 +108,43 @@ def test_gn_silu_quant_with_a_per_sample_addend(env, oracle, Nb, H, W, C, G, n, 
     assert (unpack_nibbles_np(codes.cpu().numpy()) != q_ref).mean() > 0.2
 
 
+@pytest.mark.parametrize("Nb,H,W,c1,c2,G,n,pre", [(3, 8, 8, 256, 512, 32, 256, False), (2, 8, 8, 128, 128, 32, 128, True),
+                                                  (5, 4, 8, 512, 256, 32, 256, True)])
+def test_gn_silu_quant_of_a_concatenation_read_in_place(env, oracle, Nb, H, W, c1, c2, G, n, pre):
+    """GroupNorm + SiLU + transform + quantize of [x | x2] without the concatenation being written: the groups' statistics
+    run over both tensors (a group may lie in either), codes and scales as the oracle's on the concatenated tensor and
+    bit-identical to the call on the written-out concatenation."""
+    torch, hq = env
+    C = c1 + c2
+    a = inputs.activations((Nb, H, W, c1), outlier_count=2, outlier_scale=8.0, seed=c1) + np.float32(0.3)
+    b = inputs.activations((Nb, H, W, c2), outlier_count=1, outlier_scale=4.0, seed=c2 + 3) * np.float32(2.0) - np.float32(0.5)
+    ta, tb = torch.from_numpy(a).cuda().to(torch.bfloat16), torch.from_numpy(b).cuda().to(torch.bfloat16)
+    cat = torch.cat([ta, tb], dim=3).contiguous()
+    x = cat.float().cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(C)
+    gamma = (1.0 + 0.2 * rng.standard_normal(C)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(C)).astype(np.float32)
+    et = torch.from_numpy(inputs.activations((Nb, C), seed=9)).cuda().to(torch.bfloat16) if pre else None
+    if pre:
+        x = x + et.float().cpu().numpy().astype(np.float64)[:, None, None, :]
+    rows = Nb * H * W
+    out = []
+    for two in (True, False):
+        codes = torch.zeros((rows, C // 2), dtype=torch.uint8, device="cuda")
+        scales = torch.zeros((rows,), dtype=torch.float32, device="cuda")
+        scratch = torch.empty((Nb * G * 24,), dtype=torch.uint8, device="cuda")
+        hq.hq_gn_silu_quant(ta if two else cat, G, torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), 1e-5, n, 4,
+                            codes, hq.HQ_CODES_NIBBLE, scratch, scales=scales, pre_bias=et, x2=tb if two else None)
+        torch.cuda.synchronize()
+        out.append((codes.cpu().numpy(), scales.cpu().numpy()))
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    u = oracle.transform(oracle.groupnorm_silu(x, G, gamma, beta, 1e-5).reshape(rows, C), n)
+    q_ref, s_ref, v = oracle.quantize(u, 4, want_v=True)
+    assert float(np.abs(out[0][1] / s_ref - 1.0).max()) <= GN_SCALE_RTOL
+    check_codes(unpack_nibbles_np(out[0][0]), q_ref, v, f"groupnorm prologue on a concatenation {Nb}x{H}x{W}x({c1}+{c2})",
+                tie_rel=GN_TIE_REL, mismatch_frac=GN_MISMATCH_FRAC)
+
+
 def test_gn_silu_quant_on_an_input_aligned_to_8_bytes_only(env, oracle):
     """A bf16 tensor that starts 8 bytes into an allocation: the statistics pass then reads four channels per load."""
     torch, hq = env

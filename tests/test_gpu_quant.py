@@ -171,3 +171,51 @@ def test_quant_full_size_sampled_rows(env, oracle):
     # properties that hold for every row: codes in range, each row reaches +-qmax
     assert q.min() >= -7 and q.max() <= 7
     assert np.all(np.abs(q).max(axis=1) == 7)
+
+
+@pytest.mark.parametrize("rows,c1,c2,had_block,dt,static", [
+    (300, 256, 512, 256, "bf16", False),        # [h | skip] of the up-sampling path: the blocks of a row come from two tensors
+    (130, 128, 128, 128, "f32", True),
+    (64, 1024, 768, 256, "bf16", False),
+])
+def test_quant_of_a_concatenation_read_in_place(env, oracle, rows, c1, c2, had_block, dt, static):
+    """hq_hadamard_quant with a second source: codes and scales are those of the oracle on the concatenated matrix, and
+    bit-identical to the call on the written-out concatenation."""
+    torch, hq = env
+    a = inputs.activations((rows, c1), outlier_count=2, outlier_scale=10.0, seed=c1)
+    b = inputs.activations((rows, c2), outlier_count=1, outlier_scale=5.0, seed=c2 + 1) * np.float32(0.5)
+    ta, tb = torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda()
+    if dt == "bf16":
+        ta, tb = ta.to(torch.bfloat16), tb.to(torch.bfloat16)
+    cat = torch.cat([ta, tb], dim=1).contiguous()
+    x = cat.float().cpu().numpy()
+    cols = c1 + c2
+    ss = torch.tensor([0.37], dtype=torch.float32, device="cuda") if static else None
+    out = []
+    for two in (True, False):
+        codes = torch.full((rows, cols // 2), 0x5A, dtype=torch.uint8, device="cuda")
+        scales = torch.full((rows,), -1.0, dtype=torch.float32, device="cuda")
+        if two:
+            hq.hq_hadamard_quant(ta, had_block, 4, codes, hq.HQ_CODES_NIBBLE, scales=scales, static_scale=ss, x2=tb)
+        else:
+            hq.hq_hadamard_quant(cat, had_block, 4, codes, hq.HQ_CODES_NIBBLE, scales=scales, static_scale=ss)
+        torch.cuda.synchronize()
+        out.append((codes.cpu().numpy(), scales.cpu().numpy()))
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    u = oracle.transform(x, had_block)
+    q_ref, s_ref, v = oracle.quantize(u, 4, static_scale=0.37 if static else None, want_v=True)
+    if static:
+        v = np.clip(v, oracle.qmin(4) - 0.25, oracle.qmax(4) + 0.25)
+    else:
+        assert np.allclose(out[0][1], s_ref, rtol=SCALE_RTOL, atol=0)
+    check_codes(unpack_nibbles_np(out[0][0]), q_ref, v, f"concatenated input {rows}x({c1}+{c2}) {dt}")
+
+
+def test_quant_of_a_concatenation_refuses_a_block_across_the_seam(env):
+    torch, hq = env
+    ta = torch.zeros((32, 128), dtype=torch.bfloat16, device="cuda")
+    tb = torch.zeros((32, 384), dtype=torch.bfloat16, device="cuda")
+    codes = torch.zeros((32, 256), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((32,), dtype=torch.float32, device="cuda")
+    with pytest.raises(hq.HqError):
+        hq.hq_hadamard_quant(ta, 256, 4, codes, hq.HQ_CODES_NIBBLE, scales=scales, x2=tb)     # 128 is not a multiple of 256

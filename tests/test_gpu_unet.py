@@ -58,6 +58,8 @@ def test_every_layer_matches_the_oracle_on_the_devices_own_input(run, oracle):
         name, op = r["name"], r["op"]
         if op in ("conv3", "conv1"):
             x = host(r["x"])
+            if r.get("x2") is not None:                            # a skip connection joined by concatenation, read in place
+                x = np.concatenate([x, host(r["x2"])], axis=-1)
             Nb, H, W, C = x.shape
             w, b = P[name + ".w"], P[name + ".b"]
             stride = r.get("stride", 1)
@@ -138,6 +140,8 @@ def test_every_layer_matches_the_oracle_on_the_devices_own_input(run, oracle):
     # every call of the forward was checked: 16 residual blocks x 3-4 layers, 11 attention blocks x 2, 6 resampling convs, 2 embedding linears
     assert checked["q"] == len([1 for tag, _, _ in net.tape if tag == "q"]) and checked["q"] >= 80
     assert checked["g"] == len([1 for tag, _, _ in net.tape if tag == "g"])
+    # every residual block of the up-sampling path read [h | skip] in place, in its first and in its 1x1 skip convolution
+    assert sum(1 for r in run["rec"] if r.get("x2") is not None) == 2 * sum(1 for r in run["rec"] if r["name"].startswith("up") and r["name"].endswith(".conv2"))
     # every residual block's second convolution took the block's embedding as its addend
     assert [r["name"] for r in run["rec"] if r.get("pre_bias") is not None] == [r["name"] for r in run["rec"] if r["name"].endswith(".conv2")]
 
