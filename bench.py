@@ -340,9 +340,10 @@ def measure_variants(torch, hq, device, layers, status, stream, rank):
                 acc.setdefault(L["name"], []).append(b.elapsed_time(c2))
             return {k: float(np.median(v)) for k, v in acc.items()}
         lin = [L for L in layers if L["kind"] == "linear" and L["K"] <= 512]
-        one_cta = gemm_only_ms(lin)
-        before = hq.hq_set_pair_gemm(True)
+        before = hq.hq_set_pair_gemm(0)
         try:
+            one_cta = gemm_only_ms(lin)
+            hq.hq_set_pair_gemm(1)
             paired = gemm_only_ms(lin)
         finally:
             hq.hq_set_pair_gemm(before)
@@ -616,6 +617,8 @@ def main_unet(args):
     from paper_2512_05746_b200.unet import UNet, quantized_layers
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
+    if args.pair_gemm:
+        hq.hq_set_pair_gemm(1)
     batch = 64 if args.rows == 32768 else max(1, int(args.rows))          # --rows N: a reduced batch for profiler captures
     cfg = inputs.unet_config(batch=batch)
     t_setup = time.time()
@@ -919,7 +922,7 @@ def main():
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     ap.add_argument("--pair-gemm", action="store_true",
-                    help="run the short-reduction products on pairs of SMs (tcgen05.mma.cta_group::2; hq_set_pair_gemm)")
+                    help="run every covered product on pairs of SMs, the short reductions too (hq_set_pair_gemm(1); the default mode 2\n                         takes pairs for streamed weights and convolutions only)")
     ap.add_argument("--print-csrc-digest", action="store_true", help="print the digest profiles/dram_traffic.json records")
     ap.add_argument("--profile-forward", action="store_true",
                     help="--workload unet: run one forward between cudaProfilerStart / Stop and exit (for a profiler's "
@@ -979,8 +982,8 @@ def main():
     warmup = max(args.warmup, 3)
     R = max(1, args.passes_per_step)
     if args.pair_gemm:
-        hq.hq_set_pair_gemm(True)
-        WORKLOAD = WORKLOAD + ", K <= 512 products on SM pairs"
+        hq.hq_set_pair_gemm(1)
+        WORKLOAD = WORKLOAD + ", every covered product on SM pairs"
     layers = build_layers(torch, hq, device, seed=rank)
     status = torch.zeros((1,), dtype=torch.int32, device=device)
     stream = torch.cuda.current_stream()

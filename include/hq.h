@@ -363,10 +363,14 @@ hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, 
                              int a_bits, hq_scale_mode mode, const float* static_scale, void* y, hq_dtype ydt,
                              int64_t ldy, int32_t* dev_status, void* stream);
 
-/* Tuning switch: whether hq_qgemm and the fused layer calls run short-reduction products (K_pad <= 512, one code per
- * byte, bf16 output, M >= 256) on pairs of SMs (tcgen05.mma.cta_group::2: each CTA of a 2-CTA cluster holds half of the
- * weight tile).  Results are identical either way.  Returns the previous setting.  Process-wide, not thread-safe. */
-int hq_set_pair_gemm(int enable);
+/* Tuning switch: where hq_qgemm, hq_qconv2d and the fused layer calls run their products on pairs of SMs
+ * (tcgen05.mma.cta_group::2: each CTA of a 2-CTA cluster holds half of the weight tile or of every streamed weight block;
+ * one code per byte, bf16 output, one activation scale per row or one static scale, at least 256 rows).
+ *   0  nowhere;
+ *   1  wherever a pair kernel covers the problem (also short reductions, K_pad <= 512, where it measures level);
+ *   2  (default) where it measured faster: reductions with streamed weights (K_pad > 512) and convolutions.
+ * Results are bit-identical in every mode.  Returns the previous mode.  Process-wide, not thread-safe. */
+int hq_set_pair_gemm(int mode);
 
 /* alpha of the rescale for a descriptor: 2^(-k/2) for FOLDED weights (the second normalisation of Eq. 12), else 1. */
 float hq_alpha_for(const hq_weight_desc* desc);

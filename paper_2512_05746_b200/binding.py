@@ -452,9 +452,10 @@ def hq_qlinear_fused(x, pw: PreparedWeight, bias, a_bits: int, y, static_scale=N
                                 _dptr(dev_status), _stream(stream)), "hq_qlinear_fused")
 
 
-def hq_set_pair_gemm(enable: bool) -> bool:
-    """Whether short-reduction products run on pairs of SMs (cta_group::2); returns the previous setting."""
-    return bool(lib.hq_set_pair_gemm(int(bool(enable))))
+def hq_set_pair_gemm(mode: int) -> int:
+    """Where products run on pairs of SMs (cta_group::2): 0 nowhere, 1 (or True) wherever covered, 2 (the default) where
+    it measured faster (streamed weights, convolutions); returns the previous mode."""
+    return int(lib.hq_set_pair_gemm(int(mode)))
 
 
 def hq_mma_i8_probe_pair(pairs: int, iters: int, dev_status=None, stream=None) -> None:

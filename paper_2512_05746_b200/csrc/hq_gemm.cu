@@ -27,7 +27,16 @@ hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t l
                             const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
                             const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
                             bool after_quant);
-int g_pair_gemm = 0;       // hq_set_pair_gemm
+bool pair_stream_covers_gemm(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,
+                             const int32_t* acc_out, bool combine_fast);
+bool pair_stream_covers_conv(hq_container cont, const gemm::GemmParams& g);
+hq_status launch_qgemm_pair_stream(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
+                                   const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
+                                   const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
+                                   bool after_quant);
+hq_status launch_qconv_pair(const gemm::GemmParams& g, const CUtensorMap& tmA, const CUtensorMap& tmY,
+                            const hq_weight_desc* desc, const void* w_dev, cudaStream_t st);
+int g_pair_gemm = 2;       // hq_set_pair_gemm: 0 never, 1 wherever the pair kernels cover, 2 where they measured faster
 
 namespace {
 
@@ -288,9 +297,12 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
                   dev_status);
 
-    if (g_pair_gemm && pair_kernel_covers(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))
+    if (g_pair_gemm == 1 && pair_kernel_covers(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))
         return launch_qgemm_pair(a_codes, M, K, lda, desc, w_dev, scale_a, scale_a_is_scalar, scale_w, bias, alpha, y, ldy,
                                  dev_status, st, after_quant);
+    if (g_pair_gemm && pair_stream_covers_gemm(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))
+        return launch_qgemm_pair_stream(a_codes, M, K, lda, desc, w_dev, scale_a, scale_a_is_scalar, scale_w, bias, alpha, y,
+                                        ldy, dev_status, st, after_quant);
 
     CUtensorMap tmA, tmB, tmY{};
     const bool nib = cont == HQ_CODES_NIBBLE;
@@ -369,6 +381,7 @@ hq_status launch_qconv2d(const void* a_codes, hq_container cont, int a_bits, int
     if (!encode_4d(&tmA, a_codes, dims, box, estr, !nib)) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad) * desc->RS;
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, kBN, true)) return HQ_ERR_CUDA;
+    if (g_pair_gemm && pair_stream_covers_conv(cont, p)) return launch_qconv_pair(p, tmA, tmY, desc, w_dev, st);
     s = launch(nib, tmA, tmB, tmY, p, st);
     if (s == HQ_OK && per_tap && desc->limbs == 1) {      // the other 64 of every warp's 128 columns
         p.col_pass = 1;
@@ -398,9 +411,9 @@ extern "C" hq_status hq_qconv2d(const void* a_codes, hq_container cont, int a_bi
                               static_cast<cudaStream_t>(stream), false);
 }
 
-extern "C" int hq_set_pair_gemm(int enable) {
+extern "C" int hq_set_pair_gemm(int mode) {
     const int before = hq::g_pair_gemm;
-    hq::g_pair_gemm = enable ? 1 : 0;
+    hq::g_pair_gemm = mode < 0 ? 0 : (mode > 2 ? 2 : mode);
     return before;
 }
 

@@ -360,6 +360,189 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
 }
 
+// ---- long reductions and convolutions on pairs of SMs: weights streamed --------------------------------------------
+// Where the reduction does not fit a resident weight tile (K_pad > 512, every 3x3 convolution), the one-CTA kernel's
+// issuing lane needs about as long per 128-byte K block (barrier wait, four MMAs, commit: ~600 cycles) as the tensor
+// pipe needs to run it (536), and its ring holds four 48 KB stages.  On a pair of SMs one lane issues a K block for
+// both tensor cores, each CTA brings its own 128 activation rows and HALF of the 256 weight rows of the block (32 KB
+// per stage and CTA: six stages), and the same MMA count serves twice the rows.  Tiles are taken in row-major order,
+// pair c the tiles c, c + G, ..., so that the pairs working side by side share their activation rows in L2.
+// Convolution: a tile's 128 rows are 128 consecutive output pixels (whole output rows; checked by the host), fetched per
+// filter tap by a 4-D bulk tensor load whose out-of-range coordinates supply the zero padding.
+struct PairStreamParams {
+    int64_t M; int N, limbs, num_kb, tiles_m2, tiles_n, stages;
+    const float* scale_a; int sa_scalar;
+    const float* scale_w; const float* bias; float alpha;
+    int pdl;
+    int32_t* dev_status;
+    // convolution geometry (CONV instantiations)
+    int kb_per_tap, S, stride, pad, bw, bh, bn, tiles_w, tiles_h;
+};
+
+constexpr int kPairStageBytes = kABytes + kPairBBytes;      // 32 KB: this CTA's activation rows and its half of the weights
+
+struct PairStreamLayout { int ring_off, staging_off, param_off, ctl_off, total; };
+__host__ __device__ inline PairStreamLayout pair_stream_layout(int stages) {
+    PairStreamLayout L;
+    L.ring_off = 0;
+    L.staging_off = stages * kPairStageBytes;
+    L.param_off = L.staging_off + kEpiWarps * 2 * kStagingBytes;
+    L.ctl_off = L.param_off + kPairParamBytes;
+    L.total = L.ctl_off + int(sizeof(PairCtl)) + 1024;
+    return L;
+}
+
+__device__ __forceinline__ void tma_load_4d_pair(void* smem_dst, const void* tmap, uint32_t bar_cluster_addr, int c0, int c1,
+                                                 int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2),
+          "r"(c3)
+        : "memory");
+}
+
+template <int LIMBS, bool CONV>
+__global__ void __launch_bounds__(kPairThreads, 1)
+qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmY, const PairStreamParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const PairStreamLayout L = pair_stream_layout(p.stages);
+    unsigned char* sRing = smem + L.ring_off;
+    unsigned char* sStage = smem + L.staging_off;
+    float* sParam = reinterpret_cast<float*>(smem + L.param_off);
+    PairCtl* ctl = reinterpret_cast<PairCtl*>(smem + L.ctl_off);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();                 // 0: leader (issues the MMAs), 1: its peer
+    const int nstages = p.stages, num_kb = p.num_kb;
+    const int T = p.tiles_m2 * p.tiles_n, G = gridDim.x >> 1, c = blockIdx.x >> 1;
+    const int count = c < T ? (T - c + G - 1) / G : 0;    // tiles c, c + G, ... of the row-major order
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPairMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 2 * kEpiWarps); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+        tma_prefetch_desc(&tmY);
+    }
+    if (warp == 1) { __syncwarp(); tmem_alloc_pair(&ctl->tmem_base, kTmemCols); tmem_relinquish_pair(); }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers are initialised and both tensor memories allocated
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (one per CTA, its own halves)
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            if (p.pdl) griddep_wait();                     // the codes come from the kernel before this one
+            for (int i = 0; i < count && ok; ++i) {
+                const int u = c + i * G;
+                const int m2 = u / p.tiles_n, n_tile = u - m2 * p.tiles_n;
+                const int m_tile = m2 * 2 + int(rank);     // this CTA's 128 rows
+                int w0 = 0, h0 = 0, n0 = 0;
+                if (CONV) {
+                    const int tw = m_tile % p.tiles_w;
+                    const int th = (m_tile / p.tiles_w) % p.tiles_h;
+                    const int tn = m_tile / (p.tiles_w * p.tiles_h);
+                    w0 = tw * p.bw; h0 = th * p.bh; n0 = tn * p.bn;      // past the last image: the load delivers zeros
+                }
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!wait_pair(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
+                    const uint32_t fbar = map_to_cta(&ctl->full[stage], 0);
+                    if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(kPairStageBytes));
+                    unsigned char* dst = sRing + stage * kPairStageBytes;
+                    if (CONV) {
+                        const int tap = kb / p.kb_per_tap, kc = kb - tap * p.kb_per_tap;
+                        const int r = tap / p.S, s = tap - r * p.S;
+                        tma_load_4d_pair(dst, &tmA, fbar, kc * kBK, w0 * p.stride + s - p.pad, h0 * p.stride + r - p.pad, n0);
+                    } else {
+                        tma_load_2d_pair(dst, &tmA, fbar, kb * kBK, m_tile * kBM);
+                    }
+                    tma_load_2d_pair(dst + kABytes, &tmB, fbar, kb * kBK, n_tile * kBN + int(rank) * 128);
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_i8(256, kBN);
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int i = 0; i < count && ok; ++i) {
+                const int as = i & 1;
+                if (!wait_pair(&ctl->tempty[as], (uint32_t(i >> 1) & 1u) ^ 1u, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!wait_pair(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sRing + stage * kPairStageBytes));
+                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sRing + stage * kPairStageBytes + kABytes));
+#pragma unroll
+                    for (int k = 0; k < kBK / 32; ++k)
+                        mma_i8_pair(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                    mma_commit_pair(&ctl->empty[stage]);
+                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                mma_commit_pair(&ctl->tfull[as]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2-9 of both CTAs)
+        const int ew = warp - 2;
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        const int chalf = ew >> 2;                    // which half of the tile's columns this warp takes
+        unsigned char* stg = sStage + ew * 2 * kStagingBytes;
+        float* prm_sw = sParam + ew * 2 * (kBN / 2);
+        float* prm_b = prm_sw + kBN / 2;
+        constexpr int cols_per_tile = LIMBS == 2 ? kBN / 2 : kBN;
+        constexpr int cols_per_warp = cols_per_tile / 2;
+        const int wc0 = chalf * cols_per_warp;
+        const uint32_t tempty_leader[2] = {map_to_cta(&ctl->tempty[0], 0), map_to_cta(&ctl->tempty[1], 0)};
+        int last_n = -1;
+        bool ok = true;
+        if (p.pdl) griddep_wait();                    // scale_a comes from the kernel before this one
+        for (int i = 0; i < count && ok; ++i) {
+            const int u = c + i * G;
+            const int m2 = u / p.tiles_n, n_tile = u - m2 * p.tiles_n;
+            const int as = i & 1;
+            const int col_base = n_tile * cols_per_tile;
+            if (n_tile != last_n) {
+                last_n = n_tile;
+                __syncwarp();
+                for (int cc = lane; cc < cols_per_warp; cc += 32) {
+                    const int col = col_base + wc0 + cc;
+                    prm_sw[cc] = col < p.N ? __ldg(p.scale_w + col) : 0.f;
+                    prm_b[cc] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
+                }
+                __syncwarp();
+            }
+            const int64_t my_row = int64_t(m2) * 256 + int(rank) * 128 + q * 32 + lane;
+            const float sa = p.sa_scalar ? __ldg(p.scale_a) : (my_row < p.M ? __ldg(p.scale_a + my_row) : 0.f);
+            if (!wait_pair(&ctl->tfull[as], uint32_t(i >> 1) & 1u, ctl, p.dev_status, kStatusAccumWait)) { ok = false; break; }
+            tc_fence_after();
+            const float sa_eff = p.alpha * sa;
+            const int row0 = m2 * 256 + int(rank) * 128 + q * 32;
+            const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
+            epilogue_pair<LIMBS>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as]);
+        }
+        if (lane == 0) bulk_wait_read_all();           // shared memory must outlive the copy engine's reads
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // neither CTA leaves while its peer may still signal its barriers or read its operands
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
+}
+
 // Issue-rate probe of the paired int8 MMA: back-to-back 256 x 256 x 32 MMAs of a 2-CTA cluster on resident tiles.
 __global__ void __launch_bounds__(128, 1) mma_pair_probe_kernel(int iters, int32_t* dev_status) {
     extern __shared__ unsigned char smem_raw[];
@@ -440,7 +623,113 @@ int max_pairs(size_t smem) {
     return slot;
 }
 
+template <int LIMBS, bool CONV>
+cudaError_t launch_pair_stream(int pairs_wanted, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
+                               const CUtensorMap& tmY, const PairStreamParams& p) {
+    auto kern = qgemm_pair_stream_kernel<LIMBS, CONV>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(unsigned(kPairThreads));
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    // how many 2-CTA clusters the device runs at once (the SM count of a GPC need not be even), once per device
+    static int cached[64] = {};
+    int dev = 0, pairs_max = sm_count() / 2 - 2;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        if (cached[dev] == 0) {
+            int n = 0;
+            cfg.gridDim = dim3(unsigned(sm_count() / 2 * 2));
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0)
+                cached[dev] = n < sm_count() / 2 ? n : sm_count() / 2;
+            else
+                cached[dev] = pairs_max;
+        }
+        pairs_max = cached[dev];
+    }
+    const int pairs = pairs_wanted < pairs_max ? pairs_wanted : pairs_max;
+    cfg.gridDim = dim3(unsigned(2 * pairs));
+    int na = 1;
+    if (p.pdl) {
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        na = 2;
+    }
+    cfg.numAttrs = unsigned(na);
+    return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
+}
+
+bool pair_stream_stages(PairStreamParams& p, size_t& smem) {
+    for (int stages = kPairMaxStages; stages >= 3; --stages) {
+        const PairStreamLayout L = pair_stream_layout(stages);
+        if (L.total <= kSmemLimit) { p.stages = stages; smem = size_t(L.total); return true; }
+    }
+    return false;
+}
+
 }  // namespace
+
+// Whether the streamed pair kernel covers a plain GEMM / a convolution planned by the one-CTA path (`g`: that plan).
+bool pair_stream_covers_gemm(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,
+                             const int32_t* acc_out, bool combine_fast) {
+    return cont == HQ_CODES_INT8 && desc->RS == 1 && desc->C_pad > int64_t(kResidentKb) * kBK && y != nullptr &&
+           acc_out == nullptr && ydt == HQ_BF16 && aligned16(y) && (ldy * 2) % 16 == 0 && combine_fast && M >= 256;
+}
+bool pair_stream_covers_conv(hq_container cont, const gemm::GemmParams& g) {
+    return cont == HQ_CODES_INT8 && g.conv && g.tma_store && !g.per_tap && g.sa_scalar && g.bw * g.bh * g.bn == kBM &&
+           int64_t(g.tiles_m) >= 2;
+}
+
+hq_status launch_qgemm_pair_stream(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
+                                   const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
+                                   const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
+                                   bool after_quant) {
+    PairStreamParams p{};
+    p.M = M; p.N = int(desc->N); p.limbs = desc->limbs;
+    p.num_kb = int(desc->C_pad / kBK);
+    p.tiles_m2 = int((M + 255) / 256);
+    p.tiles_n = int(desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
+    p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
+    p.pdl = after_quant ? 1 : 0; p.dev_status = dev_status;
+    size_t smem = 0;
+    if (!pair_stream_stages(p, smem)) return HQ_ERR_UNSUPPORTED;
+    CUtensorMap tmA, tmB, tmY;
+    if (!encode_2d(&tmA, a_codes, uint64_t(K), uint64_t(M), uint64_t(lda), kBK, kBM, true)) return HQ_ERR_CUDA;
+    const uint64_t Kp = uint64_t(desc->C_pad);
+    if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
+    if (!encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
+    const int tiles = p.tiles_m2 * p.tiles_n;
+    cudaError_t e = desc->limbs == 2 ? launch_pair_stream<2, false>(tiles, smem, st, tmA, tmB, tmY, p)
+                                     : launch_pair_stream<1, false>(tiles, smem, st, tmA, tmB, tmY, p);
+    return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
+
+// The convolution the one-CTA path has planned in `g` (tile geometry, epilogue parameters) on pairs of SMs; tmA and tmY are
+// that plan's tensor maps (the activation boxes are the same 128 pixels), the weight map is rebuilt with 128-row boxes.
+hq_status launch_qconv_pair(const gemm::GemmParams& g, const CUtensorMap& tmA, const CUtensorMap& tmY,
+                            const hq_weight_desc* desc, const void* w_dev, cudaStream_t st) {
+    PairStreamParams p{};
+    p.M = int64_t(g.Nb) * g.Ho * g.Wo; p.N = g.N; p.limbs = g.limbs;
+    p.num_kb = g.kb_per_tap * g.taps;
+    p.tiles_m2 = (g.tiles_m + 1) / 2;
+    p.tiles_n = g.tiles_n;
+    p.scale_a = g.scale_a; p.sa_scalar = g.sa_scalar; p.scale_w = g.scale_w; p.bias = g.bias; p.alpha = g.alpha;
+    p.pdl = g.pdl; p.dev_status = g.dev_status;
+    p.kb_per_tap = g.kb_per_tap; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
+    p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.tiles_w = g.tiles_w; p.tiles_h = g.tiles_h;
+    size_t smem = 0;
+    if (!pair_stream_stages(p, smem)) return HQ_ERR_UNSUPPORTED;
+    CUtensorMap tmB;
+    const uint64_t Kp = uint64_t(desc->C_pad) * desc->RS;
+    if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
+    const int tiles = p.tiles_m2 * p.tiles_n;
+    cudaError_t e = desc->limbs == 2 ? launch_pair_stream<2, true>(tiles, smem, st, tmA, tmB, tmY, p)
+                                     : launch_pair_stream<1, true>(tiles, smem, st, tmA, tmB, tmY, p);
+    return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
+}
 
 // Whether the pair kernel covers a problem (see the top of this file); the caller has validated the arguments.
 bool pair_kernel_covers(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,

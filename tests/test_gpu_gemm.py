@@ -310,6 +310,12 @@ PAIR_CASES = [
     (300, 128, 72, 128, "folded"),        # one K block
     (40000, 256, 384, 256, "double"),     # more pair tiles than clusters; the weight tile changes inside a pair's range
     (256, 384, 136, 128, "folded"),       # three K blocks
+    # reductions beyond the resident weight tile: weights streamed through the pair's ring
+    (1000, 1024, 384, 1024, "folded"),    # eight K blocks, ragged rows, three column tiles
+    (4096, 2048, 512, 2048, "folded"),    # the shape of the step's FF2 at an eighth of its rows
+    (777, 640, 328, 128, "plain"),        # five K blocks, one weight limb, ragged columns
+    (38000, 768, 256, 256, "folded"),     # more pair tiles than clusters: tiles c, c + G, ... per pair
+    (300, 1152, 72, 128, "double"),       # nine K blocks
 ]
 
 
@@ -330,9 +336,10 @@ def test_qgemm_on_sm_pairs_matches_oracle(env, oracle, M, K, N, n, mode):
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")
     y_one = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
     y_pair = torch.full((M, N), 3.0, dtype=torch.bfloat16, device="cuda")
-    hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_one, dev_status=status)
-    before = hq.hq_set_pair_gemm(True)
+    before = hq.hq_set_pair_gemm(0)
     try:
+        hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_one, dev_status=status)
+        hq.hq_set_pair_gemm(1)
         hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_pair, dev_status=status)
         torch.cuda.synchronize()
     finally:
@@ -349,3 +356,48 @@ def test_paired_tensor_pipe_probe_runs(env):
     hq.hq_mma_i8_probe_pair(2, 64, dev_status=status)
     torch.cuda.synchronize()
     hq.hq_check_status(status)
+
+
+PAIR_CONV_CASES = [
+    # Nb, H, W, C, Cout, R, stride, pad, mode
+    (8, 32, 32, 256, 256, 3, 1, 1, "folded"),      # the small conv configuration: 64 tiles of 128 pixels, two column tiles
+    (3, 8, 8, 256, 128, 3, 1, 1, "folded"),        # tiles span two images; an odd number of tiles (the peer's last tile is empty)
+    (2, 64, 64, 128, 128, 3, 1, 1, "plain"),       # two output rows per tile, one weight limb
+    (2, 32, 32, 256, 256, 3, 2, 1, "folded"),      # the down-sampling convolution of a UNet level
+    (4, 16, 16, 768, 320, 1, 1, 0, "folded"),      # 1x1 skip convolution with six K blocks, ragged columns
+    (5, 16, 16, 384, 256, 3, 1, 1, "double"),      # 27 K blocks, five images of two tiles each
+]
+
+
+@pytest.mark.parametrize("Nb,H,W,C,Cout,R,stride,pad,mode", PAIR_CONV_CASES)
+def test_qconv2d_on_sm_pairs_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, stride, pad, mode):
+    """The implicit-GEMM convolution on pairs of SMs (weights streamed, each CTA half of every weight K block): bf16 output
+    against the oracle's rescale of the oracle's integer convolution, and bit for bit against the one-CTA kernel."""
+    torch, hq = env
+    hb = 128
+    q = inputs.codes((Nb, H, W, C), 4, seed=H + C + Cout)
+    w = inputs.weights((Cout, R, R, C), seed=C + Cout)
+    pw = hq.hq_weight_prepare(w, 4, hb, hq.WEIGHT_MODES[mode], hq.HQ_CODES_INT8).to_device()
+    B_ref = weight_integers(oracle, pw, w, 4, hb, mode).reshape(Cout, R, R, C)
+    b = inputs.bias(Cout, seed=2)
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
+    a_dev = to_container(torch, hq, q, hq.HQ_CODES_INT8)
+    s_a = torch.tensor([0.05], device="cuda")
+    b_dev = torch.from_numpy(b).cuda()
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y_one = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
+    y_pair = torch.full((Nb, Ho, Wo, Cout), 3.0, dtype=torch.bfloat16, device="cuda")
+    before = hq.hq_set_pair_gemm(0)
+    try:
+        hq.hq_qconv2d(a_dev, hq.HQ_CODES_INT8, 4, Nb, H, W, C, pw, R, R, stride, pad, scale_a=s_a, bias=b_dev, alpha=pw.alpha,
+                      y=y_one, dev_status=status)
+        hq.hq_set_pair_gemm(1)
+        hq.hq_qconv2d(a_dev, hq.HQ_CODES_INT8, 4, Nb, H, W, C, pw, R, R, stride, pad, scale_a=s_a, bias=b_dev, alpha=pw.alpha,
+                      y=y_pair, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        hq.hq_set_pair_gemm(before)
+    hq.hq_check_status(status)
+    y_ref = oracle.dequant(oracle.conv2d_int(q, B_ref, stride, pad), np.array([0.05], np.float32), pw.s_w, b, pw.alpha)
+    assert rel_err(y_pair.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
+    assert torch.equal(y_pair, y_one)
