@@ -679,8 +679,9 @@ bool pair_stream_covers_gemm(hq_container cont, const hq_weight_desc* desc, int6
            acc_out == nullptr && ydt == HQ_BF16 && aligned16(y) && (ldy * 2) % 16 == 0 && combine_fast && M >= 256;
 }
 bool pair_stream_covers_conv(hq_container cont, const gemm::GemmParams& g) {
-    return cont == HQ_CODES_INT8 && g.conv && g.tma_store && !g.per_tap && g.sa_scalar && g.bw * g.bh * g.bn == kBM &&
-           int64_t(g.tiles_m) >= 2;
+    // one static scale, or one scale per output pixel of a 1x1 convolution (per_tap marks per-pixel scales under a window)
+    return cont == HQ_CODES_INT8 && g.conv && g.tma_store && !g.per_tap && g.bw * g.bh * g.bn == kBM &&
+           g.kb_per_tap * g.taps > kResidentKb && int64_t(g.tiles_m) >= 2;
 }
 
 hq_status launch_qgemm_pair_stream(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,

@@ -382,7 +382,9 @@ def test_qconv2d_on_sm_pairs_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, s
     b = inputs.bias(Cout, seed=2)
     Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
     a_dev = to_container(torch, hq, q, hq.HQ_CODES_INT8)
-    s_a = torch.tensor([0.05], device="cuda")
+    # one static scale; the 1x1 convolution takes one scale per pixel instead (the skip projections of the UNet)
+    sa_np = inputs.positive_scales(Nb * H * W, seed=H) if R == 1 else np.array([0.05], np.float32)
+    s_a = torch.from_numpy(sa_np).cuda()
     b_dev = torch.from_numpy(b).cuda()
     status = torch.zeros((1,), dtype=torch.int32, device="cuda")
     y_one = torch.zeros((Nb, Ho, Wo, Cout), dtype=torch.bfloat16, device="cuda")
@@ -398,6 +400,7 @@ def test_qconv2d_on_sm_pairs_matches_oracle(env, oracle, Nb, H, W, C, Cout, R, s
     finally:
         hq.hq_set_pair_gemm(before)
     hq.hq_check_status(status)
-    y_ref = oracle.dequant(oracle.conv2d_int(q, B_ref, stride, pad), np.array([0.05], np.float32), pw.s_w, b, pw.alpha)
+    acc_ref = oracle.conv2d_int(q, B_ref, stride, pad)
+    y_ref = oracle.dequant(acc_ref.reshape(-1, Cout), sa_np, pw.s_w, b, pw.alpha).reshape(acc_ref.shape)
     assert rel_err(y_pair.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
     assert torch.equal(y_pair, y_one)
