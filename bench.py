@@ -57,7 +57,7 @@ def ws_views(torch, ws, rows, cols):
     return ws[: rows * pitch].view(rows, pitch), ws[off: off + rows * 4].view(torch.float32)
 
 
-STEP_KERNEL_SOURCES = ("hq_common.cuh", "hq_fwht.cuh", "hq_quant.cu", "hq_gemm_kernel.cuh", "hq_gemm.cu", "hq_api.cu",
+STEP_KERNEL_SOURCES = ("hq_common.cuh", "hq_fwht.cuh", "hq_quant.cu", "hq_gemm_kernel.cuh", "hq_gemm.cu", "hq_gemm_pair.cu", "hq_api.cu",
                        "hq_gemm_inst_i8_gemm.cu", "hq_gemm_inst_i8_conv.cu", "hq_gemm_inst_nibble_gemm.cu",
                        "hq_gemm_inst_nibble_conv.cu")
 
