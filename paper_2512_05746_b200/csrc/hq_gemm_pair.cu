@@ -472,7 +472,13 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && rank == 0) {
+            // A lone lane spends several cycles per instruction, and this lane's path per K block is what paces the
+            // kernel: the operand descriptors advance by constants (a stage is 32 KB = 2048 descriptor units on, the
+            // weights 1024 units behind the activations), and only the very first MMA of a tile overwrites.
             const uint32_t idesc = make_idesc_i8(256, kBN);
+            const uint64_t desc0 = make_sw128_kmajor_desc(smem_u32(sRing));
+            constexpr uint64_t kStageUnits = kPairStageBytes >> 4, kBUnits = kABytes >> 4;
+            uint64_t a_desc = desc0;
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int i = 0; i < count && ok; ++i) {
@@ -480,16 +486,19 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 if (!wait_pair(&ctl->tempty[as], (uint32_t(i >> 1) & 1u) ^ 1u, ctl, p.dev_status, kStatusAccumFree)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                uint32_t acc = 0;                          // 0 for the first MMA of the tile only
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_pair(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t a_desc = make_sw128_kmajor_desc(smem_u32(sRing + stage * kPairStageBytes));
-                    const uint64_t b_desc = make_sw128_kmajor_desc(smem_u32(sRing + stage * kPairStageBytes + kABytes));
-#pragma unroll
-                    for (int k = 0; k < kBK / 32; ++k)
-                        mma_i8_pair(d_tmem, a_desc + uint64_t(k * 2), b_desc + uint64_t(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                    const uint64_t b_desc = a_desc + kBUnits;
+                    mma_i8_pair(d_tmem, a_desc, b_desc, idesc, acc);
+                    mma_i8_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
+                    mma_i8_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
+                    mma_i8_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+                    acc = 1u;
                     mma_commit_pair(&ctl->empty[stage]);
-                    if (++stage == nstages) { stage = 0; phase ^= 1; }
+                    a_desc += kStageUnits;
+                    if (++stage == nstages) { stage = 0; phase ^= 1; a_desc = desc0; }
                 }
                 if (!ok) break;
                 mma_commit_pair(&ctl->tfull[as]);
