@@ -50,6 +50,17 @@ def codes_name():
     return "nibble" if CODES[0] == 0 else "int8"
 
 
+def gemm_kernel_name(L):
+    """The kernel the library's default dispatch takes for a layer of the step (see hq_set_pair_gemm in include/hq.h)."""
+    if codes_name() != "int8":
+        return "qgemm_kernel<nibble>"
+    if L["kind"] == "conv" or L["K"] > 512:
+        return "qgemm_pair_stream_kernel (pairs of SMs, streamed weights)"
+    if L["K"] in (256, 512):
+        return "qgemm_pair_kernel (pairs of SMs, resident weights, two K blocks per ring stage)"
+    return "qgemm_kernel<int8>"
+
+
 def ws_views(torch, ws, rows, cols):
     """Codes [rows, pitch] and scales [rows] inside the workspace of a fused layer call (the documented layout)."""
     pitch = (code_pitch(cols) + 15) // 16 * 16
@@ -922,7 +933,8 @@ def main():
     ap.add_argument("--rows", type=int, default=M_TOKENS,
                     help="rows per layer (default: the full 32768; smaller values are for profiler captures only)")
     ap.add_argument("--pair-gemm", action="store_true",
-                    help="run every covered product on pairs of SMs, the short reductions too (hq_set_pair_gemm(1); the default mode 2\n                         takes pairs for streamed weights and convolutions only)")
+                    help="run every covered product on pairs of SMs (hq_set_pair_gemm(1)); the default mode 2 takes pairs where they "
+                         "measured faster")
     ap.add_argument("--print-csrc-digest", action="store_true", help="print the digest profiles/dram_traffic.json records")
     ap.add_argument("--profile-forward", action="store_true",
                     help="--workload unet: run one forward between cudaProfilerStart / Stop and exit (for a profiler's "
@@ -1118,7 +1130,7 @@ def main():
         L = dom["L"]
         gemm_ms = dom["gemm_ms"]
         ach = L["ops"] / (gemm_ms * 1e-3) / 1e12
-        roofline = dict(bound="tensor", kernel=f"qgemm_kernel<{codes_name()}> ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
+        roofline = dict(bound="tensor", kernel=f"{gemm_kernel_name(L)} ({L['name']}: M={L['M']} K={L['K']} N={L['N']} "
                                                 f"limbs={L['limbs']})",
                         achieved=ach, peak=int8_peak, unit="TOPS", frac=ach / int8_peak,
                         achieved_counts="2*M*N*K*limbs (the tensor work issued; the layer's own 2*M*N*K is achieved/limbs)",

@@ -367,8 +367,10 @@ hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, 
  * (tcgen05.mma.cta_group::2: each CTA of a 2-CTA cluster holds half of the weight tile or of every streamed weight block;
  * one code per byte, bf16 output, one activation scale per row or one static scale, at least 256 rows).
  *   0  nowhere;
- *   1  wherever a pair kernel covers the problem (also short reductions, K_pad <= 512, where it measures level);
- *   2  (default) where it measured faster: reductions with streamed weights (K_pad > 512) and convolutions.
+ *   1  wherever a pair kernel covers the problem (also K_pad 128 or 384 and problems of few tiles, where it measures level
+ *      or slower);
+ *   2  (default) where it measured faster: reductions with streamed weights (K_pad > 512), convolutions, and K_pad 256 or
+ *      512 on problems of at least one 256-row tile per SM.
  * Results are bit-identical in every mode.  Returns the previous mode.  Process-wide, not thread-safe. */
 int hq_set_pair_gemm(int mode);
 

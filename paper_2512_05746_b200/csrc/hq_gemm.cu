@@ -27,6 +27,7 @@ hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t l
                             const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
                             const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
                             bool after_quant);
+bool pair_kernel_pays(const hq_weight_desc* desc, int64_t M);
 bool pair_stream_covers_gemm(hq_container cont, const hq_weight_desc* desc, int64_t M, const void* y, hq_dtype ydt, int64_t ldy,
                              const int32_t* acc_out, bool combine_fast);
 bool pair_stream_covers_conv(hq_container cont, const gemm::GemmParams& g);
@@ -297,7 +298,8 @@ hq_status launch_qgemm(const void* a_codes, hq_container cont, int a_bits, int64
     fill_epilogue(p, cont, a_bits, desc, K, scale_a, scale_a_is_scalar, scale_w, bias, alpha, acc_out, y, ydt, ldy,
                   dev_status);
 
-    if (g_pair_gemm == 1 && pair_kernel_covers(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))
+    if (g_pair_gemm && pair_kernel_covers(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0) &&
+        (g_pair_gemm == 1 || pair_kernel_pays(desc, M)))
         return launch_qgemm_pair(a_codes, M, K, lda, desc, w_dev, scale_a, scale_a_is_scalar, scale_w, bias, alpha, y, ldy,
                                  dev_status, st, after_quant);
     if (g_pair_gemm && pair_stream_covers_gemm(cont, desc, M, y, ydt, ldy, acc_out, p.combine_fast != 0))

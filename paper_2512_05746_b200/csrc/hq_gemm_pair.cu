@@ -44,11 +44,12 @@ struct PairCtl {
 };
 
 struct PairLayout { int b_off, a_off, staging_off, param_off, ctl_off, total; };
-__host__ __device__ inline PairLayout pair_layout(int num_kb, int stages) {
+// kps: K blocks of a tile's activations per ring stage
+__host__ __device__ inline PairLayout pair_layout(int num_kb, int stages, int kps = 1) {
     PairLayout L;
     L.b_off = 0;
     L.a_off = num_kb * kPairBBytes;
-    L.staging_off = L.a_off + stages * kABytes;
+    L.staging_off = L.a_off + stages * kps * kABytes;
     L.param_off = L.staging_off + kEpiWarps * 2 * kStagingBytes;       // two staging buffers per epilogue warp
     L.ctl_off = L.param_off + kPairParamBytes;
     L.total = L.ctl_off + int(sizeof(PairCtl)) + 1024;
@@ -98,6 +99,19 @@ __device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, ui
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The same with the shared-memory descriptors given as (low word, high word): only the address field in the low word
+// varies within a kernel, so the issuing lane advances a descriptor with one 32-bit addition.  ACC is a constant.
+template <bool ACC>
+__device__ __forceinline__ void mma_i8_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "n"(ACC ? 1 : 0)
         : "memory");
 }
 // Arrive on the barrier at the same offset in both CTAs of the pair once all MMAs issued so far have completed.
@@ -198,13 +212,20 @@ __device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg
     }
 }
 
-template <int LIMBS>
+// NKB > 0: the reduction has exactly NKB K blocks (compile-time loops) and a ring stage holds KPS = 2 of them (32 KB):
+// one barrier round and one commit per two K blocks.  The issuing lane needs about 70 cycles per MMA and about 180 per
+// barrier round, which for one K block per stage is as long as the tensor pipe runs the block (536 cycles); with two the
+// lane is ahead of the pipe.  Three 32 KB stages fit beside the 64 KB weight half of K_pad = 512 (the pair halves the
+// weights; the one-CTA kernel has 64 KB for all its stages).
+template <int LIMBS, int NKB, int KPS>
 __global__ void __launch_bounds__(kPairThreads, 1)
 qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmY, const PairParams p) {
+    constexpr bool WHOLE = NKB > 0;
+    static_assert(NKB == 0 ? KPS == 1 : (KPS > 1 && NKB % KPS == 0), "a stage holds a whole fraction of the tile's K blocks");
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const PairLayout L = pair_layout(p.num_kb, p.stages);
+    const PairLayout L = pair_layout(p.num_kb, p.stages, KPS);
     unsigned char* sB = smem + L.b_off;
     unsigned char* sA = smem + L.a_off;
     unsigned char* sStage = smem + L.staging_off;
@@ -257,12 +278,27 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     cur_n = n_tile; ++reloads;
                 }
                 if (i == 0 && p.pdl) griddep_wait();       // the codes come from the kernel before this one
+                if constexpr (WHOLE) {
+#pragma unroll
+                    for (int h = 0; h < NKB / KPS; ++h) {
+                        if (!wait_pair(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
+                        if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(KPS * kABytes));
+                        const uint32_t fbar = map_to_cta(&ctl->full[stage], 0);
+#pragma unroll
+                        for (int k = 0; k < KPS; ++k)
+                            tma_load_2d_pair(sA + (stage * KPS + k) * kABytes, &tmA, fbar, (h * KPS + k) * kBK,
+                                             m2 * 256 + int(rank) * 128);
+                        if (++stage == nstages) { stage = 0; phase ^= 1; }
+                    }
+                    if (!ok) break;
+                } else {
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!wait_pair(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
                     if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(kABytes));
                     tma_load_2d_pair(sA + stage * kABytes, &tmA, map_to_cta(&ctl->full[stage], 0), kb * kBK,
                                      m2 * 256 + int(rank) * 128);
                     if (++stage == nstages) { stage = 0; phase ^= 1; }
+                }
                 }
             }
         }
@@ -273,6 +309,58 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int stage = 0; uint32_t phase = 0;
             int cur_n = -1, reloads = 0;
             bool ok = true;
+            if constexpr (WHOLE) {
+                // A lone lane runs its instructions one dependent step at a time (about five cycles each), so this loop is
+                // kept to the instructions the tile needs: tile coordinates advance by counting, descriptors by one
+                // 32-bit addition, the weight-tile barriers are visited only on the first tile of a column tile.
+                const uint64_t dsc = make_sw128_kmajor_desc(smem_u32(sA));
+                const uint32_t desc_hi = uint32_t(dsc >> 32), a_lo0 = uint32_t(dsc);
+                const uint32_t b_lo0 = uint32_t(make_sw128_kmajor_desc(smem_u32(sB)));
+                constexpr uint32_t kStageUnits = uint32_t(KPS * kABytes) >> 4;
+                uint32_t a_lo = a_lo0;
+                int m2 = first % p.tiles_m2;
+                bool new_b = true;
+                for (int i = 0; i < count; ++i) {
+                    const int as = i & 1;
+                    if (!wait_pair(&ctl->tempty[as], (uint32_t(i >> 1) & 1u) ^ 1u, ctl, p.dev_status, kStatusAccumFree)) break;
+                    if (new_b) {
+                        ++reloads;
+                        bool okb = true;
+#pragma unroll
+                        for (int kb = 0; kb < NKB; ++kb)
+                            okb = okb && wait_pair(&ctl->bfull[kb], uint32_t(reloads - 1) & 1u, ctl, p.dev_status, kStatusTmaWait);
+                        if (!okb) break;
+                        new_b = false;
+                    }
+                    const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
+                    bool okt = true;
+#pragma unroll
+                    for (int h = 0; h < NKB / KPS; ++h) {
+                        if (!wait_pair(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { okt = false; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int kk = 0; kk < KPS; ++kk) {
+                            constexpr uint32_t kAUnits = uint32_t(kABytes) >> 4, kBUnits = uint32_t(kPairBBytes) >> 4;
+                            const uint32_t al = a_lo + uint32_t(kk) * kAUnits, bl = b_lo0 + uint32_t(h * KPS + kk) * kBUnits;
+                            if (h == 0 && kk == 0) mma_i8_pair_lh<false>(d_tmem, al, bl, desc_hi, idesc);
+                            else mma_i8_pair_lh<true>(d_tmem, al, bl, desc_hi, idesc);
+                            mma_i8_pair_lh<true>(d_tmem, al + 2, bl + 2, desc_hi, idesc);
+                            mma_i8_pair_lh<true>(d_tmem, al + 4, bl + 4, desc_hi, idesc);
+                            mma_i8_pair_lh<true>(d_tmem, al + 6, bl + 6, desc_hi, idesc);
+                        }
+                        mma_commit_pair(&ctl->empty[stage]);
+                        a_lo += kStageUnits;
+                        if (++stage == nstages) { stage = 0; phase ^= 1; a_lo = a_lo0; }
+                    }
+                    if (!okt) break;
+                    mma_commit_pair(&ctl->tfull[as]);
+                    // the next tile of the range starts a new weight tile: tell both producers when the MMAs on the old one are done
+                    if (++m2 == p.tiles_m2) {
+                        m2 = 0; new_b = true;
+                        if (i + 1 < count) mma_commit_pair(&ctl->bfree);
+                    }
+                }
+            } else
             for (int i = 0; i < count && ok; ++i) {
                 const int u = first + i;
                 const int n_tile = u / p.tiles_m2, m2 = u - n_tile * p.tiles_m2;
@@ -585,10 +673,10 @@ __global__ void __launch_bounds__(128, 1) mma_pair_probe_kernel(int iters, int32
     if (threadIdx.x >= 32 && threadIdx.x < 64) tmem_dealloc_pair(tmem_base, 256);
 }
 
-template <int LIMBS>
+template <int LIMBS, int NKB, int KPS>
 cudaError_t launch_pair(int grid, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                         const CUtensorMap& tmY, const PairParams& p) {
-    auto kern = qgemm_pair_kernel<LIMBS>;
+    auto kern = qgemm_pair_kernel<LIMBS, NKB, KPS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -608,14 +696,14 @@ cudaError_t launch_pair(int grid, size_t smem, cudaStream_t st, const CUtensorMa
 }
 
 // How many 2-CTA clusters of this kernel the device runs at once (the SM count of a GPC need not be even).
-template <int LIMBS>
+template <int LIMBS, int NKB, int KPS>
 int max_pairs(size_t smem) {
     static int cached[64][2] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return sm_count() / 2;
     int& slot = cached[dev][LIMBS - 1];
     if (slot == 0) {
-        auto kern = qgemm_pair_kernel<LIMBS>;
+        auto kern = qgemm_pair_kernel<LIMBS, NKB, KPS>;
         int n = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(unsigned(sm_count() / 2 * 2)); cfg.blockDim = dim3(unsigned(kPairThreads));
@@ -748,6 +836,14 @@ bool pair_kernel_covers(hq_container cont, const hq_weight_desc* desc, int64_t M
            acc_out == nullptr && ydt == HQ_BF16 && aligned16(y) && (ldy * 2) % 16 == 0 && combine_fast && M >= 256;
 }
 
+// Where the pair kernel is also the faster one: the reductions whose ring stages hold two K blocks (K_pad 256 or 512),
+// on problems with at least two tiles per pair of SMs (below that the one-CTA kernel's 128-row tiles fill the GPU better).
+bool pair_kernel_pays(const hq_weight_desc* desc, int64_t M) {
+    const int num_kb = int(desc->C_pad / kBK);
+    const int64_t tiles = ((M + 255) / 256) * (desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
+    return (num_kb == 2 || num_kb == 4) && tiles >= int64_t(sm_count());
+}
+
 hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
                             const void* w_dev, const float* scale_a, int scale_a_is_scalar, const float* scale_w,
                             const float* bias, float alpha, void* y, int64_t ldy, int32_t* dev_status, cudaStream_t st,
@@ -759,9 +855,10 @@ hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t l
     p.tiles_n = int(desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
     p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
     p.pdl = after_quant ? 1 : 0; p.dev_status = dev_status;
+    const bool whole = p.num_kb == 4 || p.num_kb == 2;     // two K blocks per ring stage (see the kernel)
     size_t smem = 0;
     for (int stages = kPairMaxStages; stages >= 2; --stages) {
-        const PairLayout L = pair_layout(p.num_kb, stages);
+        const PairLayout L = pair_layout(p.num_kb, stages, whole ? 2 : 1);
         if (L.total <= kSmemLimit) { p.stages = stages; smem = size_t(L.total); break; }
     }
     if (smem == 0) return HQ_ERR_UNSUPPORTED;
@@ -771,10 +868,19 @@ hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t l
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
     if (!encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
     const int tiles = p.tiles_m2 * p.tiles_n;
-    const int pairs_max = desc->limbs == 2 ? max_pairs<2>(smem) : max_pairs<1>(smem);
+    const int nkb = whole ? p.num_kb : 0;
+    const bool two = desc->limbs == 2;
+    const int pairs_max = nkb == 4 ? (two ? max_pairs<2, 4, 2>(smem) : max_pairs<1, 4, 2>(smem))
+                        : nkb == 2 ? (two ? max_pairs<2, 2, 2>(smem) : max_pairs<1, 2, 2>(smem))
+                                   : (two ? max_pairs<2, 0, 1>(smem) : max_pairs<1, 0, 1>(smem));
     const int pairs = tiles < pairs_max ? tiles : pairs_max;
-    cudaError_t e = desc->limbs == 2 ? launch_pair<2>(2 * pairs, smem, st, tmA, tmB, tmY, p)
-                                     : launch_pair<1>(2 * pairs, smem, st, tmA, tmB, tmY, p);
+    const int grid = 2 * pairs;
+    cudaError_t e;
+#define HQ_PAIR_GO(L, N, K) launch_pair<L, N, K>(grid, smem, st, tmA, tmB, tmY, p)
+    if (nkb == 4) e = two ? HQ_PAIR_GO(2, 4, 2) : HQ_PAIR_GO(1, 4, 2);
+    else if (nkb == 2) e = two ? HQ_PAIR_GO(2, 2, 2) : HQ_PAIR_GO(1, 2, 2);
+    else e = two ? HQ_PAIR_GO(2, 0, 1) : HQ_PAIR_GO(1, 0, 1);
+#undef HQ_PAIR_GO
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
