@@ -19,6 +19,9 @@ namespace hq {
 namespace {
 using namespace gemm;
 
+#ifndef HQ_PAIR_PREG
+#define HQ_PAIR_PREG 2
+#endif
 constexpr int kPairThreads = 320;              // producer warp, MMA warp, eight epilogue warps
 constexpr int kPairMaxStages = 8;
 constexpr int kPairBBytes = 128 * kBK;         // this CTA's half of a weight K block: 128 rows x 128 bytes
@@ -153,10 +156,15 @@ __device__ __forceinline__ bool wait_pair(uint64_t* bar, uint32_t parity, PairCt
 // The row-per-lane bulk-store epilogue of the one-CTA kernel (16 columns at a time: two tensor-memory loads, 256 * hi + lo,
 // rescale, bf16 into a staging buffer in the 64-byte swizzle of the output tensor map, one bulk tensor store per 32
 // columns), with the accumulator handed back by an arrival on the LEADER's barrier (a cluster address).
-template <int LIMBS>
+// PREG > 0: the column parameters of the warp's first PREG 16-column steps are in registers (`rsw`, `rb`; the caller
+// loads them once per column tile).  Every lane needs all of them, so from shared memory they arrive as broadcast reads,
+// 128 wavefronts per warp and tile, 1024 per tile on the data pipe that also feeds the tensor core its operands (1024 per
+// tile) and takes the staging stores and the bulk stores' reads (520): together more than the 2144 cycles of a tile's MMAs.
+template <int LIMBS, int PREG = 0>
 __device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
                                               const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0, int row0,
-                                              uint32_t tempty_leader) {
+                                              uint32_t tempty_leader, const float (&rsw)[PREG > 0 ? PREG * 16 : 1] = {0.f},
+                                              const float (&rb)[PREG > 0 ? PREG * 16 : 1] = {0.f}) {
     constexpr int NSTEPS = LIMBS == 2 ? kBN / 2 / 2 / 16 : kBN / 2 / 16;
     const uint32_t wsw = (lane >> 1) & 3;
     uint32_t hi[16], lo[16];
@@ -193,7 +201,14 @@ __device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg
         const float4* b4 = reinterpret_cast<const float4*>(prm_b + st * 16);
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            const float4 s0 = sw4[2 * j], s1 = sw4[2 * j + 1], c0 = b4[2 * j], c1 = b4[2 * j + 1];
+            float4 s0, s1, c0, c1;
+            if (st < PREG) {
+                const int e = st * 16 + 8 * j;
+                s0 = make_float4(rsw[e], rsw[e + 1], rsw[e + 2], rsw[e + 3]); s1 = make_float4(rsw[e + 4], rsw[e + 5], rsw[e + 6], rsw[e + 7]);
+                c0 = make_float4(rb[e], rb[e + 1], rb[e + 2], rb[e + 3]); c1 = make_float4(rb[e + 4], rb[e + 5], rb[e + 6], rb[e + 7]);
+            } else {
+                s0 = sw4[2 * j]; s1 = sw4[2 * j + 1]; c0 = b4[2 * j]; c1 = b4[2 * j + 1];
+            }
             uint4 o;
             o.x = pack_bf16x2(fmaf(float(w[8 * j + 0]) * s0.x, sa_eff, c0.x), fmaf(float(w[8 * j + 1]) * s0.y, sa_eff, c0.y));
             o.y = pack_bf16x2(fmaf(float(w[8 * j + 2]) * s0.z, sa_eff, c0.z), fmaf(float(w[8 * j + 3]) * s0.w, sa_eff, c0.w));
@@ -403,6 +418,8 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int last_n = -1;
         bool ok = true;
         float sa_next = 0.f;
+        constexpr int PREG = WHOLE ? HQ_PAIR_PREG : 0;   // steps of 16 columns whose parameters stay in registers
+        float rsw[PREG > 0 ? PREG * 16 : 1], rb[PREG > 0 ? PREG * 16 : 1];
         if (p.pdl) griddep_wait();                    // scale_a comes from the kernel before this one
         for (int i = 0; i < count && ok; ++i) {
             const int u = first + i;
@@ -418,6 +435,10 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     prm_b[cc] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.f;
                 }
                 __syncwarp();
+                if constexpr (PREG > 0) {
+#pragma unroll
+                    for (int e = 0; e < PREG * 16; ++e) { rsw[e] = prm_sw[e]; rb[e] = prm_b[e]; }
+                }
             }
             // the row scale of this tile was requested while the previous tile was processed
             float sa = sa_next;
@@ -437,7 +458,7 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const float sa_eff = p.alpha * sa;
             const int row0 = m2 * 256 + int(rank) * 128 + q * 32;
             const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
-            epilogue_pair<LIMBS>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as]);
+            epilogue_pair<LIMBS, PREG>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as], rsw, rb);
         }
         if (lane == 0) bulk_wait_read_all();           // shared memory must outlive the copy engine's reads
     }
