@@ -56,7 +56,7 @@ def gemm_kernel_name(L):
         return "qgemm_kernel<nibble>"
     if L["kind"] == "conv" or L["K"] > 512:
         return "qgemm_pair_stream_kernel (pairs of SMs, streamed weights)"
-    if L["K"] in (256, 512):
+    if L["K"] == 512 and L.get("limbs", 2) == 2:
         return "qgemm_pair_kernel (pairs of SMs, resident weights, two K blocks per ring stage)"
     return "qgemm_kernel<int8>"
 

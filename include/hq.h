@@ -369,8 +369,8 @@ hq_status hq_qlinear_noalloc(const void* x, hq_dtype xdt, int64_t M, int64_t K, 
  *   0  nowhere;
  *   1  wherever a pair kernel covers the problem (also K_pad 128 or 384 and problems of few tiles, where it measures level
  *      or slower);
- *   2  (default) where it measured faster: reductions with streamed weights (K_pad > 512), convolutions, and K_pad 256 or
- *      512 on problems of at least one 256-row tile per SM.
+ *   2  (default) where it measured faster: reductions with streamed weights (K_pad > 512), convolutions, and two-limb
+ *      weights at K_pad 512 on problems of at least one 256-row tile per SM.
  * Results are bit-identical in every mode.  Returns the previous mode.  Process-wide, not thread-safe. */
 int hq_set_pair_gemm(int mode);
 

@@ -857,12 +857,13 @@ bool pair_kernel_covers(hq_container cont, const hq_weight_desc* desc, int64_t M
            acc_out == nullptr && ydt == HQ_BF16 && aligned16(y) && (ldy * 2) % 16 == 0 && combine_fast && M >= 256;
 }
 
-// Where the pair kernel is also the faster one: the reductions whose ring stages hold two K blocks (K_pad 256 or 512),
-// on problems with at least two tiles per pair of SMs (below that the one-CTA kernel's 128-row tiles fill the GPU better).
+// Where the pair kernel is also the faster one: two-limb weights at K_pad = 512 (the epilogue's share of a tile is
+// smallest there) on problems with at least one 256-row tile per SM.  With one limb or at K_pad = 256 a tile has as much
+// epilogue as MMA work and the shape sweep measured the one-CTA kernel level or up to 15 % faster.
 bool pair_kernel_pays(const hq_weight_desc* desc, int64_t M) {
     const int num_kb = int(desc->C_pad / kBK);
-    const int64_t tiles = ((M + 255) / 256) * (desc->limbs == 2 ? desc->N_pad / 128 : (desc->N_pad + 255) / 256);
-    return (num_kb == 2 || num_kb == 4) && tiles >= int64_t(sm_count());
+    const int64_t tiles = ((M + 255) / 256) * (desc->N_pad / 128);
+    return desc->limbs == 2 && num_kb == 4 && tiles >= int64_t(sm_count());
 }
 
 hq_status launch_qgemm_pair(const void* a_codes, int64_t M, int64_t K, int64_t lda, const hq_weight_desc* desc,
