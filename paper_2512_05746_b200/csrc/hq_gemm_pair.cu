@@ -4,10 +4,12 @@
 // operand-B rows in its shared memory (with two weight limbs: one CTA the "hi" rows, the other the "lo" rows), one lane of
 // the leader CTA issues every MMA for both tensor cores, and each CTA's tensor memory receives the 128 x 256 accumulator of
 // its own rows.  Per SM and MMA the tensor core reads 8 KB of operands from its shared memory instead of 12 KB -- the
-// shared-memory data pipe, not the tensor pipe, is what bounds the one-CTA kernel on short reductions -- and the resident
-// weight tile shrinks to 64 KB, which leaves room for an activation ring of eight stages.
+// shared-memory data pipe is the busiest unit of the one-CTA kernel on short reductions -- and the resident weight tile
+// shrinks to 64 KB, which leaves room for an activation ring of eight 16 KB stages, or of three 32 KB stages (two K blocks
+// each, K_pad 256 / 512: half the barrier rounds for the issuing lane).
 //
-// Covered: plain GEMM, one code per byte, K_pad <= 512 (weights resident), bf16 output through bulk tensor stores.
+// Covered: plain GEMM, one code per byte, K_pad <= 512 (weights resident), bf16 output through bulk tensor stores; below
+// this kernel, the same protocol with streamed weights for longer reductions and convolutions.
 // Every CTA issues its own TMA loads (no multicast); the loads of the second CTA signal the leader's barriers; MMA
 // completion is committed to both CTAs' barriers; the second CTA's epilogue warps release the accumulators with remote
 // barrier arrivals.  Every wait is bounded.
@@ -19,9 +21,9 @@ namespace hq {
 namespace {
 using namespace gemm;
 
-#ifndef HQ_PAIR_PREG
-#define HQ_PAIR_PREG 2
-#endif
+// 16-column epilogue steps whose column parameters stay in registers in the kernels with two K blocks per ring stage
+// (two of a two-limb warp's four: 64 registers; with three the kernel spills and measured slower).
+constexpr int kPairRegSteps = 2;
 constexpr int kPairThreads = 320;              // producer warp, MMA warp, eight epilogue warps
 constexpr int kPairMaxStages = 8;
 constexpr int kPairBBytes = 128 * kBK;         // this CTA's half of a weight K block: 128 rows x 128 bytes
@@ -418,7 +420,7 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int last_n = -1;
         bool ok = true;
         float sa_next = 0.f;
-        constexpr int PREG = WHOLE ? HQ_PAIR_PREG : 0;   // steps of 16 columns whose parameters stay in registers
+        constexpr int PREG = WHOLE ? kPairRegSteps : 0;
         float rsw[PREG > 0 ? PREG * 16 : 1], rb[PREG > 0 ? PREG * 16 : 1];
         if (p.pdl) griddep_wait();                    // scale_a comes from the kernel before this one
         for (int i = 0; i < count && ok; ++i) {
