@@ -162,7 +162,8 @@ __device__ __forceinline__ bool wait_pair(uint64_t* bar, uint32_t parity, PairCt
 // loads them once per column tile).  Every lane needs all of them, so from shared memory they arrive as broadcast reads,
 // 128 wavefronts per warp and tile, 1024 per tile on the data pipe that also feeds the tensor core its operands (1024 per
 // tile) and takes the staging stores and the bulk stores' reads (520): together more than the 2144 cycles of a tile's MMAs.
-template <int LIMBS, int PREG = 0>
+// NBUF: the warp's staging buffers (two used in turn, or one).
+template <int LIMBS, int PREG = 0, int NBUF = 2>
 __device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg, int lane, const float* prm_sw,
                                               const float* prm_b, float sa_eff, const CUtensorMap* tmY, int col0, int row0,
                                               uint32_t tempty_leader, const float (&rsw)[PREG > 0 ? PREG * 16 : 1] = {0.f},
@@ -193,10 +194,10 @@ __device__ __forceinline__ void epilogue_pair(uint32_t t_row, unsigned char* stg
             if (lane == 0) mbar_arrive_cluster(tempty_leader);
         }
         // two staging buffers, used in turn: the copy engine must be done reading the one written two stores ago
-        unsigned char* buf = stg + ((st >> 1) & 1) * kStagingBytes;
+        unsigned char* buf = NBUF == 2 ? stg + ((st >> 1) & 1) * kStagingBytes : stg;
         unsigned char* wr = buf + lane * 64;
         if ((st & 1) == 0) {
-            if (lane == 0) bulk_wait_read_1();
+            if (lane == 0) { if (NBUF == 2) bulk_wait_read_1(); else bulk_wait_read_all(); }
             __syncwarp();
         }
         const float4* sw4 = reinterpret_cast<const float4*>(prm_sw + st * 16);
@@ -493,11 +494,12 @@ struct PairStreamParams {
 constexpr int kPairStageBytes = kABytes + kPairBBytes;      // 32 KB: this CTA's activation rows and its half of the weights
 
 struct PairStreamLayout { int ring_off, staging_off, param_off, ctl_off, total; };
-__host__ __device__ inline PairStreamLayout pair_stream_layout(int stages) {
+// kps: K blocks per ring stage; with two, 64 KB stages, the epilogue warps have one staging buffer each instead of two
+__host__ __device__ inline PairStreamLayout pair_stream_layout(int stages, int kps = 1) {
     PairStreamLayout L;
     L.ring_off = 0;
-    L.staging_off = stages * kPairStageBytes;
-    L.param_off = L.staging_off + kEpiWarps * 2 * kStagingBytes;
+    L.staging_off = stages * kps * kPairStageBytes;
+    L.param_off = L.staging_off + kEpiWarps * (kps == 2 ? 1 : 2) * kStagingBytes;
     L.ctl_off = L.param_off + kPairParamBytes;
     L.total = L.ctl_off + int(sizeof(PairCtl)) + 1024;
     return L;
@@ -512,13 +514,15 @@ __device__ __forceinline__ void tma_load_4d_pair(void* smem_dst, const void* tma
         : "memory");
 }
 
-template <int LIMBS, bool CONV>
+// KPS = 2 (even K block counts): two K blocks per ring stage, laid out [A0 | B0 | A1 | B1]: the issuing lane's barrier
+// rounds halve (a wait, a fence, eight MMAs and a commit per 64 KB stage); three stages fit.
+template <int LIMBS, bool CONV, int KPS>
 __global__ void __launch_bounds__(kPairThreads, 1)
 qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmY, const PairStreamParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const PairStreamLayout L = pair_stream_layout(p.stages);
+    const PairStreamLayout L = pair_stream_layout(p.stages, KPS);
     unsigned char* sRing = smem + L.ring_off;
     unsigned char* sStage = smem + L.staging_off;
     float* sParam = reinterpret_cast<float*>(smem + L.param_off);
@@ -563,19 +567,23 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     const int tn = m_tile / (p.tiles_w * p.tiles_h);
                     w0 = tw * p.bw; h0 = th * p.bh; n0 = tn * p.bn;      // past the last image: the load delivers zeros
                 }
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb0 = 0; kb0 < num_kb; kb0 += KPS) {
                     if (!wait_pair(&ctl->empty[stage], phase ^ 1, ctl, p.dev_status, kStatusEmptyWait)) { ok = false; break; }
                     const uint32_t fbar = map_to_cta(&ctl->full[stage], 0);
-                    if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(kPairStageBytes));
-                    unsigned char* dst = sRing + stage * kPairStageBytes;
-                    if (CONV) {
-                        const int tap = kb / p.kb_per_tap, kc = kb - tap * p.kb_per_tap;
-                        const int r = tap / p.S, s = tap - r * p.S;
-                        tma_load_4d_pair(dst, &tmA, fbar, kc * kBK, w0 * p.stride + s - p.pad, h0 * p.stride + r - p.pad, n0);
-                    } else {
-                        tma_load_2d_pair(dst, &tmA, fbar, kb * kBK, m_tile * kBM);
+                    if (rank == 0) mbar_expect_tx(&ctl->full[stage], 2u * uint32_t(KPS * kPairStageBytes));
+#pragma unroll
+                    for (int k = 0; k < KPS; ++k) {
+                        const int kb = kb0 + k;
+                        unsigned char* dst = sRing + (stage * KPS + k) * kPairStageBytes;
+                        if (CONV) {
+                            const int tap = kb / p.kb_per_tap, kc = kb - tap * p.kb_per_tap;
+                            const int r = tap / p.S, s = tap - r * p.S;
+                            tma_load_4d_pair(dst, &tmA, fbar, kc * kBK, w0 * p.stride + s - p.pad, h0 * p.stride + r - p.pad, n0);
+                        } else {
+                            tma_load_2d_pair(dst, &tmA, fbar, kb * kBK, m_tile * kBM);
+                        }
+                        tma_load_2d_pair(dst + kABytes, &tmB, fbar, kb * kBK, n_tile * kBN + int(rank) * 128);
                     }
-                    tma_load_2d_pair(dst + kABytes, &tmB, fbar, kb * kBK, n_tile * kBN + int(rank) * 128);
                     if (++stage == nstages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -588,7 +596,7 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             // weights 1024 units behind the activations), and only the very first MMA of a tile overwrites.
             const uint32_t idesc = make_idesc_i8(256, kBN);
             const uint64_t desc0 = make_sw128_kmajor_desc(smem_u32(sRing));
-            constexpr uint64_t kStageUnits = kPairStageBytes >> 4, kBUnits = kABytes >> 4;
+            constexpr uint64_t kBlockUnits = kPairStageBytes >> 4, kStageUnits = KPS * kBlockUnits, kBUnits = kABytes >> 4;
             uint64_t a_desc = desc0;
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
@@ -598,7 +606,7 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + uint32_t(as * kBN);
                 uint32_t acc = 0;                          // 0 for the first MMA of the tile only
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < num_kb; kb += KPS) {
                     if (!wait_pair(&ctl->full[stage], phase, ctl, p.dev_status, kStatusTmaWait)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t b_desc = a_desc + kBUnits;
@@ -606,6 +614,12 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
                     mma_i8_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
                     mma_i8_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
                     mma_i8_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+                    if (KPS == 2) {
+                        mma_i8_pair(d_tmem, a_desc + kBlockUnits, b_desc + kBlockUnits, idesc, 1u);
+                        mma_i8_pair(d_tmem, a_desc + (kBlockUnits + 2), b_desc + (kBlockUnits + 2), idesc, 1u);
+                        mma_i8_pair(d_tmem, a_desc + (kBlockUnits + 4), b_desc + (kBlockUnits + 4), idesc, 1u);
+                        mma_i8_pair(d_tmem, a_desc + (kBlockUnits + 6), b_desc + (kBlockUnits + 6), idesc, 1u);
+                    }
                     acc = 1u;
                     mma_commit_pair(&ctl->empty[stage]);
                     a_desc += kStageUnits;
@@ -620,7 +634,8 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
         const int ew = warp - 2;
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         const int chalf = ew >> 2;                    // which half of the tile's columns this warp takes
-        unsigned char* stg = sStage + ew * 2 * kStagingBytes;
+        constexpr int NBUF = KPS == 2 ? 1 : 2;
+        unsigned char* stg = sStage + ew * NBUF * kStagingBytes;
         float* prm_sw = sParam + ew * 2 * (kBN / 2);
         float* prm_b = prm_sw + kBN / 2;
         constexpr int cols_per_tile = LIMBS == 2 ? kBN / 2 : kBN;
@@ -652,7 +667,7 @@ qgemm_pair_stream_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_c
             const float sa_eff = p.alpha * sa;
             const int row0 = m2 * 256 + int(rank) * 128 + q * 32;
             const uint32_t t_fast = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(as * kBN + wc0);
-            epilogue_pair<LIMBS>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as]);
+            epilogue_pair<LIMBS, 0, NBUF>(t_fast, stg, lane, prm_sw, prm_b, sa_eff, &tmY, col_base + wc0, row0, tempty_leader[as]);
         }
         if (lane == 0) bulk_wait_read_all();           // shared memory must outlive the copy engine's reads
     }
@@ -743,10 +758,10 @@ int max_pairs(size_t smem) {
     return slot;
 }
 
-template <int LIMBS, bool CONV>
+template <int LIMBS, bool CONV, int KPS>
 cudaError_t launch_pair_stream(int pairs_wanted, size_t smem, cudaStream_t st, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                const CUtensorMap& tmY, const PairStreamParams& p) {
-    auto kern = qgemm_pair_stream_kernel<LIMBS, CONV>;
+    auto kern = qgemm_pair_stream_kernel<LIMBS, CONV, KPS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
@@ -782,9 +797,9 @@ cudaError_t launch_pair_stream(int pairs_wanted, size_t smem, cudaStream_t st, c
     return cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
 }
 
-bool pair_stream_stages(PairStreamParams& p, size_t& smem) {
+bool pair_stream_stages(PairStreamParams& p, size_t& smem, int kps) {
     for (int stages = kPairMaxStages; stages >= 3; --stages) {
-        const PairStreamLayout L = pair_stream_layout(stages);
+        const PairStreamLayout L = pair_stream_layout(stages, kps);
         if (L.total <= kSmemLimit) { p.stages = stages; smem = size_t(L.total); return true; }
     }
     return false;
@@ -816,15 +831,15 @@ hq_status launch_qgemm_pair_stream(const void* a_codes, int64_t M, int64_t K, in
     p.scale_a = scale_a; p.sa_scalar = scale_a_is_scalar; p.scale_w = scale_w; p.bias = bias; p.alpha = alpha;
     p.pdl = after_quant ? 1 : 0; p.dev_status = dev_status;
     size_t smem = 0;
-    if (!pair_stream_stages(p, smem)) return HQ_ERR_UNSUPPORTED;
+    if (!pair_stream_stages(p, smem, 1)) return HQ_ERR_UNSUPPORTED;    // two K blocks per stage measured 2 % slower here
     CUtensorMap tmA, tmB, tmY;
     if (!encode_2d(&tmA, a_codes, uint64_t(K), uint64_t(M), uint64_t(lda), kBK, kBM, true)) return HQ_ERR_CUDA;
     const uint64_t Kp = uint64_t(desc->C_pad);
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
     if (!encode_y(&tmY, y, uint64_t(desc->N), uint64_t(M), uint64_t(ldy))) return HQ_ERR_CUDA;
     const int tiles = p.tiles_m2 * p.tiles_n;
-    cudaError_t e = desc->limbs == 2 ? launch_pair_stream<2, false>(tiles, smem, st, tmA, tmB, tmY, p)
-                                     : launch_pair_stream<1, false>(tiles, smem, st, tmA, tmB, tmY, p);
+    cudaError_t e = desc->limbs == 2 ? launch_pair_stream<2, false, 1>(tiles, smem, st, tmA, tmB, tmY, p)
+                                     : launch_pair_stream<1, false, 1>(tiles, smem, st, tmA, tmB, tmY, p);
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
@@ -842,13 +857,17 @@ hq_status launch_qconv_pair(const gemm::GemmParams& g, const CUtensorMap& tmA, c
     p.kb_per_tap = g.kb_per_tap; p.S = g.S; p.stride = g.stride; p.pad = g.pad;
     p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.tiles_w = g.tiles_w; p.tiles_h = g.tiles_h;
     size_t smem = 0;
-    if (!pair_stream_stages(p, smem)) return HQ_ERR_UNSUPPORTED;
+    const int kps = p.num_kb % 2 == 0 ? 2 : 1;      // two K blocks per ring stage: 6 % faster on the 3x3 convolutions
+    if (!pair_stream_stages(p, smem, kps)) return HQ_ERR_UNSUPPORTED;
     CUtensorMap tmB;
     const uint64_t Kp = uint64_t(desc->C_pad) * desc->RS;
     if (!encode_2d(&tmB, w_dev, Kp, uint64_t(desc->N_pad) * desc->limbs, Kp, kBK, 128, true)) return HQ_ERR_CUDA;
     const int tiles = p.tiles_m2 * p.tiles_n;
-    cudaError_t e = desc->limbs == 2 ? launch_pair_stream<2, true>(tiles, smem, st, tmA, tmB, tmY, p)
-                                     : launch_pair_stream<1, true>(tiles, smem, st, tmA, tmB, tmY, p);
+    cudaError_t e;
+    if (kps == 2) e = desc->limbs == 2 ? launch_pair_stream<2, true, 2>(tiles, smem, st, tmA, tmB, tmY, p)
+                                       : launch_pair_stream<1, true, 2>(tiles, smem, st, tmA, tmB, tmY, p);
+    else e = desc->limbs == 2 ? launch_pair_stream<2, true, 1>(tiles, smem, st, tmA, tmB, tmY, p)
+                              : launch_pair_stream<1, true, 1>(tiles, smem, st, tmA, tmB, tmY, p);
     return e == cudaSuccess ? HQ_OK : HQ_ERR_CUDA;
 }
 
