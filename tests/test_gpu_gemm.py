@@ -309,6 +309,7 @@ PAIR_CASES = [
     (777, 512, 328, 512, "plain"),        # one weight limb, ragged columns
     (300, 128, 72, 128, "folded"),        # one K block
     (40000, 256, 384, 256, "double"),     # more pair tiles than clusters; the weight tile changes inside a pair's range
+    (40000, 512, 384, 512, "folded"),     # the same with four K blocks and two limbs: what the default dispatch sends to pairs
     (256, 384, 136, 128, "folded"),       # three K blocks
     # reductions beyond the resident weight tile: weights streamed through the pair's ring
     (1000, 1024, 384, 1024, "folded"),    # eight K blocks, ragged rows, three column tiles
@@ -341,6 +342,9 @@ def test_qgemm_on_sm_pairs_matches_oracle(env, oracle, M, K, N, n, mode):
         hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_one, dev_status=status)
         hq.hq_set_pair_gemm(1)
         hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_pair, dev_status=status)
+        hq.hq_set_pair_gemm(2)                 # the default: whichever kernel the library picks for this shape
+        y_def = torch.full((M, N), 5.0, dtype=torch.bfloat16, device="cuda")
+        hq.hq_qgemm(a_dev, 1, 4, K, pw, scale_a=sa_dev, bias=b_dev, alpha=pw.alpha, y=y_def, dev_status=status)
         torch.cuda.synchronize()
     finally:
         hq.hq_set_pair_gemm(before)
@@ -348,6 +352,7 @@ def test_qgemm_on_sm_pairs_matches_oracle(env, oracle, M, K, N, n, mode):
     y_ref = oracle.dequant(oracle.gemm_int(q, B), s_a, pw.s_w, b, pw.alpha)
     assert rel_err(y_pair.float().cpu().numpy(), y_ref) <= Y_BF16_RTOL
     assert torch.equal(y_pair, y_one)
+    assert torch.equal(y_def, y_one)
 
 
 def test_paired_tensor_pipe_probe_runs(env):
