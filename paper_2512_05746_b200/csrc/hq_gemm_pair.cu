@@ -253,10 +253,21 @@ qgemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();                 // 0: leader (issues the MMAs), 1: its peer
     const int nstages = p.stages, num_kb = p.num_kb;
-    // the pair's contiguous range of 256-row tiles in column-tile-major order (consecutive tiles share their weights)
-    const int T = p.tiles_m2 * p.tiles_n, G = gridDim.x >> 1, c = blockIdx.x >> 1;
-    const int first = int(int64_t(c) * T / G);
-    const int count = int(int64_t(c + 1) * T / G) - first;
+    // the pair's contiguous range of 256-row tiles in column-tile-major order (consecutive tiles share their weights).
+    // A change of weight tile inside a range stalls the pair for about one tile (the old tile's MMAs drain, then 64 KB
+    // per CTA arrive), and the slowest pair sets the kernel's time: the ranges are cut in units of cost, a column tile
+    // costing its row tiles plus one, so that a pair that changes weights gets one tile fewer.
+    const int G = gridDim.x >> 1, c = blockIdx.x >> 1;
+    const int W = p.tiles_m2 + 1;
+    const int64_t C = int64_t(p.tiles_n) * W;
+    auto first_tile = [&](int pair) {
+        const int64_t lo = (int64_t(pair) * C + G - 1) / G;        // first cost position of the pair
+        int n = int(lo / W), m = int(lo - int64_t(n) * W);
+        if (m == p.tiles_m2) { ++n; m = 0; }                        // the slot that stands for the weight change
+        return n * p.tiles_m2 + m;
+    };
+    const int first = first_tile(c);
+    const int count = first_tile(c + 1) - first;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPairMaxStages; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
